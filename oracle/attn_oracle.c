@@ -1,0 +1,223 @@
+/*
+ * attn_oracle.c -- TEST INFRASTRUCTURE, not product code.
+ *
+ * Plain fp64 CPU statement of the attention operator of Section 2.2 of the paper:
+ *
+ *     Attention(Q, K, V) = Softmax(Mask(Q K^T / sqrt(d))) V
+ *
+ * written out as the definition: one score row at a time, a max, a sum of
+ * exponentials, a weighted sum of V rows.  No tiling, no online softmax, no
+ * exp2, no blocking.  FlashAttention-style kernels are an exact reformulation
+ * of this (up to rounding order), so the definition is the oracle.
+ *
+ * Readings where the paper is silent (each is stated again in the design notes):
+ *   - scale is an explicit argument (the paper uses 1/sqrt(d));
+ *   - the causal mask is lower-triangular including the diagonal and aligned
+ *     to the top-left corner: key j is visible to query i iff j <= i, also
+ *     when Sq != Sk;
+ *   - the per-row logsumexp is the natural log of the sum of exponentials of
+ *     the SCALED visible scores;
+ *   - a row with no visible key gives O = 0 and LSE = -inf.
+ *
+ * Only tests, the smoke check and the benchmark's cpu_baseline leg may call
+ * this file.  It shares nothing with the CUDA path.
+ *
+ * Build:  gcc -O2 -fopenmp -shared -fPIC -o liboracle.so attn_oracle.c -lm
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---- 16-bit storage formats -> double (exact widening) ------------------ */
+
+/* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+double oracle_f16_bits_to_f64(uint16_t h)
+{
+    int sign = (h >> 15) & 1;
+    int e = (h >> 10) & 0x1f;
+    int f = h & 0x3ff;
+    double mag;
+    if (e == 0)
+        mag = ldexp((double)f, -24); /* subnormal: f * 2^-10 * 2^-14 */
+    else if (e == 31)
+        mag = f ? NAN : INFINITY;
+    else
+        mag = ldexp(1.0 + (double)f / 1024.0, e - 15);
+    return sign ? -mag : mag;
+}
+
+/* bfloat16: 1 sign, 8 exponent (bias 127), 7 fraction bits. */
+double oracle_bf16_bits_to_f64(uint16_t h)
+{
+    int sign = (h >> 15) & 1;
+    int e = (h >> 7) & 0xff;
+    int f = h & 0x7f;
+    double mag;
+    if (e == 0)
+        mag = ldexp((double)f, -133); /* subnormal: f * 2^-7 * 2^-126 */
+    else if (e == 255)
+        mag = f ? NAN : INFINITY;
+    else
+        mag = ldexp(1.0 + (double)f / 128.0, e - 127);
+    return sign ? -mag : mag;
+}
+
+/* dtype: 0 = binary16, 1 = bfloat16 (same numbering as the library's enum,
+ * restated here because the two sides share no header). */
+void oracle_widen(const uint16_t *src, double *dst, int64_t n, int dtype)
+{
+    int64_t i;
+#pragma omp parallel for schedule(static)
+    for (i = 0; i < n; ++i)
+        dst[i] = dtype == 0 ? oracle_f16_bits_to_f64(src[i]) : oracle_bf16_bits_to_f64(src[i]);
+}
+
+/* ---- one query row ------------------------------------------------------ */
+
+/* q: [D]; k, v: [Sk, D] of the row's (batch, head); s: scratch of Sk doubles.
+ * n_vis = number of visible keys (keys 0 .. n_vis-1).  Writes o[D], *lse and,
+ * when prowsum != NULL, the sum of the row's probabilities. */
+static void attn_row(const double *q, const double *k, const double *v, double *s, double *o,
+                     double *lse, double *prowsum, int64_t n_vis, int D, double scale)
+{
+    int64_t j;
+    int d;
+    if (n_vis <= 0) {
+        for (d = 0; d < D; ++d)
+            o[d] = 0.0;
+        *lse = -INFINITY;
+        if (prowsum)
+            *prowsum = 0.0;
+        return;
+    }
+    /* s_j = scale * <q, k_j> */
+    double m = -INFINITY;
+    for (j = 0; j < n_vis; ++j) {
+        double acc = 0.0;
+        for (d = 0; d < D; ++d)
+            acc += q[d] * k[j * D + d];
+        s[j] = scale * acc;
+        if (s[j] > m)
+            m = s[j];
+    }
+    /* e_j = exp(s_j - m),  l = sum_j e_j */
+    double l = 0.0;
+    for (j = 0; j < n_vis; ++j) {
+        s[j] = exp(s[j] - m);
+        l += s[j];
+    }
+    /* p_j = e_j / l,  o = sum_j p_j v_j */
+    for (d = 0; d < D; ++d)
+        o[d] = 0.0;
+    double psum = 0.0;
+    for (j = 0; j < n_vis; ++j) {
+        double p = s[j] / l;
+        psum += p;
+        for (d = 0; d < D; ++d)
+            o[d] += p * v[j * D + d];
+    }
+    *lse = m + log(l);
+    if (prowsum)
+        *prowsum = psum;
+}
+
+static int64_t visible_keys(int64_t i, int64_t Sk, int causal)
+{
+    if (!causal)
+        return Sk;
+    return (i + 1 < Sk) ? i + 1 : Sk;
+}
+
+/* ---- whole problem ------------------------------------------------------ */
+
+/* q: [B,H,Sq,D], k,v: [B,H,Sk,D], o: [B,H,Sq,D], lse: [B,H,Sq],
+ * prowsum: [B,H,Sq] or NULL.  All row-major contiguous doubles on the host.
+ * Returns 0, or -1 when scratch cannot be allocated. */
+int attn_oracle_f64(const double *q, const double *k, const double *v, double *o, double *lse,
+                    double *prowsum, int B, int H, int Sq, int Sk, int D, double scale, int causal)
+{
+    int64_t rows = (int64_t)B * H * Sq;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(Sk > 0 ? Sk : 1));
+        if (!s) {
+#pragma omp atomic write
+            failed = 1;
+        }
+        int64_t r;
+#pragma omp for schedule(dynamic, 16)
+        for (r = 0; r < rows; ++r) {
+            if (!s)
+                continue;
+            int64_t bh = r / Sq, i = r % Sq;
+            attn_row(q + r * D, k + bh * Sk * D, v + bh * Sk * D, s, o + r * D, lse + r,
+                     prowsum ? prowsum + r : NULL, visible_keys(i, Sk, causal), D, scale);
+        }
+        free(s);
+    }
+    return failed ? -1 : 0;
+}
+
+/* Same arithmetic for a chosen subset of rows, reading the 16-bit inputs
+ * directly (widened exactly, element by element) so that full-size problems
+ * need no fp64 copy of Q, K, V.
+ * rows[n_rows]: flat row indices r = (b*H + h)*Sq + i.
+ * o: [n_rows, D], lse: [n_rows]. */
+int attn_oracle_rows_16(const uint16_t *q, const uint16_t *k, const uint16_t *v, int dtype,
+                        const int64_t *rows, int64_t n_rows, double *o, double *lse, int B, int H,
+                        int Sq, int Sk, int D, double scale, int causal)
+{
+    int failed = 0;
+    (void)B;
+    (void)H;
+#pragma omp parallel
+    {
+        size_t nk = (size_t)(Sk > 0 ? Sk : 1);
+        double *s = (double *)malloc(sizeof(double) * nk);
+        double *qd = (double *)malloc(sizeof(double) * (size_t)D);
+        double *kd = (double *)malloc(sizeof(double) * nk * (size_t)D);
+        double *vd = (double *)malloc(sizeof(double) * nk * (size_t)D);
+        if (!s || !qd || !kd || !vd) {
+#pragma omp atomic write
+            failed = 1;
+        }
+        int64_t t;
+#pragma omp for schedule(dynamic, 1)
+        for (t = 0; t < n_rows; ++t) {
+            if (!s || !qd || !kd || !vd)
+                continue;
+            int64_t r = rows[t];
+            int64_t bh = r / Sq, i = r % Sq;
+            int64_t n_vis = visible_keys(i, Sk, causal);
+            int64_t e;
+            for (e = 0; e < D; ++e)
+                qd[e] = dtype == 0 ? oracle_f16_bits_to_f64(q[r * D + e])
+                                   : oracle_bf16_bits_to_f64(q[r * D + e]);
+            for (e = 0; e < n_vis * D; ++e) {
+                uint16_t kb = k[bh * Sk * D + e], vb = v[bh * Sk * D + e];
+                kd[e] = dtype == 0 ? oracle_f16_bits_to_f64(kb) : oracle_bf16_bits_to_f64(kb);
+                vd[e] = dtype == 0 ? oracle_f16_bits_to_f64(vb) : oracle_bf16_bits_to_f64(vb);
+            }
+            attn_row(qd, kd, vd, s, o + t * D, lse + t, NULL, n_vis, D, scale);
+        }
+        free(s);
+        free(qd);
+        free(kd);
+        free(vd);
+    }
+    return failed ? -1 : 0;
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

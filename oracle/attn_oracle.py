@@ -1,0 +1,125 @@
+"""ctypes front end of the fp64 CPU oracle (oracle/attn_oracle.c).
+
+TEST INFRASTRUCTURE, not product code: only tests, the smoke check and the
+benchmark's cpu_baseline / reference legs may import this module.  It imports
+nothing from the CUDA package.
+
+The arithmetic lives in the C file (Section 2.2 of the paper, written out as
+the definition); this module only compiles it with gcc, loads it and passes
+numpy arrays through.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "attn_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+DTYPE_FP16 = 0
+DTYPE_BF16 = 1
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP) if the shared object is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        dp = ctypes.POINTER(ctypes.c_double)
+        u16p = ctypes.POINTER(ctypes.c_uint16)
+        i64p = ctypes.POINTER(ctypes.c_int64)
+        lib.attn_oracle_f64.restype = ctypes.c_int
+        lib.attn_oracle_f64.argtypes = [dp, dp, dp, dp, dp, dp] + [ctypes.c_int] * 5 + [
+            ctypes.c_double, ctypes.c_int]
+        lib.attn_oracle_rows_16.restype = ctypes.c_int
+        lib.attn_oracle_rows_16.argtypes = [u16p, u16p, u16p, ctypes.c_int, i64p, ctypes.c_int64,
+                                            dp, dp] + [ctypes.c_int] * 5 + [ctypes.c_double,
+                                                                            ctypes.c_int]
+        lib.oracle_widen.restype = None
+        lib.oracle_widen.argtypes = [u16p, dp, ctypes.c_int64, ctypes.c_int]
+        lib.oracle_num_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _dptr(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _u16ptr(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_uint16))
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def widen(bits: np.ndarray, dtype: int) -> np.ndarray:
+    """Exact widening of fp16 (dtype 0) / bf16 (dtype 1) bit patterns (uint16) to float64."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    out = np.empty(bits.shape, dtype=np.float64)
+    _load().oracle_widen(_u16ptr(bits), _dptr(out), bits.size, int(dtype))
+    return out
+
+
+def attention(q, k, v, scale: float, causal: bool, return_rowsum: bool = False):
+    """O, LSE (and optionally the row sums of the probabilities) for float64 arrays.
+
+    q: [B,H,Sq,D]; k, v: [B,H,Sk,D].  Returns o [B,H,Sq,D], lse [B,H,Sq].
+    """
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    k = np.ascontiguousarray(k, dtype=np.float64)
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    B, H, Sq, D = q.shape
+    Sk = k.shape[2]
+    assert k.shape == (B, H, Sk, D) and v.shape == (B, H, Sk, D)
+    o = np.empty((B, H, Sq, D), dtype=np.float64)
+    lse = np.empty((B, H, Sq), dtype=np.float64)
+    rs = np.empty((B, H, Sq), dtype=np.float64) if return_rowsum else None
+    rc = _load().attn_oracle_f64(_dptr(q), _dptr(k), _dptr(v), _dptr(o), _dptr(lse),
+                                 _dptr(rs) if rs is not None else None,
+                                 B, H, Sq, Sk, D, float(scale), int(bool(causal)))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return (o, lse, rs) if return_rowsum else (o, lse)
+
+
+def attention_rows_16(q_bits, k_bits, v_bits, dtype: int, rows, scale: float, causal: bool):
+    """Oracle for a chosen subset of rows, straight from 16-bit inputs.
+
+    q_bits: uint16 [B,H,Sq,D]; k_bits, v_bits: uint16 [B,H,Sk,D]; rows: flat
+    row indices (b*H + h)*Sq + i.  Returns o [n,D] and lse [n] in float64.
+    """
+    q_bits = np.ascontiguousarray(q_bits, dtype=np.uint16)
+    k_bits = np.ascontiguousarray(k_bits, dtype=np.uint16)
+    v_bits = np.ascontiguousarray(v_bits, dtype=np.uint16)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    B, H, Sq, D = q_bits.shape
+    Sk = k_bits.shape[2]
+    assert k_bits.shape == (B, H, Sk, D) and v_bits.shape == (B, H, Sk, D)
+    assert rows.size == 0 or (rows.min() >= 0 and rows.max() < B * H * Sq)
+    o = np.empty((rows.size, D), dtype=np.float64)
+    lse = np.empty((rows.size,), dtype=np.float64)
+    rc = _load().attn_oracle_rows_16(
+        _u16ptr(q_bits), _u16ptr(k_bits), _u16ptr(v_bits), int(dtype),
+        rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), rows.size, _dptr(o), _dptr(lse),
+        B, H, Sq, Sk, D, float(scale), int(bool(causal)))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return o, lse

@@ -1,0 +1,271 @@
+"""Pins for the fp64 CPU oracle (CPU only).
+
+Each test holds the oracle against something other than itself: hand-derived
+cases, closed forms, invariants of the definition in Section 2.2 of the paper,
+a separately written dense brute force, and torch's fp64 library attention.
+A plausible mistake anywhere in the oracle (dropped scale, wrong sign, base-2
+log, transposed K, off-by-one causal edge, un-normalised P) fails at least one.
+"""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import attn_oracle as orc
+from paper_2506_12355_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "hand_cases.json")
+
+
+def rand(shape, seed, sigma=1.0):
+    return np.random.default_rng(seed).normal(0.0, sigma, size=shape)
+
+
+# ------------------------------------------------------------------ converters
+
+def test_fp16_widening_all_patterns():
+    allbits = np.arange(65536, dtype=np.uint16)
+    got = orc.widen(allbits, orc.DTYPE_FP16)
+    want = allbits.view(np.float16).astype(np.float64)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan], want[~nan])
+    assert np.array_equal(np.signbit(got[~nan]), np.signbit(want[~nan]))
+
+
+def test_bf16_widening_all_patterns():
+    allbits = np.arange(65536, dtype=np.uint16)
+    got = orc.widen(allbits, orc.DTYPE_BF16)
+    # a bf16 is the upper half of an fp32
+    with np.errstate(invalid="ignore"):
+        want = (allbits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan], want[~nan])
+    t = torch.from_numpy(allbits.view(np.int16).copy()).view(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(got[~nan], t[~nan])
+
+
+# ------------------------------------------------------------------ hand cases
+
+def _ev(x):
+    if isinstance(x, (int, float)):
+        return float(x)
+    env = {"e": math.e, "ln": math.log}
+    s = x
+    for name in ("ln2", "ln3", "ln4", "ln6", "ln8"):
+        s = s.replace(name, "ln(%s)" % name[2:])
+    return float(eval(s, {"__builtins__": {}}, env))
+
+
+def _mat(m):
+    return np.array([[_ev(x) for x in row] for row in m], dtype=np.float64)
+
+
+@pytest.mark.parametrize("case", ["case_2x2", "case_3x3"])
+@pytest.mark.parametrize("mode", ["noncausal", "causal"])
+def test_hand_cases(case, mode):
+    c = json.load(open(GOLDEN))[case]
+    q, k, v = (_mat(c[n])[None, None] for n in ("Q", "K", "V"))
+    o, lse, rs = orc.attention(q, k, v, c["scale"], mode == "causal", return_rowsum=True)
+    np.testing.assert_allclose(o[0, 0], _mat(c[mode]["O"]), rtol=0, atol=1e-14)
+    np.testing.assert_allclose(lse[0, 0], [_ev(x) for x in c[mode]["LSE"]], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(rs, 1.0, atol=1e-14)
+
+
+def test_hand_case_2x2_literal_digits():
+    # the same 2x2 case against digits worked out separately (e/(e+1) = 0.7310585786300049)
+    q = np.eye(2)[None, None]
+    v = np.array([[1.0, 2.0], [3.0, 4.0]])[None, None]
+    o, lse = orc.attention(q, q, v, 1.0, False)
+    np.testing.assert_allclose(o[0, 0, 0], [1.5378828427399902, 2.5378828427399904], atol=1e-14)
+    np.testing.assert_allclose(o[0, 0, 1], [2.46211715726001, 3.4621171572600096], atol=1e-14)
+    np.testing.assert_allclose(lse[0, 0], [1.3132616875182228] * 2, atol=1e-14)
+
+
+# ------------------------------------------------------------------ invariants
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_probability_rows_sum_to_one(causal):
+    q, k, v = rand((2, 3, 37, 16), 1), rand((2, 3, 53, 16), 2), rand((2, 3, 53, 16), 3)
+    _, _, rs = orc.attention(q, k, v, 0.25, causal, return_rowsum=True)
+    assert np.max(np.abs(rs - 1.0)) <= 1e-12
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_constant_v_returns_constant(causal):
+    q, k = rand((1, 2, 19, 8), 4), rand((1, 2, 31, 8), 5)
+    v = np.full((1, 2, 31, 8), -3.25)
+    o, _ = orc.attention(q, k, v, 0.7, causal)
+    assert np.max(np.abs(o + 3.25)) <= 1e-12
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_identical_keys_give_mean_of_v(causal):
+    B, H, Sq, Sk, D = 1, 2, 9, 13, 8
+    q, v = rand((B, H, Sq, D), 6), rand((B, H, Sk, D), 7)
+    k0 = rand((B, H, 1, D), 8)
+    k = np.repeat(k0, Sk, axis=2)
+    scale = 0.3
+    o, lse = orc.attention(q, k, v, scale, causal)
+    for i in range(Sq):
+        n = min(i + 1, Sk) if causal else Sk
+        np.testing.assert_allclose(o[:, :, i], v[:, :, :n].mean(axis=2), atol=1e-12)
+        want = scale * np.einsum("bhd,bhd->bh", q[:, :, i], k0[:, :, 0]) + math.log(n)
+        np.testing.assert_allclose(lse[:, :, i], want, atol=1e-12)
+
+
+def test_zero_queries_and_zero_scale():
+    B, H, Sq, Sk, D = 1, 1, 5, 11, 4
+    k, v = rand((B, H, Sk, D), 9), rand((B, H, Sk, D), 10)
+    o, lse = orc.attention(np.zeros((B, H, Sq, D)), k, v, 1.0, False)
+    np.testing.assert_allclose(lse, math.log(Sk), atol=1e-13)
+    np.testing.assert_allclose(o, np.broadcast_to(v.mean(axis=2, keepdims=True), o.shape), atol=1e-13)
+    o2, lse2 = orc.attention(rand((B, H, Sq, D), 11), k, v, 0.0, True)
+    for i in range(Sq):
+        np.testing.assert_allclose(lse2[0, 0, i], math.log(i + 1), atol=1e-13)
+        np.testing.assert_allclose(o2[0, 0, i], v[0, 0, :i + 1].mean(axis=0), atol=1e-13)
+
+
+@pytest.mark.parametrize("Sq,Sk", [(7, 7), (5, 9), (9, 5)])
+def test_causal_first_row_and_alignment(Sq, Sk):
+    q, k, v = rand((1, 2, Sq, 8), 12), rand((1, 2, Sk, 8), 13), rand((1, 2, Sk, 8), 14)
+    scale = 0.5
+    oc, lc = orc.attention(q, k, v, scale, True)
+    on, ln_ = orc.attention(q, k, v, scale, False)
+    np.testing.assert_allclose(oc[:, :, 0], v[:, :, 0], atol=1e-14)
+    np.testing.assert_allclose(lc[:, :, 0], scale * np.einsum("bhd,bhd->bh", q[:, :, 0], k[:, :, 0]),
+                               atol=1e-14)
+    # top-left alignment: every row i >= Sk-1 sees all keys, i.e. equals the unmasked result
+    for i in range(Sq):
+        if i >= Sk - 1:
+            np.testing.assert_allclose(oc[:, :, i], on[:, :, i], atol=1e-14)
+            np.testing.assert_allclose(lc[:, :, i], ln_[:, :, i], atol=1e-14)
+        else:
+            # row i equals an unmasked problem over the first i+1 keys
+            oi, li = orc.attention(q[:, :, i:i + 1], k[:, :, :i + 1], v[:, :, :i + 1], scale, False)
+            np.testing.assert_allclose(oc[:, :, i], oi[:, :, 0], atol=1e-14)
+            np.testing.assert_allclose(lc[:, :, i], li[:, :, 0], atol=1e-14)
+
+
+def test_key_shift_invariance():
+    q, k, v = rand((1, 2, 6, 8), 15), rand((1, 2, 10, 8), 16), rand((1, 2, 10, 8), 17)
+    u = rand((1, 2, 1, 8), 18)
+    scale = 0.4
+    o1, l1 = orc.attention(q, k, v, scale, False)
+    o2, l2 = orc.attention(q, k + u, v, scale, False)
+    np.testing.assert_allclose(o2, o1, atol=1e-12)
+    np.testing.assert_allclose(l2 - l1, scale * np.einsum("bhid,bhd->bhi", q, u[:, :, 0]), atol=1e-12)
+
+
+def test_key_permutation_invariance():
+    q, k, v = rand((1, 1, 6, 8), 19), rand((1, 1, 21, 8), 20), rand((1, 1, 21, 8), 21)
+    perm = np.random.default_rng(22).permutation(21)
+    o1, l1 = orc.attention(q, k, v, 0.35, False)
+    o2, l2 = orc.attention(q, k[:, :, perm], v[:, :, perm], 0.35, False)
+    np.testing.assert_allclose(o2, o1, atol=1e-12)
+    np.testing.assert_allclose(l2, l1, atol=1e-12)
+
+
+def test_split_combine_identity():
+    q, k, v = rand((1, 2, 8, 8), 23), rand((1, 2, 24, 8), 24), rand((1, 2, 24, 8), 25)
+    o, lse = orc.attention(q, k, v, 0.3, False)
+    oa, la = orc.attention(q, k[:, :, :10], v[:, :, :10], 0.3, False)
+    ob, lb = orc.attention(q, k[:, :, 10:], v[:, :, 10:], 0.3, False)
+    l = np.logaddexp(la, lb)
+    oc = np.exp(la - l)[..., None] * oa + np.exp(lb - l)[..., None] * ob
+    np.testing.assert_allclose(l, lse, atol=1e-12)
+    np.testing.assert_allclose(oc, o, atol=1e-12)
+
+
+def test_one_hot_limit_is_overflow_safe():
+    q, k, v = rand((1, 1, 4, 8), 26), rand((1, 1, 16, 8), 27), rand((1, 1, 16, 8), 28)
+    scale = 1e4
+    o, lse = orc.attention(q, k, v, scale, False)
+    s = scale * np.einsum("id,jd->ij", q[0, 0], k[0, 0])
+    arg = s.argmax(axis=1)
+    assert np.all(np.isfinite(o)) and np.all(np.isfinite(lse))
+    np.testing.assert_allclose(o[0, 0], v[0, 0, arg], atol=1e-9)
+    np.testing.assert_allclose(lse[0, 0], s.max(axis=1), rtol=1e-9)
+
+
+def test_no_visible_key_convention():
+    q = rand((1, 1, 3, 4), 29)
+    k = np.zeros((1, 1, 0, 4))
+    o, lse = orc.attention(q, k, k, 1.0, False)
+    assert np.all(o == 0.0) and np.all(np.isneginf(lse))
+
+
+# ------------------------------------------------------------------ brute force and library
+
+def dense_brute_force(q, k, v, scale, causal):
+    """Builds the full score, mask and probability matrices -- written separately from the oracle."""
+    B, H, Sq, D = q.shape
+    Sk = k.shape[2]
+    o = np.zeros((B, H, Sq, D))
+    lse = np.zeros((B, H, Sq))
+    for b in range(B):
+        for h in range(H):
+            S = (q[b, h] @ k[b, h].T) * scale
+            if causal:
+                mask = np.triu(np.ones((Sq, Sk), dtype=bool), k=1)
+                S = np.where(mask, -np.inf, S)
+            E = np.exp(S)                       # small inputs: no overflow without max-subtraction
+            Z = E.sum(axis=1, keepdims=True)
+            o[b, h] = (E / Z) @ v[b, h]
+            lse[b, h] = np.log(Z[:, 0])
+    return o, lse
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("shape", [(1, 1, 1, 1, 1), (2, 2, 16, 16, 8), (1, 2, 5, 12, 3), (2, 1, 13, 4, 7)])
+def test_against_dense_brute_force(shape, causal):
+    B, H, Sq, Sk, D = shape
+    q, k, v = rand((B, H, Sq, D), 30), rand((B, H, Sk, D), 31), rand((B, H, Sk, D), 32)
+    o, lse = orc.attention(q, k, v, 1.0 / math.sqrt(D), causal)
+    ob, lb = dense_brute_force(q, k, v, 1.0 / math.sqrt(D), causal)
+    np.testing.assert_allclose(o, ob, atol=1e-12)
+    np.testing.assert_allclose(lse, lb, atol=1e-12)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_against_torch_sdpa_fp64(causal):
+    B, H, Sq, Sk, D = 2, 3, 65, 65, 32
+    q, k, v = rand((B, H, Sq, D), 33), rand((B, H, Sk, D), 34), rand((B, H, Sk, D), 35)
+    scale = 0.17
+    o, lse = orc.attention(q, k, v, scale, causal)
+    tq, tk, tv = (torch.from_numpy(x) for x in (q, k, v))
+    to = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=causal, scale=scale)
+    np.testing.assert_allclose(o, to.numpy(), atol=1e-10)
+    s = (tq @ tk.transpose(-1, -2)) * scale
+    if causal:
+        s = s.masked_fill(torch.triu(torch.ones(Sq, Sk, dtype=torch.bool), 1), float("-inf"))
+    np.testing.assert_allclose(lse, torch.logsumexp(s, dim=-1).numpy(), atol=1e-10)
+
+
+# ------------------------------------------------------------------ the 16-bit row-subset entry
+
+@pytest.mark.parametrize("dtype", [inputs.DTYPE_FP16, inputs.DTYPE_BF16])
+@pytest.mark.parametrize("causal", [False, True])
+def test_row_subset_entry_matches_full(dtype, causal):
+    B, H, Sq, Sk, D = 2, 2, 40, 56, 16
+    q, k, v = inputs.make_qkv(B, H, Sq, Sk, D, dtype, seed=77)
+    qb, kb, vb = inputs.bits(q), inputs.bits(k), inputs.bits(v)
+    o, lse = orc.attention(orc.widen(qb, dtype), orc.widen(kb, dtype), orc.widen(vb, dtype), 0.25, causal)
+    rows = np.array([0, 1, 39, 40, 79, 100, 159], dtype=np.int64)
+    orows, lrows = orc.attention_rows_16(qb, kb, vb, dtype, rows, 0.25, causal)
+    np.testing.assert_array_equal(orows, o.reshape(-1, D)[rows])
+    np.testing.assert_array_equal(lrows, lse.reshape(-1)[rows])
+
+
+def test_input_generator_is_seeded_and_rounded():
+    a = inputs.randn16((3, 5), 123, inputs.DTYPE_BF16)
+    b = inputs.randn16((3, 5), 123, inputs.DTYPE_BF16)
+    c = inputs.randn16((3, 5), 124, inputs.DTYPE_BF16)
+    assert torch.equal(a, b) and not torch.equal(a, c)
+    assert a.dtype == torch.bfloat16
+    w = orc.widen(inputs.bits(a), inputs.DTYPE_BF16)
+    np.testing.assert_array_equal(w, a.to(torch.float64).numpy())

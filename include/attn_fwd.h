@@ -1,0 +1,114 @@
+/*
+ * attn_fwd.h -- C ABI of the fused attention forward operator for NVIDIA B200 (sm_100a).
+ *
+ * The operator is the one defined in Section 2.2 of the paper,
+ *
+ *     Attention(Q, K, V) = Softmax(Mask(Q K^T / sqrt(d))) V ,
+ *
+ * evaluated FlashAttention-style (Section 2.2 / the kernel loop of Appendix C's
+ * listings: a Q tile stays on chip, K/V tiles stream through shared memory, the
+ * softmax is computed online with a running maximum and running sum, and the
+ * S x S score matrix never reaches global memory).  In addition to O the library
+ * returns the per-row logsumexp of the scaled, masked scores.
+ *
+ * Conventions
+ *   - All tensors are row-major and contiguous:  Q, O: [B, H, Sq, D];  K, V: [B, H, Sk, D];
+ *     LSE: [B, H, Sq] in fp32.  Q, K, V, O share one 16-bit type (attn_dtype_t).
+ *   - scale multiplies Q K^T (the paper uses 1/sqrt(d)); it must be finite and >= 0.
+ *   - causal != 0 applies the lower-triangular mask aligned to the top-left corner:
+ *     key j is visible to query i iff j <= i, also when Sq != Sk.
+ *   - LSE[i] = ln( sum over visible j of exp(scale * <q_i, k_j>) )   (natural log).
+ *   - A row without any visible key (only possible when Sk == 0) gives O = 0, LSE = -inf.
+ *   - Accumulation is fp32; the probabilities are rounded to the 16-bit input type
+ *     before the second product; O is rounded once at the end.
+ *
+ * Ownership and asynchrony
+ *   - The caller owns every buffer.  The library allocates no device memory.
+ *   - Device entry points only enqueue work on `stream` (a cudaStream_t, may be NULL for
+ *     the default stream) and return; they never synchronise.
+ *   - Nothing throws; every entry point returns an attn_status_t (0 = success).
+ *   - Q, K, V must not alias O or LSE.
+ *
+ * There is no CPU fallback: on a device that is not compute capability 10.x the entry
+ * points return ATTN_ERR_UNSUPPORTED_ARCH.
+ */
+#ifndef ATTN_FWD_H_
+#define ATTN_FWD_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { ATTN_DTYPE_FP16 = 0, ATTN_DTYPE_BF16 = 1 } attn_dtype_t;
+
+typedef enum {
+    ATTN_OK = 0,
+    ATTN_ERR_NULL_POINTER = 1,         /* a required pointer is NULL */
+    ATTN_ERR_BAD_SHAPE = 2,            /* negative extent, or an extent/product out of range */
+    ATTN_ERR_UNSUPPORTED_HEAD_DIM = 3, /* D is not 64, 128 or 256 */
+    ATTN_ERR_UNSUPPORTED_DTYPE = 4,    /* dtype is not an attn_dtype_t */
+    ATTN_ERR_MISALIGNED = 5,           /* q/k/v/o not 16-byte aligned, lse not 4-byte aligned */
+    ATTN_ERR_BAD_SCALE = 6,            /* scale is NaN, infinite or negative */
+    ATTN_ERR_UNSUPPORTED_ARCH = 7,     /* current device is not compute capability 10.x */
+    ATTN_ERR_CUDA = 8,                 /* a CUDA runtime/driver call failed */
+    ATTN_ERR_DEVICE_TIMEOUT = 9,       /* a kernel gave up on a bounded on-chip wait */
+    ATTN_ERR_WORKSPACE = 10            /* workspace missing, misaligned or too small */
+} attn_status_t;
+
+/*
+ * attn_fwd -- the hot path (Section 2.2; kernel loop as in Appendix C, Listings 1-2).
+ *
+ * q, k, v : device pointers, 16-byte aligned, layouts above, element type `dtype`.
+ * o       : device pointer, 16-byte aligned, [B,H,Sq,D], element type `dtype` (written).
+ * lse     : device pointer, [B,H,Sq] fp32 (written).
+ * B, H, Sq, Sk >= 0;  D in {64, 128, 256};  B*H <= 2^31-1, Sq, Sk <= 2^31-1-256.
+ * B*H*Sq == 0 is a successful no-op.  Sk == 0 writes O = 0 and LSE = -inf.
+ * Runs on sm_100a tensor cores (tcgen05 MMAs with TMEM accumulators, TMA tile loads).
+ * Validation happens on the host before anything is enqueued; on an error nothing is
+ * launched.
+ */
+int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq,
+             int Sk, int D, float scale, int causal, int dtype, void* stream);
+
+/*
+ * attn_fwd_simt -- same operator, same arguments, same conventions, computed by a plain
+ * CUDA-core kernel (one warp per query row, fp32 arithmetic, online softmax).  It is one to
+ * two orders of magnitude slower than attn_fwd and exists as an on-device cross-check that
+ * uses none of the tensor-core machinery.
+ */
+int attn_fwd_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H,
+                  int Sq, int Sk, int D, float scale, int causal, int dtype, void* stream);
+
+/*
+ * attn_fwd_host -- attn_fwd for HOST buffers.  q, k, v, o, lse are host pointers (pinned
+ * memory makes the copies asynchronous); `workspace` is a caller-owned DEVICE buffer of at
+ * least attn_fwd_host_workspace_bytes(...) bytes, 256-byte aligned.  Enqueues on `stream`:
+ * three host-to-device copies, the attention kernel, two device-to-host copies.  The results
+ * are valid once the caller has synchronised `stream`.
+ * Errors: as attn_fwd, plus ATTN_ERR_WORKSPACE.
+ */
+int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
+                  float* lse_host, int B, int H, int Sq, int Sk, int D, float scale, int causal,
+                  int dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of device workspace attn_fwd_host needs for this problem (0 for an invalid shape). */
+size_t attn_fwd_host_workspace_bytes(int B, int H, int Sq, int Sk, int D);
+
+/* ATTN_OK if attn_fwd supports (D, dtype, causal) on the current device, otherwise the
+ * status attn_fwd would return.  Launches nothing. */
+int attn_query_support(int D, int dtype, int causal);
+
+/* Synchronises `stream`, then returns and clears the device-side status word of the current
+ * device: ATTN_OK, or ATTN_ERR_DEVICE_TIMEOUT if any kernel since the last call gave up on a
+ * bounded wait (its output is then undefined).  ATTN_ERR_CUDA if the synchronisation fails. */
+int attn_last_device_status(void* stream);
+
+/* Static, human-readable name of a status code. */
+const char* attn_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATTN_FWD_H_ */

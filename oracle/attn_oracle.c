@@ -163,53 +163,62 @@ int attn_oracle_f64(const double *q, const double *k, const double *v, double *o
     return failed ? -1 : 0;
 }
 
-/* Same arithmetic for a chosen subset of rows, reading the 16-bit inputs
- * directly (widened exactly, element by element) so that full-size problems
- * need no fp64 copy of Q, K, V.
- * rows[n_rows]: flat row indices r = (b*H + h)*Sq + i.
- * o: [n_rows, D], lse: [n_rows]. */
+/* Same arithmetic for a chosen subset of rows, reading the 16-bit inputs directly
+ * (widened exactly) so that full-size problems need no fp64 copy of Q, K, V.
+ * rows[n_rows]: flat row indices r = (b*H + h)*Sq + i, in ascending order.
+ * o: [n_rows, D], lse: [n_rows].
+ * Rows of one (batch, head) share one widened copy of that head's K and V. */
 int attn_oracle_rows_16(const uint16_t *q, const uint16_t *k, const uint16_t *v, int dtype,
                         const int64_t *rows, int64_t n_rows, double *o, double *lse, int B, int H,
                         int Sq, int Sk, int D, double scale, int causal)
 {
-    int failed = 0;
     (void)B;
     (void)H;
+    size_t nk = (size_t)(Sk > 0 ? Sk : 1);
+    double *kd = (double *)malloc(sizeof(double) * nk * (size_t)D);
+    double *vd = (double *)malloc(sizeof(double) * nk * (size_t)D);
+    int failed = (!kd || !vd);
+    int64_t t0 = 0;
+    while (!failed && t0 < n_rows) {
+        /* the run of requested rows that belong to one (batch, head) */
+        int64_t bh = rows[t0] / Sq, t1 = t0;
+        int64_t need = 0; /* keys that the run's longest row sees */
+        while (t1 < n_rows && rows[t1] / Sq == bh) {
+            int64_t nv = visible_keys(rows[t1] % Sq, Sk, causal);
+            if (nv > need)
+                need = nv;
+            ++t1;
+        }
+        oracle_widen(k + bh * Sk * D, kd, need * D, dtype);
+        oracle_widen(v + bh * Sk * D, vd, need * D, dtype);
 #pragma omp parallel
-    {
-        size_t nk = (size_t)(Sk > 0 ? Sk : 1);
-        double *s = (double *)malloc(sizeof(double) * nk);
-        double *qd = (double *)malloc(sizeof(double) * (size_t)D);
-        double *kd = (double *)malloc(sizeof(double) * nk * (size_t)D);
-        double *vd = (double *)malloc(sizeof(double) * nk * (size_t)D);
-        if (!s || !qd || !kd || !vd) {
+        {
+            double *s = (double *)malloc(sizeof(double) * nk);
+            double *qd = (double *)malloc(sizeof(double) * (size_t)D);
+            if (!s || !qd) {
 #pragma omp atomic write
-            failed = 1;
-        }
-        int64_t t;
-#pragma omp for schedule(dynamic, 1)
-        for (t = 0; t < n_rows; ++t) {
-            if (!s || !qd || !kd || !vd)
-                continue;
-            int64_t r = rows[t];
-            int64_t bh = r / Sq, i = r % Sq;
-            int64_t n_vis = visible_keys(i, Sk, causal);
-            int64_t e;
-            for (e = 0; e < D; ++e)
-                qd[e] = dtype == 0 ? oracle_f16_bits_to_f64(q[r * D + e])
-                                   : oracle_bf16_bits_to_f64(q[r * D + e]);
-            for (e = 0; e < n_vis * D; ++e) {
-                uint16_t kb = k[bh * Sk * D + e], vb = v[bh * Sk * D + e];
-                kd[e] = dtype == 0 ? oracle_f16_bits_to_f64(kb) : oracle_bf16_bits_to_f64(kb);
-                vd[e] = dtype == 0 ? oracle_f16_bits_to_f64(vb) : oracle_bf16_bits_to_f64(vb);
+                failed = 1;
             }
-            attn_row(qd, kd, vd, s, o + t * D, lse + t, NULL, n_vis, D, scale);
+            int64_t t;
+#pragma omp for schedule(dynamic, 1)
+            for (t = t0; t < t1; ++t) {
+                if (!s || !qd)
+                    continue;
+                int64_t r = rows[t];
+                int e;
+                for (e = 0; e < D; ++e)
+                    qd[e] = dtype == 0 ? oracle_f16_bits_to_f64(q[r * D + e])
+                                       : oracle_bf16_bits_to_f64(q[r * D + e]);
+                attn_row(qd, kd, vd, s, o + t * D, lse + t, NULL,
+                         visible_keys(r % Sq, Sk, causal), D, scale);
+            }
+            free(s);
+            free(qd);
         }
-        free(s);
-        free(qd);
-        free(kd);
-        free(vd);
+        t0 = t1;
     }
+    free(kd);
+    free(vd);
     return failed ? -1 : 0;
 }
 

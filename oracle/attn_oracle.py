@@ -114,6 +114,7 @@ def attention_rows_16(q_bits, k_bits, v_bits, dtype: int, rows, scale: float, ca
     Sk = k_bits.shape[2]
     assert k_bits.shape == (B, H, Sk, D) and v_bits.shape == (B, H, Sk, D)
     assert rows.size == 0 or (rows.min() >= 0 and rows.max() < B * H * Sq)
+    assert np.all(np.diff(rows) >= 0), "rows must be in ascending order"
     o = np.empty((rows.size, D), dtype=np.float64)
     lse = np.empty((rows.size,), dtype=np.float64)
     rc = _load().attn_oracle_rows_16(

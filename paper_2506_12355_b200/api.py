@@ -1,0 +1,161 @@
+"""Python binding of the C ABI in include/attn_fwd.h.
+
+Argument marshalling only: every step of the attention forward pass runs in the
+CUDA kernels of libattn_fwd.so.  PyTorch supplies device memory and streams.
+There is no fallback: if the library is missing the import of a symbol fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+DTYPE_FP16 = 0
+DTYPE_BF16 = 1
+
+STATUS_NAMES = {
+    0: "ATTN_OK", 1: "ATTN_ERR_NULL_POINTER", 2: "ATTN_ERR_BAD_SHAPE",
+    3: "ATTN_ERR_UNSUPPORTED_HEAD_DIM", 4: "ATTN_ERR_UNSUPPORTED_DTYPE", 5: "ATTN_ERR_MISALIGNED",
+    6: "ATTN_ERR_BAD_SCALE", 7: "ATTN_ERR_UNSUPPORTED_ARCH", 8: "ATTN_ERR_CUDA",
+    9: "ATTN_ERR_DEVICE_TIMEOUT", 10: "ATTN_ERR_WORKSPACE",
+}
+
+# every symbol include/attn_fwd.h declares
+EXPORTS = ["attn_fwd", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
+           "attn_query_support", "attn_last_device_status", "attn_status_string"]
+
+_lib = None
+
+
+class AttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (%d)" % (where, STATUS_NAMES.get(status, "?"), status))
+
+
+def lib_path() -> str:
+    return _build.LIB_PATH
+
+
+def load() -> ctypes.CDLL:
+    """Loads libattn_fwd.so (built in-tree).  Raises if it does not exist: there is no fallback."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = lib_path()
+    if not os.path.exists(path):
+        raise ImportError("libattn_fwd.so is not built; run `python -m paper_2506_12355_b200.build` "
+                          "or __graft_entry__.build()")
+    lib = ctypes.CDLL(path)
+    vp, i, f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    sig = [vp, vp, vp, vp, vp, i, i, i, i, i, f, i, i, vp]
+    lib.attn_fwd.restype = i
+    lib.attn_fwd.argtypes = sig
+    lib.attn_fwd_simt.restype = i
+    lib.attn_fwd_simt.argtypes = sig
+    lib.attn_fwd_host.restype = i
+    lib.attn_fwd_host.argtypes = sig[:-1] + [vp, ctypes.c_size_t, vp]
+    lib.attn_fwd_host_workspace_bytes.restype = ctypes.c_size_t
+    lib.attn_fwd_host_workspace_bytes.argtypes = [i] * 5
+    lib.attn_query_support.restype = i
+    lib.attn_query_support.argtypes = [i, i, i]
+    lib.attn_last_device_status.restype = i
+    lib.attn_last_device_status.argtypes = [vp]
+    lib.attn_status_string.restype = ctypes.c_char_p
+    lib.attn_status_string.argtypes = [i]
+    _lib = lib
+    return lib
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float16:
+        return DTYPE_FP16
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    raise TypeError("q/k/v must be float16 or bfloat16, got %s" % t.dtype)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _check_qkv(q, k, v):
+    if q.dim() != 4 or k.dim() != 4 or v.dim() != 4:
+        raise ValueError("q, k, v must be [B,H,S,D]")
+    B, H, Sq, D = q.shape
+    Sk = k.shape[2]
+    if tuple(k.shape) != (B, H, Sk, D) or tuple(v.shape) != (B, H, Sk, D):
+        raise ValueError("k, v must be [B,H,Sk,D] matching q's B, H, D")
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+        raise ValueError("q, k, v must be contiguous")
+    if not (q.dtype == k.dtype == v.dtype):
+        raise TypeError("q, k, v must share one dtype")
+    return B, H, Sq, Sk, D
+
+
+def _call_device(fn_name, q, k, v, scale, causal, out, lse, stream):
+    B, H, Sq, Sk, D = _check_qkv(q, k, v)
+    if not (q.is_cuda and k.is_cuda and v.is_cuda):
+        raise ValueError("q, k, v must be CUDA tensors")
+    dt = _dtype_code(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(q.device):
+        rc = getattr(load(), fn_name)(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                      lse.data_ptr(), B, H, Sq, Sk, D, float(scale),
+                                      int(bool(causal)), dt, _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, fn_name)
+    return out, lse
+
+
+def attn_fwd(q, k, v, scale: float, causal: bool = False, out=None, lse=None, stream=None):
+    """O [B,H,Sq,D] (dtype of q) and LSE [B,H,Sq] (fp32) on the tensor-core kernel.
+
+    Enqueues on `stream` (default: torch's current stream) and returns without synchronising.
+    """
+    return _call_device("attn_fwd", q, k, v, scale, causal, out, lse, stream)
+
+
+def attn_fwd_simt(q, k, v, scale: float, causal: bool = False, out=None, lse=None, stream=None):
+    """Same operator on the slow CUDA-core cross-check kernel."""
+    return _call_device("attn_fwd_simt", q, k, v, scale, causal, out, lse, stream)
+
+
+def attn_fwd_host_workspace_bytes(B, H, Sq, Sk, D) -> int:
+    return int(load().attn_fwd_host_workspace_bytes(B, H, Sq, Sk, D))
+
+
+def attn_fwd_host(q, k, v, scale: float, causal: bool, out, lse, workspace, stream=None):
+    """attn_fwd for HOST tensors (pinned for asynchronous copies); `workspace` is a CUDA uint8
+    tensor of at least attn_fwd_host_workspace_bytes(...) bytes.  Results are valid after the
+    stream has been synchronised."""
+    B, H, Sq, Sk, D = _check_qkv(q, k, v)
+    dt = _dtype_code(q)
+    with torch.cuda.device(workspace.device):
+        rc = load().attn_fwd_host(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                  lse.data_ptr(), B, H, Sq, Sk, D, float(scale), int(bool(causal)),
+                                  dt, workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                  _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_fwd_host")
+    return out, lse
+
+
+def attn_query_support(D: int, dtype: int, causal: bool) -> int:
+    return int(load().attn_query_support(int(D), int(dtype), int(bool(causal))))
+
+
+def attn_last_device_status(stream=None) -> int:
+    return int(load().attn_last_device_status(_stream_ptr(stream)))
+
+
+def attn_status_string(status: int) -> str:
+    return load().attn_status_string(int(status)).decode()

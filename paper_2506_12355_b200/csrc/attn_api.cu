@@ -1,0 +1,257 @@
+// C ABI of the attention forward library (declared in include/attn_fwd.h):
+// host-side validation, TMA tensor-map construction and kernel dispatch.
+// There is no CPU fallback anywhere in this file.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "../../include/attn_fwd.h"
+#include "attn_simt.cuh"
+#include "attn_tc_basic.cuh"
+
+namespace {
+
+// Device-side status word: 0, or ATTN_ERR_DEVICE_TIMEOUT once a kernel gave up on a wait.
+__device__ int g_device_status = 0;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// Rank-3 map over a [BH, S, D] row-major 16-bit tensor; box = [1, box_rows, 64 columns],
+// 128-byte swizzle, out-of-range rows read as zero.
+bool make_map(CUtensorMap* map, const void* base, int dtype, int64_t BH, int64_t S, int D, int box_rows) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S), static_cast<cuuint64_t>(BH)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(S) * D * 2};
+    cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(map, dtype == ATTN_DTYPE_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                     3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int check_arch() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ATTN_ERR_CUDA;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ATTN_ERR_CUDA;
+    return major == 10 ? ATTN_OK : ATTN_ERR_UNSUPPORTED_ARCH;
+}
+
+constexpr int kMaxSeq = 2147483647 - 256;
+
+// Validation shared by every entry point; no CUDA call happens here.
+int validate(const void* q, const void* k, const void* v, const void* o, const void* lse, int B, int H, int Sq,
+             int Sk, int D, float scale, int dtype, bool device_pointers) {
+    if (!q || !k || !v || !o || !lse) return ATTN_ERR_NULL_POINTER;
+    if (B < 0 || H < 0 || Sq < 0 || Sk < 0 || D < 0) return ATTN_ERR_BAD_SHAPE;
+    if (Sq > kMaxSeq || Sk > kMaxSeq) return ATTN_ERR_BAD_SHAPE;
+    if (static_cast<int64_t>(B) * H > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
+    if (D != 64 && D != 128 && D != 256) return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
+    if (dtype != ATTN_DTYPE_FP16 && dtype != ATTN_DTYPE_BF16) return ATTN_ERR_UNSUPPORTED_DTYPE;
+    if (device_pointers) {
+        if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(v) |
+             reinterpret_cast<uintptr_t>(o)) & 15u)
+            return ATTN_ERR_MISALIGNED;
+        if (reinterpret_cast<uintptr_t>(lse) & 3u) return ATTN_ERR_MISALIGNED;
+    }
+    if (!isfinite(scale) || scale < 0.f) return ATTN_ERR_BAD_SCALE;
+    return ATTN_OK;
+}
+
+int* device_status_ptr() {
+    int* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_device_status) != cudaSuccess) return nullptr;
+    return p;
+}
+
+int fill_empty(void* o, float* lse, int64_t n_o, int64_t n_lse, cudaStream_t st) {
+    attn_simt::attn_fill_empty_kernel<<<148, 256, 0, st>>>(static_cast<uint16_t*>(o), lse, n_o, n_lse);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+template <int D, int DTYPE>
+int launch_tc_basic(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
+                    float scale, int causal, cudaStream_t st) {
+    using C = attn_tc::BasicCfg<D>;
+    auto kern = attn_tc::attn_fwd_tc_basic_kernel<D, DTYPE>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    });
+    if (attr_err != cudaSuccess) return ATTN_ERR_CUDA;
+    const int64_t BH = static_cast<int64_t>(B) * H;
+    CUtensorMap mq, mk, mv;
+    if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, BH, Sk, D, C::BN) ||
+        !make_map(&mv, v, DTYPE, BH, Sk, D, C::BN))
+        return ATTN_ERR_CUDA;
+    attn_tc::Params prm;
+    prm.o = o;
+    prm.lse = lse;
+    prm.Sq = Sq;
+    prm.Sk = Sk;
+    prm.scale = scale;
+    prm.scale_log2 = scale * 1.4426950408889634f;
+    prm.causal = causal ? 1 : 0;
+    prm.status = device_status_ptr();
+    if (!prm.status) return ATTN_ERR_CUDA;
+    const int64_t q_tiles = (static_cast<int64_t>(Sq) + C::BM - 1) / C::BM;
+    // grid.y is limited to 65535: fold the heads into grid.x when there are more
+    if (BH > 65535) return ATTN_ERR_BAD_SHAPE;
+    dim3 grid(static_cast<unsigned>(q_tiles), static_cast<unsigned>(BH));
+    kern<<<grid, 128, C::SMEM_BYTES, st>>>(mq, mk, mv, prm);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+template <int D, int DTYPE>
+int launch_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
+                float scale, int causal, cudaStream_t st) {
+    const int64_t BH = static_cast<int64_t>(B) * H;
+    if (BH > 65535) return ATTN_ERR_BAD_SHAPE;
+    dim3 grid(static_cast<unsigned>((static_cast<int64_t>(Sq) + attn_simt::kWarpsPerBlock - 1) / attn_simt::kWarpsPerBlock),
+              static_cast<unsigned>(BH));
+    attn_simt::attn_fwd_simt_kernel<D, DTYPE><<<grid, attn_simt::kWarpsPerBlock * 32, 0, st>>>(q, k, v, o, lse, Sq, Sk,
+                                                                                              scale, causal ? 1 : 0);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+enum class Impl { TensorCore, Simt };
+
+template <Impl IMPL>
+int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk, int D,
+             float scale, int causal, int dtype, void* stream) {
+    int rc = validate(q, k, v, o, lse, B, H, Sq, Sk, D, scale, dtype, true);
+    if (rc != ATTN_OK) return rc;
+    if (static_cast<int64_t>(B) * H * Sq == 0) return ATTN_OK;
+    rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (Sk == 0)
+        return fill_empty(o, lse, static_cast<int64_t>(B) * H * Sq * D, static_cast<int64_t>(B) * H * Sq, st);
+#define ATTN_CASE(DD, TT)                                                                              \
+    if (D == DD && dtype == TT) {                                                                      \
+        if (IMPL == Impl::Simt) return launch_simt<DD, TT>(q, k, v, o, lse, B, H, Sq, Sk, scale, causal, st); \
+        return launch_tc_basic<DD, TT>(q, k, v, o, lse, B, H, Sq, Sk, scale, causal, st);              \
+    }
+    ATTN_CASE(64, 0)
+    ATTN_CASE(64, 1)
+    ATTN_CASE(128, 0)
+    ATTN_CASE(128, 1)
+    ATTN_CASE(256, 0)
+    ATTN_CASE(256, 1)
+#undef ATTN_CASE
+    return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+}  // namespace
+
+extern "C" {
+
+int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk, int D,
+             float scale, int causal, int dtype, void* stream) {
+    return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, Sq, Sk, D, scale, causal, dtype, stream);
+}
+
+int attn_fwd_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
+                  int D, float scale, int causal, int dtype, void* stream) {
+    return dispatch<Impl::Simt>(q, k, v, o, lse, B, H, Sq, Sk, D, scale, causal, dtype, stream);
+}
+
+size_t attn_fwd_host_workspace_bytes(int B, int H, int Sq, int Sk, int D) {
+    if (B < 0 || H < 0 || Sq < 0 || Sk < 0 || D <= 0) return 0;
+    const size_t bh = static_cast<size_t>(B) * H;
+    const size_t qo = align256(bh * Sq * D * 2), kv = align256(bh * Sk * D * 2), ls = align256(bh * Sq * 4);
+    return 2 * qo + 2 * kv + ls;
+}
+
+int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host, float* lse_host, int B,
+                  int H, int Sq, int Sk, int D, float scale, int causal, int dtype, void* workspace,
+                  size_t workspace_bytes, void* stream) {
+    int rc = validate(q_host, k_host, v_host, o_host, lse_host, B, H, Sq, Sk, D, scale, dtype, false);
+    if (rc != ATTN_OK) return rc;
+    const size_t bh = static_cast<size_t>(B) * H;
+    if (bh * Sq == 0) return ATTN_OK;
+    const size_t need = attn_fwd_host_workspace_bytes(B, H, Sq, Sk, D);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)
+        return ATTN_ERR_WORKSPACE;
+    const size_t qo_b = bh * Sq * D * 2, kv_b = bh * Sk * D * 2, ls_b = bh * Sq * 4;
+    uint8_t* w = static_cast<uint8_t*>(workspace);
+    uint8_t* dq = w;
+    uint8_t* dk = dq + align256(qo_b);
+    uint8_t* dv = dk + align256(kv_b);
+    uint8_t* d_o = dv + align256(kv_b);
+    float* dl = reinterpret_cast<float*>(d_o + align256(qo_b));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(dq, q_host, qo_b, cudaMemcpyHostToDevice, st) != cudaSuccess) return ATTN_ERR_CUDA;
+    if (kv_b) {
+        if (cudaMemcpyAsync(dk, k_host, kv_b, cudaMemcpyHostToDevice, st) != cudaSuccess) return ATTN_ERR_CUDA;
+        if (cudaMemcpyAsync(dv, v_host, kv_b, cudaMemcpyHostToDevice, st) != cudaSuccess) return ATTN_ERR_CUDA;
+    }
+    rc = attn_fwd(dq, dk, dv, d_o, dl, B, H, Sq, Sk, D, scale, causal, dtype, stream);
+    if (rc != ATTN_OK) return rc;
+    if (cudaMemcpyAsync(o_host, d_o, qo_b, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ATTN_ERR_CUDA;
+    if (cudaMemcpyAsync(lse_host, dl, ls_b, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ATTN_ERR_CUDA;
+    return ATTN_OK;
+}
+
+int attn_query_support(int D, int dtype, int causal) {
+    (void)causal;
+    if (D != 64 && D != 128 && D != 256) return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
+    if (dtype != ATTN_DTYPE_FP16 && dtype != ATTN_DTYPE_BF16) return ATTN_ERR_UNSUPPORTED_DTYPE;
+    return check_arch();
+}
+
+int attn_last_device_status(void* stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return ATTN_ERR_CUDA;
+    int h = 0;
+    if (cudaMemcpyFromSymbol(&h, g_device_status, sizeof(int)) != cudaSuccess) return ATTN_ERR_CUDA;
+    if (h != 0) {
+        int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return ATTN_ERR_CUDA;
+    }
+    return h == 0 ? ATTN_OK : ATTN_ERR_DEVICE_TIMEOUT;
+}
+
+const char* attn_status_string(int status) {
+    switch (status) {
+        case ATTN_OK: return "ATTN_OK";
+        case ATTN_ERR_NULL_POINTER: return "ATTN_ERR_NULL_POINTER";
+        case ATTN_ERR_BAD_SHAPE: return "ATTN_ERR_BAD_SHAPE";
+        case ATTN_ERR_UNSUPPORTED_HEAD_DIM: return "ATTN_ERR_UNSUPPORTED_HEAD_DIM";
+        case ATTN_ERR_UNSUPPORTED_DTYPE: return "ATTN_ERR_UNSUPPORTED_DTYPE";
+        case ATTN_ERR_MISALIGNED: return "ATTN_ERR_MISALIGNED";
+        case ATTN_ERR_BAD_SCALE: return "ATTN_ERR_BAD_SCALE";
+        case ATTN_ERR_UNSUPPORTED_ARCH: return "ATTN_ERR_UNSUPPORTED_ARCH";
+        case ATTN_ERR_CUDA: return "ATTN_ERR_CUDA";
+        case ATTN_ERR_DEVICE_TIMEOUT: return "ATTN_ERR_DEVICE_TIMEOUT";
+        case ATTN_ERR_WORKSPACE: return "ATTN_ERR_WORKSPACE";
+        default: return "ATTN_ERR_UNKNOWN";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,102 @@
+"""Host-side checks of the C ABI: the library loads, exports what the header declares, and
+rejects bad arguments before touching a device (CPU only; nothing is launched)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2506_12355_b200 import api, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "attn_fwd.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return api.load()
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(attn_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_declares_the_documented_entry_points():
+    names = declared_functions()
+    assert "attn_fwd" in names and "attn_status_string" in names
+    assert sorted(api.EXPORTS) == names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    for name in declared_functions():
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    for code, name in api.STATUS_NAMES.items():
+        assert api.attn_status_string(code) == name
+    assert api.attn_status_string(12345) == "ATTN_ERR_UNKNOWN"
+
+
+GOOD = dict(q=0x1000, k=0x2000, v=0x3000, o=0x4000, lse=0x5000, B=1, H=1, Sq=128, Sk=128, D=64,
+            scale=0.125, causal=0, dtype=0, stream=None)
+
+
+def call(lib, fn="attn_fwd", **over):
+    a = dict(GOOD)
+    a.update(over)
+    return getattr(lib, fn)(a["q"], a["k"], a["v"], a["o"], a["lse"], a["B"], a["H"], a["Sq"], a["Sk"],
+                            a["D"], a["scale"], a["causal"], a["dtype"], a["stream"])
+
+
+@pytest.mark.parametrize("fn", ["attn_fwd", "attn_fwd_simt"])
+def test_argument_validation_happens_before_any_launch(lib, fn):
+    # the pointers are fake: every call below must be refused by host-side validation
+    for name in ("q", "k", "v", "o", "lse"):
+        assert call(lib, fn, **{name: None}) == 1
+    for name in ("B", "H", "Sq", "Sk"):
+        assert call(lib, fn, **{name: -1}) == 2
+    assert call(lib, fn, B=70000, H=70000) == 2
+    for d in (0, 32, 96, 192, 512):
+        assert call(lib, fn, D=d) == 3
+    assert call(lib, fn, dtype=2) == 4
+    assert call(lib, fn, dtype=-1) == 4
+    for name in ("q", "k", "v", "o"):
+        assert call(lib, fn, **{name: GOOD[name] + 8}) == 5
+    assert call(lib, fn, lse=GOOD["lse"] + 2) == 5
+    assert call(lib, fn, scale=float("nan")) == 6
+    assert call(lib, fn, scale=float("inf")) == 6
+    assert call(lib, fn, scale=-0.5) == 6
+    # empty problems are a successful no-op, decided before the device is looked at
+    assert call(lib, fn, B=0) == 0
+    assert call(lib, fn, Sq=0) == 0
+
+
+def test_host_entry_validation(lib):
+    n = lib.attn_fwd_host_workspace_bytes(2, 3, 100, 50, 64)
+    qo = (2 * 3 * 100 * 64 * 2 + 255) // 256 * 256
+    kv = (2 * 3 * 50 * 64 * 2 + 255) // 256 * 256
+    ls = (2 * 3 * 100 * 4 + 255) // 256 * 256
+    assert n == 2 * qo + 2 * kv + ls
+    assert lib.attn_fwd_host_workspace_bytes(-1, 1, 1, 1, 64) == 0
+    args = [0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 2, 3, 100, 50, 64, 0.125, 0, 0]
+    assert lib.attn_fwd_host(*args, None, 0, None) == 10            # no workspace
+    assert lib.attn_fwd_host(*args, 0x10000, n - 1, None) == 10     # too small
+    assert lib.attn_fwd_host(*args, 0x10010, n, None) == 10         # misaligned
+    bad = list(args)
+    bad[9] = 100
+    assert lib.attn_fwd_host(*bad, 0x10000, n, None) == 3
+
+
+def test_no_fallback_without_a_device(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    # valid arguments but no B200: the library must report an error, not compute on the CPU
+    assert call(lib) in (7, 8)
+    assert api.attn_query_support(64, 0, False) in (7, 8)
+    assert api.attn_query_support(96, 0, False) == 3
+    assert api.attn_query_support(64, 5, False) == 4

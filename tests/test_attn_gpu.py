@@ -1,0 +1,232 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle, element by element
+on the same seeded inputs.  Tolerances (max-abs): O 1e-2 for fp16, 2e-2 for bf16; LSE 1e-3."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import attn_oracle as orc
+from paper_2506_12355_b200 import api, inputs
+
+pytestmark = pytest.mark.gpu
+
+O_TOL = {inputs.DTYPE_FP16: 1e-2, inputs.DTYPE_BF16: 2e-2}
+LSE_TOL = 1e-3
+GUARD = 4096  # canary elements on both sides of every output buffer
+
+
+def guarded(shape, dtype, device):
+    n = int(np.prod(shape))
+    buf = torch.full((n + 2 * GUARD,), float("nan"), dtype=dtype, device=device)
+    return buf, buf[GUARD:GUARD + n].view(shape)
+
+
+def guards_intact(buf):
+    return bool(torch.isnan(buf[:GUARD]).all()) and bool(torch.isnan(buf[-GUARD:]).all())
+
+
+def run_gpu(fn, q, k, v, scale, causal):
+    dev = torch.device("cuda:0")
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    B, H, Sq, D = q.shape
+    obuf, o = guarded((B, H, Sq, D), q.dtype, dev)
+    lbuf, lse = guarded((B, H, Sq), torch.float32, dev)
+    fn(qd, kd, vd, scale, causal, out=o, lse=lse)
+    assert api.attn_last_device_status() == 0, "a kernel reported a timed-out wait"
+    assert guards_intact(obuf) and guards_intact(lbuf), "write outside the output buffers"
+    return o.cpu(), lse.cpu()
+
+
+def check_against_oracle(fn, q, k, v, dtype, scale, causal, o_tol=None):
+    o, lse = run_gpu(fn, q, k, v, scale, causal)
+    qf, kf, vf = (orc.widen(inputs.bits(t), dtype) for t in (q, k, v))
+    o_ref, lse_ref = orc.attention(qf, kf, vf, scale, causal)
+    o64 = o.to(torch.float64).numpy()
+    assert not np.isnan(o64).any(), "NaN in O (unwritten canary or arithmetic NaN)"
+    err_o = np.abs(o64 - o_ref)
+    where = np.unravel_index(err_o.argmax(), err_o.shape) if err_o.size else None
+    tol = O_TOL[dtype] if o_tol is None else o_tol
+    assert err_o.size == 0 or err_o.max() <= tol, "max |dO| = %g at %s" % (err_o.max(), where)
+    l64 = lse.to(torch.float64).numpy()
+    inf = np.isneginf(lse_ref)
+    assert np.array_equal(np.isneginf(l64), inf)
+    err_l = np.abs(l64[~inf] - lse_ref[~inf])
+    assert err_l.size == 0 or err_l.max() <= LSE_TOL, "max |dLSE| = %g" % err_l.max()
+
+
+IMPLS = {"tc": api.attn_fwd, "simt": api.attn_fwd_simt}
+
+
+# ------------------------------------------------------------------ small shapes, full comparison
+
+SMALL = [
+    # B, H, Sq, Sk
+    (1, 2, 128, 128),
+    (1, 1, 1, 1),
+    (1, 3, 17, 17),
+    (2, 1, 127, 127),
+    (1, 1, 129, 129),
+    (1, 2, 255, 255),
+    (1, 1, 100, 333),
+    (1, 1, 257, 129),
+    (1, 1, 384, 640),
+]
+
+
+@pytest.mark.parametrize("impl", ["tc", "simt"])
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("dtype", [inputs.DTYPE_FP16, inputs.DTYPE_BF16])
+@pytest.mark.parametrize("D", [64, 128, 256])
+@pytest.mark.parametrize("shape", SMALL)
+def test_small_shapes(shape, D, dtype, causal, impl):
+    B, H, Sq, Sk = shape
+    if impl == "simt" and (D == 256 or Sq * Sk > 70000) and dtype == inputs.DTYPE_BF16:
+        pytest.skip("cross-check kernel: subset only")
+    q, k, v = inputs.make_qkv(B, H, Sq, Sk, D, dtype, seed=1000 + Sq * 7 + Sk + D)
+    check_against_oracle(IMPLS[impl], q, k, v, dtype, 1.0 / math.sqrt(D), causal)
+
+
+def test_config_c1_full():
+    cfg = inputs.CONFIGS["C1"]
+    q, k, v = inputs.make_config_inputs(cfg)
+    check_against_oracle(api.attn_fwd, q, k, v, cfg.dtype, cfg.scale, cfg.causal)
+
+
+@pytest.mark.parametrize("D,dtype,causal", [(64, 0, False), (128, 1, True), (256, 0, False), (128, 0, True),
+                                            (64, 1, True)])
+def test_several_tiles_and_ragged_tail(D, dtype, causal):
+    # several 128-row Q tiles and K/V tiles plus a ragged tail, several heads
+    q, k, v = inputs.make_qkv(2, 3, 128 * 3 + 37, 128 * 4 + 91, D, dtype, seed=4242 + D)
+    check_against_oracle(api.attn_fwd, q, k, v, dtype, 1.0 / math.sqrt(D), causal)
+
+
+# ------------------------------------------------------------------ hand-derived cases on the GPU
+
+def test_hand_case_2x2_padded_into_d64():
+    # the 2x2 case of tests/golden/hand_cases.json: exactly representable in fp16, zero-padded to D = 64
+    c = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hand_cases.json")))["case_2x2"]
+    e = math.e
+    for causal, want_o, want_l in (
+            (False, [[(e + 3) / (e + 1), (2 * e + 4) / (e + 1)], [(1 + 3 * e) / (e + 1), (2 + 4 * e) / (e + 1)]],
+             [math.log(e + 1)] * 2),
+            (True, [[1.0, 2.0], [(1 + 3 * e) / (e + 1), (2 + 4 * e) / (e + 1)]], [1.0, math.log(e + 1)])):
+        for dt in (torch.float16, torch.bfloat16):
+            q = torch.zeros(1, 1, 2, 64, dtype=dt)
+            k = torch.zeros(1, 1, 2, 64, dtype=dt)
+            v = torch.zeros(1, 1, 2, 64, dtype=dt)
+            q[0, 0, :, :2] = torch.tensor(c["Q"], dtype=dt)
+            k[0, 0, :, :2] = torch.tensor(c["K"], dtype=dt)
+            v[0, 0, :, :2] = torch.tensor(c["V"], dtype=dt)
+            o, lse = run_gpu(api.attn_fwd, q, k, v, 1.0, causal)
+            tol = 1e-2 if dt == torch.float16 else 2e-2
+            np.testing.assert_allclose(o[0, 0, :, :2].double().numpy(), np.array(want_o), atol=tol)
+            assert float(o[0, 0, :, 2:].abs().max()) == 0.0
+            np.testing.assert_allclose(lse[0, 0].double().numpy(), np.array(want_l), atol=1e-3)
+
+
+# ------------------------------------------------------------------ structured inputs (layout mistakes)
+
+@pytest.mark.parametrize("D", [64, 128, 256])
+def test_constant_v_and_distinct_columns(D):
+    # V column d holds the value d/8 in every row -> O[:, d] = d/8 exactly representable
+    B, H, Sq, Sk = 1, 2, 200, 300
+    q, k, _ = inputs.make_qkv(B, H, Sq, Sk, D, inputs.DTYPE_FP16, seed=99)
+    v = (torch.arange(D, dtype=torch.float32) / 8).to(torch.float16).expand(B, H, Sk, D).contiguous()
+    o, _ = run_gpu(api.attn_fwd, q, k, v, 0.125, False)
+    want = (torch.arange(D, dtype=torch.float64) / 8).expand(B, H, Sq, D)
+    assert float((o.double() - want).abs().max()) <= 2e-2   # |O| up to 32: fp16 spacing there is 1/64..1/32
+
+
+@pytest.mark.parametrize("D", [64, 128, 256])
+def test_one_hot_selection_follows_key_index(D):
+    # query i matches key perm[i] strongly -> O row i must be V[perm[i]]: catches transposed or
+    # permuted K/V/P tiles
+    Sq = Sk = 256
+    g = torch.Generator().manual_seed(7)
+    perm = torch.randperm(Sk, generator=g)
+    basis = torch.zeros(Sk, D)
+    # distinct +-1 codes per key: code of key j = binary digits of j spread over the first 16 dims
+    for bit in range(8):
+        basis[:, bit] = ((torch.arange(Sk) >> bit) & 1).float() * 2 - 1
+    k = basis.to(torch.float16).view(1, 1, Sk, D).contiguous()
+    q = basis[perm].to(torch.float16).view(1, 1, Sq, D).contiguous()
+    v = inputs.randn16((1, 1, Sk, D), 5, inputs.DTYPE_FP16)
+    o, lse = run_gpu(api.attn_fwd, q, k, v, 16.0, False)   # score gap between best and next: 2*16
+    want = v[0, 0, perm].double()
+    assert float((o[0, 0].double() - want).abs().max()) <= 1e-2
+    np.testing.assert_allclose(lse[0, 0].numpy(), np.full(Sq, 8 * 16.0), atol=1e-3)
+
+
+def test_zero_scale_and_no_keys():
+    q, k, v = inputs.make_qkv(1, 2, 150, 150, 64, inputs.DTYPE_BF16, seed=31)
+    check_against_oracle(api.attn_fwd, q, k, v, inputs.DTYPE_BF16, 0.0, True)
+    # Sk == 0: O = 0, LSE = -inf
+    k0 = torch.empty(1, 2, 0, 64, dtype=torch.bfloat16)
+    o, lse = run_gpu(api.attn_fwd, q, k0, k0, 0.125, False)
+    assert float(o.abs().max()) == 0.0 and bool(torch.isneginf(lse).all())
+
+
+def test_large_logits_do_not_overflow():
+    q, k, v = inputs.make_qkv(1, 1, 256, 256, 128, inputs.DTYPE_FP16, seed=32)
+    check_against_oracle(api.attn_fwd, q, k, v, inputs.DTYPE_FP16, 8.0, False)
+
+
+def test_bitwise_deterministic():
+    q, k, v = inputs.make_qkv(2, 4, 512, 512, 128, inputs.DTYPE_BF16, seed=33)
+    o1, l1 = run_gpu(api.attn_fwd, q, k, v, 0.09, True)
+    o2, l2 = run_gpu(api.attn_fwd, q, k, v, 0.09, True)
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1, l2)
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+
+def test_host_entry_matches_device_entry():
+    cfg = inputs.CONFIGS["C1"]
+    q, k, v = inputs.make_config_inputs(cfg)
+    o_dev, lse_dev = run_gpu(api.attn_fwd, q, k, v, cfg.scale, cfg.causal)
+    qp, kp, vp = q.pin_memory(), k.pin_memory(), v.pin_memory()
+    o = torch.empty_like(q).pin_memory()
+    lse = torch.empty(cfg.B, cfg.H, cfg.Sq, dtype=torch.float32).pin_memory()
+    ws = torch.empty(api.attn_fwd_host_workspace_bytes(cfg.B, cfg.H, cfg.Sq, cfg.Sk, cfg.D),
+                     dtype=torch.uint8, device="cuda:0")
+    api.attn_fwd_host(qp, kp, vp, cfg.scale, cfg.causal, o, lse, ws)
+    assert api.attn_last_device_status() == 0
+    assert torch.equal(o.view(torch.int16), o_dev.view(torch.int16)) and torch.equal(lse, lse_dev)
+
+
+# ------------------------------------------------------------------ full-size configurations, sampled rows
+
+@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5"])
+def test_full_size_configs_on_sampled_rows(name):
+    cfg = inputs.CONFIGS[name]
+    q, k, v = inputs.make_config_inputs(cfg)
+    o, lse = run_gpu(api.attn_fwd, q, k, v, cfg.scale, cfg.causal)
+    rows = inputs.sample_rows(cfg.B * cfg.H * cfg.Sq, cfg.Sq, 192, seed=cfg.index)
+    o_ref, lse_ref = orc.attention_rows_16(inputs.bits(q), inputs.bits(k), inputs.bits(v), cfg.dtype, rows,
+                                           cfg.scale, cfg.causal)
+    got_o = o.view(-1, cfg.D)[torch.from_numpy(rows)].double().numpy()
+    got_l = lse.view(-1)[torch.from_numpy(rows)].double().numpy()
+    err = np.abs(got_o - o_ref)
+    assert err.max() <= O_TOL[cfg.dtype], "max |dO| = %g at sampled row %d" % (err.max(), rows[err.max(axis=1).argmax()])
+    assert np.abs(got_l - lse_ref).max() <= LSE_TOL
+    # properties that hold at any size, over ALL rows: finite outputs, |O| bounded by max |V| per head
+    assert bool(torch.isfinite(o.float()).all()) and bool(torch.isfinite(lse).all())
+    vmax = v.float().abs().amax(dim=(2, 3), keepdim=True)
+    assert bool((o.float().abs() <= vmax * (1 + 1e-2)).all())
+    if cfg.causal:   # causal row 0 returns V[0]
+        assert torch.equal(o[:, :, 0].view(torch.int16), v[:, :, 0].view(torch.int16))
+
+
+@pytest.mark.parametrize("name", ["C2", "C3"])
+def test_tensor_core_kernel_agrees_with_cross_check_kernel_everywhere(name):
+    # all rows of a full-size configuration: the two independent CUDA kernels agree within the
+    # sum of their tolerances (the oracle itself covers sampled rows above)
+    cfg = inputs.CONFIGS[name]
+    q, k, v = inputs.make_config_inputs(cfg)
+    o1, l1 = run_gpu(api.attn_fwd, q, k, v, cfg.scale, cfg.causal)
+    o2, l2 = run_gpu(api.attn_fwd_simt, q, k, v, cfg.scale, cfg.causal)
+    assert float((o1.float() - o2.float()).abs().max()) <= 2 * O_TOL[cfg.dtype]
+    assert float((l1 - l2).abs().max()) <= 2 * LSE_TOL

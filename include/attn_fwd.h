@@ -65,6 +65,8 @@ typedef enum {
  * lse     : device pointer, [B,H,Sq] fp32 (written).
  * B, H, Sq, Sk >= 0;  D in {64, 128, 256};  B*H <= 2^31-1, Sq, Sk <= 2^31-1-256.
  * B*H*Sq == 0 is a successful no-op.  Sk == 0 writes O = 0 and LSE = -inf.
+ * Pointers of tensors without elements may be NULL (q, o, lse when B*H*Sq == 0; k, v when
+ * B*H*Sk == 0); every other pointer must be non-NULL.
  * Runs on sm_100a tensor cores (tcgen05 MMAs with TMEM accumulators, TMA tile loads).
  * Validation happens on the host before anything is enqueued; on an error nothing is
  * launched.

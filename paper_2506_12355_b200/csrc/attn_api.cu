@@ -12,6 +12,7 @@
 #include "../../include/attn_fwd.h"
 #include "attn_simt.cuh"
 #include "attn_tc_basic.cuh"
+#include "attn_tc_pipe.cuh"
 
 namespace {
 
@@ -65,8 +66,11 @@ constexpr int kMaxSeq = 2147483647 - 256;
 // Validation shared by every entry point; no CUDA call happens here.
 int validate(const void* q, const void* k, const void* v, const void* o, const void* lse, int B, int H, int Sq,
              int Sk, int D, float scale, int dtype, bool device_pointers) {
-    if (!q || !k || !v || !o || !lse) return ATTN_ERR_NULL_POINTER;
     if (B < 0 || H < 0 || Sq < 0 || Sk < 0 || D < 0) return ATTN_ERR_BAD_SHAPE;
+    // empty tensors may come with NULL pointers (an allocator returns none for zero bytes)
+    const bool no_rows = static_cast<int64_t>(B) * H * Sq == 0, no_keys = static_cast<int64_t>(B) * H * Sk == 0;
+    if (!no_rows && (!q || !o || !lse)) return ATTN_ERR_NULL_POINTER;
+    if (!no_rows && !no_keys && (!k || !v)) return ATTN_ERR_NULL_POINTER;
     if (Sq > kMaxSeq || Sk > kMaxSeq) return ATTN_ERR_BAD_SHAPE;
     if (static_cast<int64_t>(B) * H > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
     if (D != 64 && D != 128 && D != 256) return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
@@ -126,6 +130,47 @@ int launch_tc_basic(const void* q, const void* k, const void* v, void* o, float*
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
+// Pipelined, warp-specialised kernel (head dims 64 and 128): one CTA per pair of 128-row Q tiles.
+template <int D, int DTYPE>
+int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
+                   float scale, int causal, cudaStream_t st) {
+    using C = attn_tc::PipeCfg<D>;
+    auto kern = attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    });
+    if (attr_err != cudaSuccess) return ATTN_ERR_CUDA;
+    const int64_t BH = static_cast<int64_t>(B) * H;
+    const int64_t n_pairs = (static_cast<int64_t>(Sq) + 2 * C::BM - 1) / (2 * C::BM);
+    if (n_pairs * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
+    CUtensorMap mq, mk, mv;
+    if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, BH, Sk, D, C::BN) ||
+        !make_map(&mv, v, DTYPE, BH, Sk, D, C::BN))
+        return ATTN_ERR_CUDA;
+    attn_tc::PipeParams prm;
+    prm.o = o;
+    prm.lse = lse;
+    prm.Sq = Sq;
+    prm.Sk = Sk;
+    prm.scale = scale;
+    prm.scale_log2 = scale * 1.4426950408889634f;
+    prm.causal = causal ? 1 : 0;
+    prm.status = device_status_ptr();
+    if (!prm.status) return ATTN_ERR_CUDA;
+    prm.n_pairs = static_cast<int>(n_pairs);
+    prm.BH = static_cast<int>(BH);
+    // walk together as many heads as keep their K and V (2 * Sk * D * 2 bytes each) inside ~48 MB of L2
+    const int64_t kv_bytes_per_head = 4LL * Sk * D;
+    int64_t hpg = (48LL << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
+    if (hpg < 1) hpg = 1;
+    if (hpg > BH) hpg = BH;
+    prm.heads_per_group = static_cast<int>(hpg);
+    kern<<<static_cast<unsigned>(n_pairs * BH), C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, prm);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
 template <int D, int DTYPE>
 int launch_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
                 float scale, int causal, cudaStream_t st) {
@@ -138,7 +183,7 @@ int launch_simt(const void* q, const void* k, const void* v, void* o, float* lse
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
-enum class Impl { TensorCore, Simt };
+enum class Impl { TensorCore, TensorCoreBasic, Simt };
 
 template <Impl IMPL>
 int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk, int D,
@@ -154,7 +199,9 @@ int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, i
 #define ATTN_CASE(DD, TT)                                                                              \
     if (D == DD && dtype == TT) {                                                                      \
         if (IMPL == Impl::Simt) return launch_simt<DD, TT>(q, k, v, o, lse, B, H, Sq, Sk, scale, causal, st); \
-        return launch_tc_basic<DD, TT>(q, k, v, o, lse, B, H, Sq, Sk, scale, causal, st);              \
+        if (IMPL == Impl::TensorCoreBasic || DD == 256)                                                \
+            return launch_tc_basic<DD, TT>(q, k, v, o, lse, B, H, Sq, Sk, scale, causal, st);          \
+        return launch_tc_pipe<(DD == 256 ? 128 : DD), TT>(q, k, v, o, lse, B, H, Sq, Sk, scale, causal, st); \
     }
     ATTN_CASE(64, 0)
     ATTN_CASE(64, 1)

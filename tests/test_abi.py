@@ -73,6 +73,9 @@ def test_argument_validation_happens_before_any_launch(lib, fn):
     # empty problems are a successful no-op, decided before the device is looked at
     assert call(lib, fn, B=0) == 0
     assert call(lib, fn, Sq=0) == 0
+    assert call(lib, fn, Sq=0, q=None, o=None, lse=None) == 0
+    # k, v may be NULL only when there are no keys (that case reaches the device check)
+    assert call(lib, fn, Sk=0, k=None, v=None) != 1
 
 
 def test_host_entry_validation(lib):

@@ -14,6 +14,13 @@
 #include "attn_tc_basic.cuh"
 #include "attn_tc_pipe.cuh"
 
+// Share of the exponentials evaluated by a polynomial on the FMA pipe instead of the special-function
+// unit (POLY_NUM of every POLY_DEN element pairs).
+#ifndef ATTN_POLY_NUM
+#define ATTN_POLY_NUM 2
+#define ATTN_POLY_DEN 5
+#endif
+
 namespace {
 
 // Device-side status word: 0, or ATTN_ERR_DEVICE_TIMEOUT once a kernel gave up on a wait.
@@ -130,12 +137,16 @@ int launch_tc_basic(const void* q, const void* k, const void* v, void* o, float*
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
+#ifdef ATTN_TC_PROFILE
+long long* g_prof_buffer = nullptr;  // development builds: per-CTA cycle sums, [grid][32]
+#endif
+
 // Pipelined, warp-specialised kernel (head dims 64 and 128): one CTA per pair of 128-row Q tiles.
 template <int D, int DTYPE>
 int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
                    float scale, int causal, cudaStream_t st) {
     using C = attn_tc::PipeCfg<D>;
-    auto kern = attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE>;
+    auto kern = attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE, ATTN_POLY_NUM, ATTN_POLY_DEN>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -167,6 +178,9 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     if (hpg < 1) hpg = 1;
     if (hpg > BH) hpg = BH;
     prm.heads_per_group = static_cast<int>(hpg);
+#ifdef ATTN_TC_PROFILE
+    prm.prof = g_prof_buffer;
+#endif
     kern<<<static_cast<unsigned>(n_pairs * BH), C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, prm);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
@@ -283,6 +297,10 @@ int attn_last_device_status(void* stream) {
     }
     return h == 0 ? ATTN_OK : ATTN_ERR_DEVICE_TIMEOUT;
 }
+
+#ifdef ATTN_TC_PROFILE
+void attn_debug_set_profile_buffer(long long* device_buffer) { g_prof_buffer = device_buffer; }
+#endif
 
 const char* attn_status_string(int status) {
     switch (status) {

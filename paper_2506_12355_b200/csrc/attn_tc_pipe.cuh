@@ -50,12 +50,32 @@ struct PipeParams {
     int n_pairs;          // 256-row Q tile pairs per head
     int BH;               // batch * heads
     int heads_per_group;  // heads whose K/V are walked together (L2 residency)
+#ifdef ATTN_TC_PROFILE
+    long long* prof;      // [grid][32] cycle sums per phase (development builds only)
+#endif
 };
+
+#ifndef ATTN_MAX3
+#define ATTN_MAX3 0
+#endif
+
+#ifndef ATTN_PROF_ROW
+#define ATTN_PROF_ROW 0
+#endif
+#ifdef ATTN_TC_PROFILE
+#define PROF_DECL(n) long long prof_t0 = clock64(), prof_acc[n] = {}
+#define PROF_LAP(i) do { const long long prof_t1 = clock64(); prof_acc[i] += prof_t1 - prof_t0; prof_t0 = prof_t1; } while (0)
+#define PROF_FLUSH(base, n) do { for (int i_ = 0; i_ < (n); ++i_) prm.prof[blockIdx.x * 32 + (base) + i_] = prof_acc[i_]; } while (0)
+#else
+#define PROF_DECL(n)
+#define PROF_LAP(i)
+#define PROF_FLUSH(base, n)
+#endif
 
 __device__ __forceinline__ void reg_inc_224() { asm volatile("setmaxnreg.inc.sync.aligned.u32 224;"); }
 __device__ __forceinline__ void reg_dec_56() { asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); }
 
-template <int D, int DTYPE>
+template <int D, int DTYPE, int POLY_NUM, int POLY_DEN>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const PipeParams prm) {
@@ -71,7 +91,8 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     // misc area: barriers
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
     const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
-    enum { B_Q = 0, B_SFULL = 2, B_PFULL = 4, B_OFINAL = 6, B_KVFULL = 8, B_KVEMPTY = 8 + NSLOT, B_COUNT = 8 + 2 * NSLOT };
+    enum { B_Q = 0, B_SFULL = 2, B_PFULL = 4, B_PFULL2 = 6, B_OFINAL = 8, B_KVFULL = 10, B_KVEMPTY = 10 + NSLOT,
+           B_COUNT = 10 + 2 * NSLOT };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 1;
@@ -113,7 +134,8 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         mbar_init(bar(B_Q + 1), 1);
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar(B_SFULL + t), 1);
-            mbar_init(bar(B_PFULL + t), 128);
+            mbar_init(bar(B_PFULL + t), 128);    // first three quarters of P_t written
+            mbar_init(bar(B_PFULL2 + t), 128);   // rest of P_t written
             mbar_init(bar(B_OFINAL + t), 1);
         }
         for (int s = 0; s < NSLOT; ++s) {
@@ -139,20 +161,32 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 
     if (warp >= 8) {
         reg_dec_56();
-        if (warp == 9 && lane == 0) {
+        // Both service warps run their loops with all 32 lanes (uniform control flow keeps the
+        // address arithmetic on the uniform datapath); one elected lane issues the TMA / MMA
+        // instructions.
+        if (warp == 9) {
             // =========================== TMA producer ===========================
+            const bool leader = elect_one();
+            PROF_DECL(2);
             auto load_q = [&](int t) {
-                mbar_arrive_expect_tx(bar(B_Q + t), C::Q_BYTES);
-                for (int bx = 0; bx < NBOX; ++bx)
-                    tma_load_3d(sQ(t) + bx * BM * 128, &tmQ, bar(B_Q + t), bx * 64, q0 + t * BM, bh);
+                if (leader) {
+                    mbar_arrive_expect_tx(bar(B_Q + t), C::Q_BYTES);
+#pragma unroll
+                    for (int bx = 0; bx < NBOX; ++bx)
+                        tma_load_3d(sQ(t) + bx * BM * 128, &tmQ, bar(B_Q + t), bx * 64, q0 + t * BM, bh);
+                }
             };
             auto load_kv = [&](const CUtensorMap* map, int item, int j) -> bool {
                 const int slot = item % NSLOT;
                 const uint32_t use = item / NSLOT;
                 if (!mbar_wait(bar(B_KVEMPTY + slot), (use & 1) ^ 1, abort_flag)) return false;
-                mbar_arrive_expect_tx(bar(B_KVFULL + slot), C::KV_BYTES);
-                for (int bx = 0; bx < NBOX; ++bx)
-                    tma_load_3d(sKV(slot) + bx * BN * 128, map, bar(B_KVFULL + slot), bx * 64, j * BN, bh);
+                PROF_LAP(0);
+                if (leader) {
+                    mbar_arrive_expect_tx(bar(B_KVFULL + slot), C::KV_BYTES);
+#pragma unroll
+                    for (int bx = 0; bx < NBOX; ++bx)
+                        tma_load_3d(sKV(slot) + bx * BN * 128, map, bar(B_KVFULL + slot), bx * 64, j * BN, bh);
+                }
                 return true;
             };
             if (n_kv[0] > 0) load_q(0);
@@ -160,25 +194,41 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (!load_kv(&tmK, 2 * j, j)) break;
                 if (j == 0 && n_kv[1] > 0) load_q(1);
                 if (!load_kv(&tmV, 2 * j + 1, j)) break;
+                PROF_LAP(1);
             }
-        } else if (warp == 8 && lane == 0) {
+#ifdef ATTN_TC_PROFILE
+            if (leader) PROF_FLUSH(24, 2);
+#endif
+        } else if (warp == 8) {
             // =========================== MMA issuer ===========================
+            const bool leader = elect_one();
             constexpr uint32_t IDESC_S = make_idesc_f16(BM, BN, DTYPE, 0, 0);
             constexpr uint32_t IDESC_O = make_idesc_f16(BM, D, DTYPE, 0, 1);
-            auto issue_s = [&](int t, int slot) {
+            constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
+            const uint32_t q_lo[2] = {smem_desc_lo(sQ(0), 16), smem_desc_lo(sQ(1), 16)};
+            const uint32_t k_lo0 = smem_desc_lo(sKV(0), 16);          // K tile in slot 0 (K-major)
+            const uint32_t v_lo0 = smem_desc_lo(sKV(0), BN * 128);    // V tile in slot 0 (MN-major)
+            auto issue_s = [&](int t, int slot) {   // S_t = Q_t K^T : D/16 instructions of K = 16
+                if (leader) {
+                    const uint32_t a0 = q_lo[t], b0 = k_lo0 + slot * (C::KV_BYTES >> 4);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * 128 * 128 + (kk & 3) * 32;
-                    mma_f16_ss(tmem + C::s_col(t), make_smem_desc_sw128(sQ(t) + off, 16, 1024),
-                               make_smem_desc_sw128(sKV(slot) + off, 16, 1024), IDESC_S, kk > 0);
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = ((kk >> 2) * 128 * 128 + (kk & 3) * 32) >> 4;
+                        mma_f16_ss_lohi(tmem + C::s_col(t), a0 + off, b0 + off, DESC_HI, IDESC_S, kk > 0);
+                    }
                 }
             };
-            auto issue_pv = [&](int t, int slot, bool accumulate) {
+            auto issue_pv = [&](int t, int slot, bool accumulate, int kk_begin, int kk_end) {
+                if (leader) {                       // O_t += P_t V : K = 16 keys per instruction
+                    const uint32_t b0 = v_lo0 + slot * (C::KV_BYTES >> 4);
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)
-                    mma_f16_ts(tmem + C::o_col(t), tmem + C::s_col(t) + kk * 8,
-                               make_smem_desc_sw128(sKV(slot) + kk * 16 * 128, BN * 128, 1024), IDESC_O,
-                               (accumulate || kk > 0) ? 1u : 0u);
+                    for (int kk = kk_begin; kk < kk_end; ++kk)
+                        mma_f16_ts_lohi(tmem + C::o_col(t), tmem + C::s_col(t) + kk * 8, b0 + ((kk * 16 * 128) >> 4),
+                                        DESC_HI, IDESC_O, (accumulate || kk > 0) ? 1u : 0u);
+                }
+            };
+            auto commit = [&](int b) {
+                if (leader) mma_commit(bar(b));
             };
             auto kv_full_wait = [&](int item) {
                 return mbar_wait(bar(B_KVFULL + item % NSLOT), (item / NSLOT) & 1, abort_flag);
@@ -190,45 +240,63 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (ok && n_kv[0] > 0) {
                     tc_fence_after_sync();
                     issue_s(0, 0);
-                    mma_commit(bar(B_SFULL + 0));
+                    commit(B_SFULL + 0);
                 }
                 if (ok && n_kv[1] > 0) {
                     ok = mbar_wait(bar(B_Q + 1), 0, abort_flag);
                     if (ok) {
                         tc_fence_after_sync();
                         issue_s(1, 0);
-                        mma_commit(bar(B_SFULL + 1));
+                        commit(B_SFULL + 1);
                     }
                 }
-                if (ok) mma_commit(bar(B_KVEMPTY + 0));
+                if (ok) commit(B_KVEMPTY + 0);
             }
+            PROF_DECL(12);
             for (int j = 0; j < n_max && ok; ++j) {
                 const int vitem = 2 * j + 1, kitem = 2 * j + 2;
                 const int vslot = vitem % NSLOT, kslot = kitem % NSLOT;
                 const uint32_t par = j & 1;
-                bool k_ready = false;
+                // both tiles of this step are normally long loaded: check them off the P -> S critical path
                 if (!(ok = kv_full_wait(vitem))) break;
+                bool k_ready = false;
+                if (j + 1 < n_max) {
+                    if (!(ok = kv_full_wait(kitem))) break;
+                    k_ready = true;
+                }
+                PROF_LAP(0);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (j < n_kv[t]) {
                         if (!(ok = mbar_wait(bar(B_PFULL + t), par, abort_flag))) break;
+                        PROF_LAP(1 + 5 * t);
                         tc_fence_after_sync();
-                        issue_pv(t, vslot, j > 0);
-                        if (j + 1 == n_kv[t]) mma_commit(bar(B_OFINAL + t));
+                        issue_pv(t, vslot, j > 0, 0, 3 * BN / 64);
+                        if (!(ok = mbar_wait(bar(B_PFULL2 + t), par, abort_flag))) break;
+                        PROF_LAP(2 + 5 * t);
+                        tc_fence_after_sync();
+                        issue_pv(t, vslot, true, 3 * BN / 64, BN / 16);
+                        if (j + 1 == n_kv[t]) commit(B_OFINAL + t);
                     }
-                    if (t == 1) mma_commit(bar(B_KVEMPTY + vslot));
+                    if (t == 1) commit(B_KVEMPTY + vslot);
+                    PROF_LAP(3 + 5 * t);
                     if (j + 1 < n_kv[t]) {
                         if (!k_ready) {
                             if (!(ok = kv_full_wait(kitem))) break;
                             k_ready = true;
                         }
+                        PROF_LAP(4 + 5 * t);
                         tc_fence_after_sync();
                         issue_s(t, kslot);
-                        mma_commit(bar(B_SFULL + t));
+                        commit(B_SFULL + t);
                     }
+                    PROF_LAP(5 + 5 * t);
                 }
-                if (ok && j + 1 < n_max) mma_commit(bar(B_KVEMPTY + kslot));
+                if (ok && j + 1 < n_max) commit(B_KVEMPTY + kslot);
             }
+#ifdef ATTN_TC_PROFILE
+            if (leader) PROF_FLUSH(0, 12);
+#endif
         }
     } else {
         // =========================== softmax groups ===========================
@@ -243,19 +311,23 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         float m = -INFINITY, l = 0.f;
         bool ok = true;
 
+        PROF_DECL(6);
         for (int j = 0; j < n; ++j) {
             if (!(ok = mbar_wait(bar(B_SFULL + t), j & 1, abort_flag))) break;
+            PROF_LAP(0);
             tc_fence_after_sync();
             uint32_t sr[BN];
 #pragma unroll
             for (int ch = 0; ch < BN / 32; ++ch) tmem_ld_32x32b_x32(tS + ch * 32, sr + ch * 32);
             tmem_ld_wait();
+            PROF_LAP(1);
 
             const int kv0 = j * BN;
             const bool need_mask = (kv0 + BN > prm.Sk) || (prm.causal && kv0 + BN - 1 > q0 + t * BM);
-            float mx = -INFINITY;
-            if (need_mask) {
+            float mx;
+            if (need_mask) {  // diagonal or ragged tile: rare, kept out of the hot path
                 const int lim = (prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1;  // last visible key
+                mx = -INFINITY;
 #pragma unroll
                 for (int e = 0; e < BN; ++e) {
                     const float s = (kv0 + e <= lim) ? __uint_as_float(sr[e]) : -INFINITY;
@@ -263,9 +335,25 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     mx = fmaxf(mx, s);
                 }
             } else {
+                float mxs[8];   // eight independent chains keep the max off the latency-bound path
 #pragma unroll
-                for (int e = 0; e < BN; ++e) mx = fmaxf(mx, __uint_as_float(sr[e]));
+                for (int i = 0; i < 8; ++i) mxs[i] = fmaxf(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
+#pragma unroll
+                for (int e = 16; e < BN; e += 16)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+#if ATTN_MAX3
+                        mxs[i] = max3(mxs[i], __uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1]));
+#else
+                        mxs[i] = fmaxf(mxs[i], fmaxf(__uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1])));
+#endif
+                    }
+                mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])), fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
             }
+#ifdef ATTN_TC_PROFILE
+            if (mx == 12345.678f) prm.prof[0] = 1;   // keeps the max in front of the lap
+#endif
+            PROF_LAP(5);
             // advance the reference maximum only when the true one ran ahead by more than 2^8
             float alpha = 1.f;
             if (j == 0) {
@@ -274,26 +362,6 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 alpha = ex2_approx((m - mx) * c);
                 m = mx;
             }
-            const float mc = m * c;
-            float rs = 0.f;
-#pragma unroll
-            for (int ch = 0; ch < BN / 32; ++ch) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    const float s0 = __uint_as_float(sr[ch * 32 + e]), s1 = __uint_as_float(sr[ch * 32 + e + 1]);
-                    float p0 = ex2_approx(fmaf(s0, c, -mc)), p1 = ex2_approx(fmaf(s1, c, -mc));
-                    if (need_mask) {  // -inf * 0 would be NaN for a zero scale
-                        p0 = (s0 == -INFINITY) ? 0.f : p0;
-                        p1 = (s1 == -INFINITY) ? 0.f : p1;
-                    }
-                    rs += p0 + p1;
-                    pk[e / 2] = pack2<DTYPE>(p0, p1);
-                }
-                tmem_st_32x32b_x16(tS + ch * 16, pk);   // P overwrites the S columns already consumed
-            }
-            l = l * alpha + rs;
-
             // rare: rescale the running O (its last update finished before S_j was produced)
             if (__any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll
@@ -306,10 +374,73 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     tmem_st_32x32b_x32(tO + ch * 32, orr);
                 }
             }
+            const float mc = m * c;
+            PROF_LAP(2);
+            float rs;
+            if (need_mask) {
+                rs = 0.f;
+#pragma unroll
+                for (int ch = 0; ch < BN / 32; ++ch) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const float s0 = __uint_as_float(sr[ch * 32 + e]), s1 = __uint_as_float(sr[ch * 32 + e + 1]);
+                        // masked entries are -inf; keep them 0 also for a zero scale (-inf * 0 = NaN)
+                        const float p0 = (s0 == -INFINITY) ? 0.f : ex2_approx(fmaf(s0, c, -mc));
+                        const float p1 = (s1 == -INFINITY) ? 0.f : ex2_approx(fmaf(s1, c, -mc));
+                        rs += p0 + p1;
+                        pk[e / 2] = pack2<DTYPE>(p0, p1);
+                    }
+                    tmem_st_32x32b_x16(tS + ch * 16, pk);   // P overwrites the S columns already consumed
+                    if (ch == BN / 32 - 2) {                // first three quarters of P are in place
+                        tmem_st_wait();
+                        tc_fence_before_sync();
+                        mbar_arrive(bar(B_PFULL + t));
+                    }
+                }
+            } else {
+                const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
+                uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // 8 partial row sums
+#pragma unroll
+                for (int ch = 0; ch < BN / 32; ++ch) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const uint64_t s2 = pack_f32x2(__uint_as_float(sr[ch * 32 + e]), __uint_as_float(sr[ch * 32 + e + 1]));
+                        const uint64_t x2 = fma_f32x2(s2, c2, nmc2);
+                        float x0, x1, p0, p1;
+                        unpack_f32x2(x2, x0, x1);
+                        if (((ch * 16 + e / 2) % POLY_DEN) < POLY_NUM) {   // this pair: polynomial on the FMA pipe
+                            ex2_poly_f32x2(pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f)), p0, p1);
+                        } else {                                           // this pair: special-function unit
+                            p0 = ex2_approx(x0);
+                            p1 = ex2_approx(x1);
+                        }
+                        acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(p0, p1));
+                        pk[e / 2] = pack2<DTYPE>(p0, p1);
+                    }
+                    tmem_st_32x32b_x16(tS + ch * 16, pk);
+                    if (ch == BN / 32 - 2) {
+                        tmem_st_wait();
+                        tc_fence_before_sync();
+                        mbar_arrive(bar(B_PFULL + t));
+                    }
+                }
+                float a0, a1, a2, a3;
+                unpack_f32x2(add_f32x2(acc[0], acc[1]), a0, a1);
+                unpack_f32x2(add_f32x2(acc[2], acc[3]), a2, a3);
+                rs = (a0 + a1) + (a2 + a3);
+            }
+            l = l * alpha + rs;
+            PROF_LAP(3);
             tmem_st_wait();
             tc_fence_before_sync();
-            mbar_arrive(bar(B_PFULL + t));
+            mbar_arrive(bar(B_PFULL2 + t));
+            PROF_LAP(4);
         }
+#ifdef ATTN_TC_PROFILE
+        if (r == ATTN_PROF_ROW) PROF_FLUSH(12 + 6 * t, 6);
+#endif
 
         // ---- epilogue: O / l and LSE ----
         if (ok && n > 0) ok = mbar_wait(bar(B_OFINAL + t), 0, abort_flag);

@@ -263,6 +263,39 @@ __device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uin
         : "memory");
 }
 
+// Same MMAs with the 64-bit shared-memory descriptors given as (low word, shared high word):
+// the high word (stride, version, swizzle) is constant, the low word holds the start address.
+__device__ __forceinline__ constexpr uint32_t smem_desc_hi_sw128(uint32_t sbo_bytes) {
+    return ((sbo_bytes >> 4) & 0x3fffu) | (1u << 14) | (2u << 29);
+}
+
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3ffffu) >> 4) | (((lbo_bytes >> 4) & 0x3fffu) << 16);
+}
+
+__device__ __forceinline__ void mma_f16_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                                uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void mma_f16_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
+                                                uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // Makes `bar` (one arrival) complete when every MMA this thread has issued so far is done.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
@@ -275,6 +308,54 @@ __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// Packed pairs of fp32 (one 64-bit register): two FMAs / adds per issued instruction.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// 2^x for a packed pair without the special-function unit: split x into a rounded integer and a
+// fraction f in [-0.5, 0.5] with the 1.5 * 2^23 magic constant, evaluate a degree-3 minimax
+// polynomial of 2^f (relative error 7.5e-5) and add the integer to the exponent bits.
+// x must already be clamped to >= -126.
+__device__ __forceinline__ void ex2_poly_f32x2(uint64_t x2, float& r0, float& r1) {
+    const uint64_t magic = pack_f32x2(12582912.f, 12582912.f), nmagic = pack_f32x2(-12582912.f, -12582912.f);
+    const uint64_t neg1 = pack_f32x2(-1.f, -1.f);
+    const uint64_t y2 = add_f32x2(x2, magic);                       // integer part in the low mantissa bits
+    const uint64_t f2 = fma_f32x2(add_f32x2(y2, nmagic), neg1, x2);  // x - round(x)
+    uint64_t p2 = fma_f32x2(f2, pack_f32x2(0.0551716628f, 0.0551716628f), pack_f32x2(0.242611122f, 0.242611122f));
+    p2 = fma_f32x2(p2, f2, pack_f32x2(0.693260987f, 0.693260987f));
+    p2 = fma_f32x2(p2, f2, pack_f32x2(0.999928074f, 0.999928074f));
+    float y0, y1, p0, p1;
+    unpack_f32x2(y2, y0, y1);
+    unpack_f32x2(p2, p0, p1);
+    r0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(y0) << 23));
+    r1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(y1) << 23));
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 
 template <int DTYPE>  // 0 = fp16, 1 = bf16; `lo` lands in bits [0,16)

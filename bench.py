@@ -31,8 +31,8 @@ METRIC = "attention fwd TFLOP/s at 1 B200 and % of dense FP16/BF16 tensor peak"
 UNIT = "TFLOP/s"
 
 # DRAM bytes (read + write) of one launch of the attention kernel on the default workload, from
-# the ncu capture summarised under profiles/ ; None until a capture exists.
-NCU_TRAFFIC_BYTES = {}
+# the ncu captures summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch).
+NCU_TRAFFIC_BYTES = {"C5": 567207168, "C3": 258795520, "C2": 52087296}
 
 
 def load_peaks():
@@ -261,7 +261,10 @@ def run_ours(args, cfg):
     # ---- the oracle timed on this machine's host cores (bounded sample) ----
     cpu = None
     if not args.no_cpu_baseline:
-        rph = ORACLE_ROWS_PER_HEAD[cfg.name]
+        # calibrate on a small sample, then size the timed sample for roughly 15 s of CPU work
+        cal = max(1, ORACLE_ROWS_PER_HEAD[cfg.name] // 8)
+        cal_t, _, _, _ = time_oracle(cfg, q, k, v, cal)
+        rph = int(min(cfg.Sq, max(cal, cal * 15.0 / max(cal_t[0], 1e-6))))
         times, fl, n_rows, cores = time_oracle(cfg, q, k, v, rph)
         cpu = {"value": fl / times[0] / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": sample_text(cfg, n_rows, rph), "seconds": times[0]}

@@ -17,8 +17,8 @@
 // Share of the exponentials evaluated by a polynomial on the FMA pipe instead of the special-function
 // unit (POLY_NUM of every POLY_DEN element pairs).
 #ifndef ATTN_POLY_NUM
-#define ATTN_POLY_NUM 2
-#define ATTN_POLY_DEN 5
+#define ATTN_POLY_NUM 1
+#define ATTN_POLY_DEN 4
 #endif
 
 namespace {

@@ -55,6 +55,9 @@ struct PipeParams {
 #endif
 };
 
+#ifndef ATTN_SUM_MODE
+#define ATTN_SUM_MODE 0
+#endif
 #ifndef ATTN_MAX3
 #define ATTN_MAX3 0
 #endif
@@ -65,10 +68,12 @@ struct PipeParams {
 #ifdef ATTN_TC_PROFILE
 #define PROF_DECL(n) long long prof_t0 = clock64(), prof_acc[n] = {}
 #define PROF_LAP(i) do { const long long prof_t1 = clock64(); prof_acc[i] += prof_t1 - prof_t0; prof_t0 = prof_t1; } while (0)
+#define PROF_STAMP(cond, slot) do { if (cond) prm.prof[blockIdx.x * 32 + (slot)] = clock64(); } while (0)
 #define PROF_FLUSH(base, n) do { for (int i_ = 0; i_ < (n); ++i_) prm.prof[blockIdx.x * 32 + (base) + i_] = prof_acc[i_]; } while (0)
 #else
 #define PROF_DECL(n)
 #define PROF_LAP(i)
+#define PROF_STAMP(cond, slot)
 #define PROF_FLUSH(base, n)
 #endif
 
@@ -273,6 +278,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         tc_fence_after_sync();
                         issue_pv(t, vslot, j > 0, 0, 3 * BN / 64);
                         if (!(ok = mbar_wait(bar(B_PFULL2 + t), par, abort_flag))) break;
+                        PROF_STAMP(leader && t == 0 && j == 64, 27);
                         PROF_LAP(2 + 5 * t);
                         tc_fence_after_sync();
                         issue_pv(t, vslot, true, 3 * BN / 64, BN / 16);
@@ -289,6 +295,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         tc_fence_after_sync();
                         issue_s(t, kslot);
                         commit(B_SFULL + t);
+                        PROF_STAMP(leader && t == 0 && j == 64, 28);
                     }
                     PROF_LAP(5 + 5 * t);
                 }
@@ -314,6 +321,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         PROF_DECL(6);
         for (int j = 0; j < n; ++j) {
             if (!(ok = mbar_wait(bar(B_SFULL + t), j & 1, abort_flag))) break;
+            PROF_STAMP(t == 0 && r == 0 && j == 65, 29);
             PROF_LAP(0);
             tc_fence_after_sync();
             uint32_t sr[BN];
@@ -324,85 +332,23 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 
             const int kv0 = j * BN;
             const bool need_mask = (kv0 + BN > prm.Sk) || (prm.causal && kv0 + BN - 1 > q0 + t * BM);
-            float mx;
-            if (need_mask) {  // diagonal or ragged tile: rare, kept out of the hot path
-                const int lim = (prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1;  // last visible key
-                mx = -INFINITY;
-#pragma unroll
-                for (int e = 0; e < BN; ++e) {
-                    const float s = (kv0 + e <= lim) ? __uint_as_float(sr[e]) : -INFINITY;
-                    sr[e] = __float_as_uint(s);
-                    mx = fmaxf(mx, s);
-                }
-            } else {
-                float mxs[8];   // eight independent chains keep the max off the latency-bound path
+            bool done = false;
+
+            if (j > 0 && !need_mask) {
+                // ---- fast path: exponentials against the reference maximum of the previous tiles,
+                // the row maximum of this tile computed on the side.  Valid when no row of the warp
+                // has grown by more than 2^8; otherwise everything is redone by the general path.
+                const float mc = m * c;
+                const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
+#if ATTN_SUM_MODE == 0
+                uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // 8 partial row sums
+#else
+                float accs[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#endif
+                float mxs[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) mxs[i] = fmaxf(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
-#pragma unroll
-                for (int e = 16; e < BN; e += 16)
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-#if ATTN_MAX3
-                        mxs[i] = max3(mxs[i], __uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1]));
-#else
-                        mxs[i] = fmaxf(mxs[i], fmaxf(__uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1])));
-#endif
-                    }
-                mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])), fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
-            }
-#ifdef ATTN_TC_PROFILE
-            if (mx == 12345.678f) prm.prof[0] = 1;   // keeps the max in front of the lap
-#endif
-            PROF_LAP(5);
-            // advance the reference maximum only when the true one ran ahead by more than 2^8
-            float alpha = 1.f;
-            if (j == 0) {
-                m = (mx == -INFINITY) ? 0.f : mx;
-            } else if ((mx - m) * c > 8.f) {
-                alpha = ex2_approx((m - mx) * c);
-                m = mx;
-            }
-            // rare: rescale the running O (its last update finished before S_j was produced)
-            if (__any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll
-                for (int ch = 0; ch < D / 32; ++ch) {
-                    uint32_t orr[32];
-                    tmem_ld_32x32b_x32(tO + ch * 32, orr);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) orr[e] = __float_as_uint(__uint_as_float(orr[e]) * alpha);
-                    tmem_st_32x32b_x32(tO + ch * 32, orr);
-                }
-            }
-            const float mc = m * c;
-            PROF_LAP(2);
-            float rs;
-            if (need_mask) {
-                rs = 0.f;
-#pragma unroll
-                for (int ch = 0; ch < BN / 32; ++ch) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const float s0 = __uint_as_float(sr[ch * 32 + e]), s1 = __uint_as_float(sr[ch * 32 + e + 1]);
-                        // masked entries are -inf; keep them 0 also for a zero scale (-inf * 0 = NaN)
-                        const float p0 = (s0 == -INFINITY) ? 0.f : ex2_approx(fmaf(s0, c, -mc));
-                        const float p1 = (s1 == -INFINITY) ? 0.f : ex2_approx(fmaf(s1, c, -mc));
-                        rs += p0 + p1;
-                        pk[e / 2] = pack2<DTYPE>(p0, p1);
-                    }
-                    tmem_st_32x32b_x16(tS + ch * 16, pk);   // P overwrites the S columns already consumed
-                    if (ch == BN / 32 - 2) {                // first three quarters of P are in place
-                        tmem_st_wait();
-                        tc_fence_before_sync();
-                        mbar_arrive(bar(B_PFULL + t));
-                    }
-                }
-            } else {
-                const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
-                uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // 8 partial row sums
-#pragma unroll
-                for (int ch = 0; ch < BN / 32; ++ch) {
+                auto exp_chunk = [&](int ch) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
@@ -416,7 +362,93 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                             p0 = ex2_approx(x0);
                             p1 = ex2_approx(x1);
                         }
+#if ATTN_SUM_MODE == 0
                         acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(p0, p1));
+#else
+                        accs[e & 7] += p0;
+                        accs[(e & 7) + 1] += p1;
+#endif
+                        pk[e / 2] = pack2<DTYPE>(p0, p1);
+                    }
+                    tmem_st_32x32b_x16(tS + ch * 16, pk);   // P overwrites the S columns already in registers
+                };
+#pragma unroll
+                for (int ch = 0; ch < BN / 32 - 1; ++ch) {
+                    exp_chunk(ch);
+                    // a third of the row maximum per chunk, off the critical path of the exponentials
+#pragma unroll
+                    for (int g = 0; g < 7; ++g) {
+                        const int e = 16 + (ch * 7 + g) * 16;
+                        if (e < BN) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                mxs[i] = max3(mxs[i], __uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1]));
+                        }
+                    }
+                }
+                const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                       fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+                if (!__any_sync(0xffffffffu, (mx - m) * c > 8.f)) {
+                    tmem_st_wait();
+                    tc_fence_before_sync();
+                    mbar_arrive(bar(B_PFULL + t));          // first three quarters of P are in place
+                    PROF_LAP(2);
+                    exp_chunk(BN / 32 - 1);
+#if ATTN_SUM_MODE == 0
+                    float a0, a1, a2, a3;
+                    unpack_f32x2(add_f32x2(acc[0], acc[1]), a0, a1);
+                    unpack_f32x2(add_f32x2(acc[2], acc[3]), a2, a3);
+                    l += (a0 + a1) + (a2 + a3);
+#else
+                    l += ((accs[0] + accs[1]) + (accs[2] + accs[3])) + ((accs[4] + accs[5]) + (accs[6] + accs[7]));
+#endif
+                    done = true;
+                }
+            }
+
+            if (!done) {
+                // ---- general path: first tile, diagonal / ragged tile, or a row maximum that ran ahead
+                const int lim = !need_mask ? 0x7fffffff
+                                           : ((prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1);  // last visible key
+                float mx = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < BN; ++e) {
+                    const float sv = (kv0 + e <= lim) ? __uint_as_float(sr[e]) : -INFINITY;
+                    sr[e] = __float_as_uint(sv);
+                    mx = fmaxf(mx, sv);
+                }
+                // advance the reference maximum only when the true one ran ahead by more than 2^8
+                float alpha = 1.f;
+                if (j == 0) {
+                    m = (mx == -INFINITY) ? 0.f : mx;
+                } else if ((mx - m) * c > 8.f) {
+                    alpha = ex2_approx((m - mx) * c);
+                    m = mx;
+                }
+                // rescale the running O (its last update finished before S_j was produced)
+                if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        uint32_t orr[32];
+                        tmem_ld_32x32b_x32(tO + ch * 32, orr);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) orr[e] = __float_as_uint(__uint_as_float(orr[e]) * alpha);
+                        tmem_st_32x32b_x32(tO + ch * 32, orr);
+                    }
+                }
+                const float mc = m * c;
+                float rs = 0.f;
+#pragma unroll
+                for (int ch = 0; ch < BN / 32; ++ch) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const float s0 = __uint_as_float(sr[ch * 32 + e]), s1 = __uint_as_float(sr[ch * 32 + e + 1]);
+                        // masked entries are -inf; keep them 0 also for a zero scale (-inf * 0 = NaN)
+                        const float p0 = (s0 == -INFINITY) ? 0.f : ex2_approx(fmaf(s0, c, -mc));
+                        const float p1 = (s1 == -INFINITY) ? 0.f : ex2_approx(fmaf(s1, c, -mc));
+                        rs += p0 + p1;
                         pk[e / 2] = pack2<DTYPE>(p0, p1);
                     }
                     tmem_st_32x32b_x16(tS + ch * 16, pk);
@@ -426,16 +458,13 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         mbar_arrive(bar(B_PFULL + t));
                     }
                 }
-                float a0, a1, a2, a3;
-                unpack_f32x2(add_f32x2(acc[0], acc[1]), a0, a1);
-                unpack_f32x2(add_f32x2(acc[2], acc[3]), a2, a3);
-                rs = (a0 + a1) + (a2 + a3);
+                l = l * alpha + rs;
             }
-            l = l * alpha + rs;
             PROF_LAP(3);
             tmem_st_wait();
             tc_fence_before_sync();
             mbar_arrive(bar(B_PFULL2 + t));
+            PROF_STAMP(t == 0 && r == 0 && j == 64, 26);
             PROF_LAP(4);
         }
 #ifdef ATTN_TC_PROFILE

@@ -18,7 +18,7 @@
 // unit (POLY_NUM of every POLY_DEN element pairs).
 #ifndef ATTN_POLY_NUM
 #define ATTN_POLY_NUM 1
-#define ATTN_POLY_DEN 4
+#define ATTN_POLY_DEN 8
 #endif
 
 namespace {

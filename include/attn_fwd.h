@@ -54,7 +54,8 @@ typedef enum {
     ATTN_ERR_UNSUPPORTED_ARCH = 7,     /* current device is not compute capability 10.x */
     ATTN_ERR_CUDA = 8,                 /* a CUDA runtime/driver call failed */
     ATTN_ERR_DEVICE_TIMEOUT = 9,       /* a kernel gave up on a bounded on-chip wait */
-    ATTN_ERR_WORKSPACE = 10            /* workspace missing, misaligned or too small */
+    ATTN_ERR_WORKSPACE = 10,           /* workspace missing, misaligned or too small */
+    ATTN_ERR_STATIC_CAPACITY = 11      /* problem does not fit the library's built-in staging buffer */
 } attn_status_t;
 
 /*
@@ -97,6 +98,47 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
 
 /* Bytes of device workspace attn_fwd_host needs for this problem (0 for an invalid shape). */
 size_t attn_fwd_host_workspace_bytes(int B, int H, int Sq, int Sk, int D);
+
+/*
+ * attn_fwd_host_static -- attn_fwd_host for callers that cannot allocate device memory.
+ * (The paper has no counterpart to this entry point; it is a convenience of this library.)
+ *
+ * Who needs it: code that holds host buffers but may not call cudaMalloc or any allocating
+ * routine at the point of the call -- for example a plug-in running inside a host application
+ * that owns the device memory budget, a real-time loop where an allocation (an implicit
+ * device-wide synchronisation) is not acceptable, or a process whose memory pool is already
+ * committed.  attn_fwd_host asks such a caller for a device workspace it has no means to
+ * provide; this variant stages Q, K, V, O and LSE in a buffer that is part of the library image
+ * itself: a file-scope `static __device__` array of ATTN_STATIC_WORKSPACE_BYTES (16 MiB), which
+ * every GPU that loads the library holds from module load until the process exits.
+ *
+ * Arguments, layouts, conventions and asynchrony are those of attn_fwd_host without the
+ * workspace pair; q, k, v, o, lse are HOST pointers and the results are valid once `stream`
+ * has been synchronised.  The call allocates nothing: no cudaMalloc, cudaFree or allocating
+ * library routine is reached on this path.
+ *
+ * Limit: attn_fwd_host_workspace_bytes(B,H,Sq,Sk,D) must not exceed
+ * attn_fwd_host_static_capacity(); larger problems are refused with ATTN_ERR_STATIC_CAPACITY
+ * before anything is enqueued.  Other errors: as attn_fwd_host.
+ *
+ * Set-up: the first call on each device looks up the device address of the built-in buffer
+ * (once per device, with that device current).  Make that first call outside any stream
+ * capture; later calls on the same device do no set-up.
+ *
+ * Sharing: there is ONE buffer per device and every call uses it from offset 0.  It keeps the
+ * previous call's bytes; nothing in it has to start at zero, because each call overwrites every
+ * region before reading it (Q, K, V by the host-to-device copies, O and LSE by the kernel).
+ * Two calls whose work overlaps on the GPU (different streams, or several host threads)
+ * race on the buffer and corrupt each other's results: issue the calls on one stream, or
+ * otherwise order them.
+ */
+#define ATTN_STATIC_WORKSPACE_BYTES (16u << 20)
+int attn_fwd_host_static(const void* q_host, const void* k_host, const void* v_host, void* o_host,
+                         float* lse_host, int B, int H, int Sq, int Sk, int D, float scale,
+                         int causal, int dtype, void* stream);
+
+/* Capacity in bytes of the built-in staging buffer used by attn_fwd_host_static. */
+size_t attn_fwd_host_static_capacity(void);
 
 /* ATTN_OK if attn_fwd supports (D, dtype, causal) on the current device, otherwise the
  * status attn_fwd would return.  Launches nothing. */

@@ -20,11 +20,12 @@ STATUS_NAMES = {
     0: "ATTN_OK", 1: "ATTN_ERR_NULL_POINTER", 2: "ATTN_ERR_BAD_SHAPE",
     3: "ATTN_ERR_UNSUPPORTED_HEAD_DIM", 4: "ATTN_ERR_UNSUPPORTED_DTYPE", 5: "ATTN_ERR_MISALIGNED",
     6: "ATTN_ERR_BAD_SCALE", 7: "ATTN_ERR_UNSUPPORTED_ARCH", 8: "ATTN_ERR_CUDA",
-    9: "ATTN_ERR_DEVICE_TIMEOUT", 10: "ATTN_ERR_WORKSPACE",
+    9: "ATTN_ERR_DEVICE_TIMEOUT", 10: "ATTN_ERR_WORKSPACE", 11: "ATTN_ERR_STATIC_CAPACITY",
 }
 
 # every symbol include/attn_fwd.h declares
 EXPORTS = ["attn_fwd", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
+           "attn_fwd_host_static", "attn_fwd_host_static_capacity",
            "attn_query_support", "attn_last_device_status", "attn_status_string"]
 
 _lib = None
@@ -60,6 +61,10 @@ def load() -> ctypes.CDLL:
     lib.attn_fwd_host.argtypes = sig[:-1] + [vp, ctypes.c_size_t, vp]
     lib.attn_fwd_host_workspace_bytes.restype = ctypes.c_size_t
     lib.attn_fwd_host_workspace_bytes.argtypes = [i] * 5
+    lib.attn_fwd_host_static.restype = i
+    lib.attn_fwd_host_static.argtypes = sig
+    lib.attn_fwd_host_static_capacity.restype = ctypes.c_size_t
+    lib.attn_fwd_host_static_capacity.argtypes = []
     lib.attn_query_support.restype = i
     lib.attn_query_support.argtypes = [i, i, i]
     lib.attn_last_device_status.restype = i
@@ -146,6 +151,30 @@ def attn_fwd_host(q, k, v, scale: float, causal: bool, out, lse, workspace, stre
                                   _stream_ptr(stream))
     if rc != 0:
         raise AttnError(rc, "attn_fwd_host")
+    return out, lse
+
+
+def attn_fwd_host_static_capacity() -> int:
+    return int(load().attn_fwd_host_static_capacity())
+
+
+def attn_fwd_host_static(q, k, v, scale: float, causal: bool, out, lse, stream=None, device=None):
+    """attn_fwd_host for callers that cannot allocate device memory: Q, K, V, O and LSE are staged in
+    the 16 MiB buffer built into the library image, so no workspace is passed and nothing is
+    allocated.  Host tensors in, host tensors out; valid after the stream has been synchronised.
+    Problems that need more staging than attn_fwd_host_static_capacity() raise
+    AttnError(ATTN_ERR_STATIC_CAPACITY).  All calls on a device share the one buffer: keep them on
+    one stream (overlapping calls race).  The first call on a device resolves the buffer's address
+    and should come before any stream capture."""
+    B, H, Sq, Sk, D = _check_qkv(q, k, v)
+    dt = _dtype_code(q)
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        rc = load().attn_fwd_host_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                         lse.data_ptr(), B, H, Sq, Sk, D, float(scale),
+                                         int(bool(causal)), dt, _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_fwd_host_static")
     return out, lse
 
 

@@ -229,6 +229,30 @@ int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, i
 
 size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
+// Built-in staging buffer of attn_fwd_host_static.  In host code this name is only a stand-in
+// for the symbol: the device address is looked up once per device (below) and that pointer, not
+// the name, is what the copies and the kernel are given.
+static __device__ __align__(256) unsigned char g_static_workspace[ATTN_STATIC_WORKSPACE_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_workspace_addr[kMaxDevices] = {};
+
+// Device address of the built-in buffer on the current device; resolved on first use per device.
+int static_workspace_ptr(void** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ATTN_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return ATTN_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_workspace_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return ATTN_ERR_CUDA;
+        g_static_workspace_addr[dev] = p;
+    }
+    *out = g_static_workspace_addr[dev];
+    return ATTN_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -280,6 +304,24 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
     return ATTN_OK;
 }
 
+size_t attn_fwd_host_static_capacity(void) { return ATTN_STATIC_WORKSPACE_BYTES; }
+
+int attn_fwd_host_static(const void* q_host, const void* k_host, const void* v_host, void* o_host, float* lse_host,
+                         int B, int H, int Sq, int Sk, int D, float scale, int causal, int dtype, void* stream) {
+    int rc = validate(q_host, k_host, v_host, o_host, lse_host, B, H, Sq, Sk, D, scale, dtype, false);
+    if (rc != ATTN_OK) return rc;
+    if (static_cast<size_t>(B) * H * Sq == 0) return ATTN_OK;
+    const size_t need = attn_fwd_host_workspace_bytes(B, H, Sq, Sk, D);
+    if (need > ATTN_STATIC_WORKSPACE_BYTES) return ATTN_ERR_STATIC_CAPACITY;
+    rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+    void* ws = nullptr;
+    rc = static_workspace_ptr(&ws);
+    if (rc != ATTN_OK) return rc;
+    return attn_fwd_host(q_host, k_host, v_host, o_host, lse_host, B, H, Sq, Sk, D, scale, causal, dtype, ws,
+                         ATTN_STATIC_WORKSPACE_BYTES, stream);
+}
+
 int attn_query_support(int D, int dtype, int causal) {
     (void)causal;
     if (D != 64 && D != 128 && D != 256) return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
@@ -315,6 +357,7 @@ const char* attn_status_string(int status) {
         case ATTN_ERR_CUDA: return "ATTN_ERR_CUDA";
         case ATTN_ERR_DEVICE_TIMEOUT: return "ATTN_ERR_DEVICE_TIMEOUT";
         case ATTN_ERR_WORKSPACE: return "ATTN_ERR_WORKSPACE";
+        case ATTN_ERR_STATIC_CAPACITY: return "ATTN_ERR_STATIC_CAPACITY";
         default: return "ATTN_ERR_UNKNOWN";
     }
 }

@@ -76,6 +76,17 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, i
              int Sk, int D, float scale, int causal, int dtype, void* stream);
 
 /*
+ * attn_fwd_gqa -- grouped-query / multi-query attention (the GQA and MQA variants of Section 2.2
+ * and Table 1): K and V carry Hkv heads, [B, Hkv, Sk, D], and query head h reads key/value head
+ * h / (H / Hkv).  H must be a multiple of Hkv (Hkv == H is attn_fwd, Hkv == 1 is MQA); otherwise
+ * ATTN_ERR_BAD_SHAPE.  Everything else -- layouts of Q, O, LSE, mask, scale, errors, asynchrony --
+ * is as for attn_fwd.  The query heads of one K/V head are scheduled next to each other so that
+ * their K/V tiles are shared through L2.
+ */
+int attn_fwd_gqa(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv,
+                 int Sq, int Sk, int D, float scale, int causal, int dtype, void* stream);
+
+/*
  * attn_fwd_simt -- same operator, same arguments, same conventions, computed by a plain
  * CUDA-core kernel (one warp per query row, fp32 arithmetic, online softmax).  It is one to
  * two orders of magnitude slower than attn_fwd and exists as an on-device cross-check that

@@ -163,6 +163,38 @@ int attn_oracle_f64(const double *q, const double *k, const double *v, double *o
     return failed ? -1 : 0;
 }
 
+/* Grouped-query attention (the GQA / MQA variants named in Section 2.2): K and V have Hkv heads,
+ * [B,Hkv,Sk,D], and query head h reads key/value head h / (H / Hkv).  Same row function. */
+int attn_oracle_gqa_f64(const double *q, const double *k, const double *v, double *o, double *lse,
+                        int B, int H, int Hkv, int Sq, int Sk, int D, double scale, int causal)
+{
+    int64_t rows = (int64_t)B * H * Sq;
+    int failed = 0;
+    if (Hkv <= 0 || H % Hkv != 0)
+        return -2;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(Sk > 0 ? Sk : 1));
+        if (!s) {
+#pragma omp atomic write
+            failed = 1;
+        }
+        int64_t r;
+#pragma omp for schedule(dynamic, 16)
+        for (r = 0; r < rows; ++r) {
+            if (!s)
+                continue;
+            int64_t bh = r / Sq, i = r % Sq;
+            int64_t b = bh / H, h = bh % H;
+            int64_t kvh = b * Hkv + h / (H / Hkv);
+            attn_row(q + r * D, k + kvh * Sk * D, v + kvh * Sk * D, s, o + r * D, lse + r, NULL,
+                     visible_keys(i, Sk, causal), D, scale);
+        }
+        free(s);
+    }
+    return failed ? -1 : 0;
+}
+
 /* Same arithmetic for a chosen subset of rows, reading the 16-bit inputs directly
  * (widened exactly) so that full-size problems need no fp64 copy of Q, K, V.
  * rows[n_rows]: flat row indices r = (b*H + h)*Sq + i, in ascending order.

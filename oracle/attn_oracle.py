@@ -51,6 +51,8 @@ def _load():
         lib.attn_oracle_rows_16.argtypes = [u16p, u16p, u16p, ctypes.c_int, i64p, ctypes.c_int64,
                                             dp, dp] + [ctypes.c_int] * 5 + [ctypes.c_double,
                                                                             ctypes.c_int]
+        lib.attn_oracle_gqa_f64.restype = ctypes.c_int
+        lib.attn_oracle_gqa_f64.argtypes = [dp, dp, dp, dp, dp] + [ctypes.c_int] * 6 + [ctypes.c_double, ctypes.c_int]
         lib.oracle_widen.restype = None
         lib.oracle_widen.argtypes = [u16p, dp, ctypes.c_int64, ctypes.c_int]
         lib.oracle_num_threads.restype = ctypes.c_int
@@ -98,6 +100,25 @@ def attention(q, k, v, scale: float, causal: bool, return_rowsum: bool = False):
     if rc != 0:
         raise MemoryError("oracle scratch allocation failed")
     return (o, lse, rs) if return_rowsum else (o, lse)
+
+
+def attention_gqa(q, k, v, scale: float, causal: bool):
+    """Grouped-query attention for float64 arrays: q [B,H,Sq,D]; k, v [B,Hkv,Sk,D], H % Hkv == 0."""
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    k = np.ascontiguousarray(k, dtype=np.float64)
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    B, H, Sq, D = q.shape
+    Hkv, Sk = k.shape[1], k.shape[2]
+    assert k.shape == (B, Hkv, Sk, D) and v.shape == (B, Hkv, Sk, D)
+    o = np.empty((B, H, Sq, D), dtype=np.float64)
+    lse = np.empty((B, H, Sq), dtype=np.float64)
+    rc = _load().attn_oracle_gqa_f64(_dptr(q), _dptr(k), _dptr(v), _dptr(o), _dptr(lse), B, H, Hkv, Sq, Sk, D,
+                                     float(scale), int(bool(causal)))
+    if rc == -2:
+        raise ValueError("H must be a multiple of Hkv")
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return o, lse
 
 
 def attention_rows_16(q_bits, k_bits, v_bits, dtype: int, rows, scale: float, causal: bool):

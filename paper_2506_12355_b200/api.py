@@ -24,7 +24,7 @@ STATUS_NAMES = {
 }
 
 # every symbol include/attn_fwd.h declares
-EXPORTS = ["attn_fwd", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
+EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
            "attn_fwd_host_static", "attn_fwd_host_static_capacity",
            "attn_query_support", "attn_last_device_status", "attn_status_string"]
 
@@ -55,6 +55,8 @@ def load() -> ctypes.CDLL:
     sig = [vp, vp, vp, vp, vp, i, i, i, i, i, f, i, i, vp]
     lib.attn_fwd.restype = i
     lib.attn_fwd.argtypes = sig
+    lib.attn_fwd_gqa.restype = i
+    lib.attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, vp]
     lib.attn_fwd_simt.restype = i
     lib.attn_fwd_simt.argtypes = sig
     lib.attn_fwd_host.restype = i
@@ -127,6 +129,31 @@ def attn_fwd(q, k, v, scale: float, causal: bool = False, out=None, lse=None, st
     Enqueues on `stream` (default: torch's current stream) and returns without synchronising.
     """
     return _call_device("attn_fwd", q, k, v, scale, causal, out, lse, stream)
+
+
+def attn_fwd_gqa(q, k, v, scale: float, causal: bool = False, out=None, lse=None, stream=None):
+    """Grouped-query / multi-query attention: q [B,H,Sq,D], k, v [B,Hkv,Sk,D] with H % Hkv == 0."""
+    if q.dim() != 4 or k.dim() != 4 or tuple(v.shape) != tuple(k.shape):
+        raise ValueError("q must be [B,H,Sq,D]; k, v must be [B,Hkv,Sk,D]")
+    B, H, Sq, D = q.shape
+    Hkv, Sk = k.shape[1], k.shape[2]
+    if k.shape[0] != B or k.shape[3] != D:
+        raise ValueError("k, v must match q's B and D")
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+        raise ValueError("q, k, v must be contiguous")
+    if not (q.is_cuda and k.is_cuda and v.is_cuda) or not (q.dtype == k.dtype == v.dtype):
+        raise ValueError("q, k, v must be CUDA tensors of one dtype")
+    dt = _dtype_code(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(q.device):
+        rc = load().attn_fwd_gqa(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                 B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)), dt, _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_fwd_gqa")
+    return out, lse
 
 
 def attn_fwd_simt(q, k, v, scale: float, causal: bool = False, out=None, lse=None, stream=None):

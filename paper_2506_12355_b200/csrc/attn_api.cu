@@ -71,11 +71,12 @@ int check_arch() {
 constexpr int kMaxSeq = 2147483647 - 256;
 
 // Validation shared by every entry point; no CUDA call happens here.
-int validate(const void* q, const void* k, const void* v, const void* o, const void* lse, int B, int H, int Sq,
+int validate(const void* q, const void* k, const void* v, const void* o, const void* lse, int B, int H, int Hkv, int Sq,
              int Sk, int D, float scale, int dtype, bool device_pointers) {
-    if (B < 0 || H < 0 || Sq < 0 || Sk < 0 || D < 0) return ATTN_ERR_BAD_SHAPE;
+    if (B < 0 || H < 0 || Hkv < 0 || Sq < 0 || Sk < 0 || D < 0) return ATTN_ERR_BAD_SHAPE;
+    if (H > 0 && (Hkv == 0 || H % Hkv != 0)) return ATTN_ERR_BAD_SHAPE;
     // empty tensors may come with NULL pointers (an allocator returns none for zero bytes)
-    const bool no_rows = static_cast<int64_t>(B) * H * Sq == 0, no_keys = static_cast<int64_t>(B) * H * Sk == 0;
+    const bool no_rows = static_cast<int64_t>(B) * H * Sq == 0, no_keys = static_cast<int64_t>(B) * Hkv * Sk == 0;
     if (!no_rows && (!q || !o || !lse)) return ATTN_ERR_NULL_POINTER;
     if (!no_rows && !no_keys && (!k || !v)) return ATTN_ERR_NULL_POINTER;
     if (Sq > kMaxSeq || Sk > kMaxSeq) return ATTN_ERR_BAD_SHAPE;
@@ -104,7 +105,7 @@ int fill_empty(void* o, float* lse, int64_t n_o, int64_t n_lse, cudaStream_t st)
 }
 
 template <int D, int DTYPE>
-int launch_tc_basic(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
+int launch_tc_basic(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
                     float scale, int causal, cudaStream_t st) {
     using C = attn_tc::BasicCfg<D>;
     auto kern = attn_tc::attn_fwd_tc_basic_kernel<D, DTYPE>;
@@ -116,8 +117,8 @@ int launch_tc_basic(const void* q, const void* k, const void* v, void* o, float*
     if (attr_err != cudaSuccess) return ATTN_ERR_CUDA;
     const int64_t BH = static_cast<int64_t>(B) * H;
     CUtensorMap mq, mk, mv;
-    if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, BH, Sk, D, C::BN) ||
-        !make_map(&mv, v, DTYPE, BH, Sk, D, C::BN))
+    if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) ||
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN))
         return ATTN_ERR_CUDA;
     attn_tc::Params prm;
     prm.o = o;
@@ -129,6 +130,8 @@ int launch_tc_basic(const void* q, const void* k, const void* v, void* o, float*
     prm.causal = causal ? 1 : 0;
     prm.status = device_status_ptr();
     if (!prm.status) return ATTN_ERR_CUDA;
+    prm.H = H;
+    prm.Hkv = Hkv;
     const int64_t q_tiles = (static_cast<int64_t>(Sq) + C::BM - 1) / C::BM;
     // grid.y is limited to 65535: fold the heads into grid.x when there are more
     if (BH > 65535) return ATTN_ERR_BAD_SHAPE;
@@ -143,7 +146,7 @@ long long* g_prof_buffer = nullptr;  // development builds: per-CTA cycle sums, 
 
 // Pipelined, warp-specialised kernel (head dims 64 and 128): one CTA per pair of 128-row Q tiles.
 template <int D, int DTYPE>
-int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
+int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
                    float scale, int causal, cudaStream_t st) {
     using C = attn_tc::PipeCfg<D>;
     auto kern = attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE, ATTN_POLY_NUM, ATTN_POLY_DEN>;
@@ -157,8 +160,8 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     const int64_t n_pairs = (static_cast<int64_t>(Sq) + 2 * C::BM - 1) / (2 * C::BM);
     if (n_pairs * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
     CUtensorMap mq, mk, mv;
-    if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, BH, Sk, D, C::BN) ||
-        !make_map(&mv, v, DTYPE, BH, Sk, D, C::BN))
+    if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) ||
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN))
         return ATTN_ERR_CUDA;
     attn_tc::PipeParams prm;
     prm.o = o;
@@ -170,12 +173,15 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     prm.causal = causal ? 1 : 0;
     prm.status = device_status_ptr();
     if (!prm.status) return ATTN_ERR_CUDA;
+    prm.H = H;
+    prm.Hkv = Hkv;
     prm.n_pairs = static_cast<int>(n_pairs);
     prm.BH = static_cast<int>(BH);
     // walk together as many heads as keep their K and V (2 * Sk * D * 2 bytes each) inside ~48 MB of L2
     const int64_t kv_bytes_per_head = 4LL * Sk * D;
     int64_t hpg = (48LL << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
     if (hpg < 1) hpg = 1;
+    hpg *= H / Hkv;  // the query heads of one K/V head share its footprint
     if (hpg > BH) hpg = BH;
     prm.heads_per_group = static_cast<int>(hpg);
 #ifdef ATTN_TC_PROFILE
@@ -186,23 +192,23 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
 }
 
 template <int D, int DTYPE>
-int launch_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
+int launch_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
                 float scale, int causal, cudaStream_t st) {
     const int64_t BH = static_cast<int64_t>(B) * H;
     if (BH > 65535) return ATTN_ERR_BAD_SHAPE;
     dim3 grid(static_cast<unsigned>((static_cast<int64_t>(Sq) + attn_simt::kWarpsPerBlock - 1) / attn_simt::kWarpsPerBlock),
               static_cast<unsigned>(BH));
     attn_simt::attn_fwd_simt_kernel<D, DTYPE><<<grid, attn_simt::kWarpsPerBlock * 32, 0, st>>>(q, k, v, o, lse, Sq, Sk,
-                                                                                              scale, causal ? 1 : 0);
+                                                                                              scale, causal ? 1 : 0, H, Hkv);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
 enum class Impl { TensorCore, TensorCoreBasic, Simt };
 
 template <Impl IMPL>
-int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk, int D,
+int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk, int D,
              float scale, int causal, int dtype, void* stream) {
-    int rc = validate(q, k, v, o, lse, B, H, Sq, Sk, D, scale, dtype, true);
+    int rc = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, dtype, true);
     if (rc != ATTN_OK) return rc;
     if (static_cast<int64_t>(B) * H * Sq == 0) return ATTN_OK;
     rc = check_arch();
@@ -212,10 +218,10 @@ int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, i
         return fill_empty(o, lse, static_cast<int64_t>(B) * H * Sq * D, static_cast<int64_t>(B) * H * Sq, st);
 #define ATTN_CASE(DD, TT)                                                                              \
     if (D == DD && dtype == TT) {                                                                      \
-        if (IMPL == Impl::Simt) return launch_simt<DD, TT>(q, k, v, o, lse, B, H, Sq, Sk, scale, causal, st); \
+        if (IMPL == Impl::Simt) return launch_simt<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
         if (IMPL == Impl::TensorCoreBasic || DD == 256)                                                \
-            return launch_tc_basic<DD, TT>(q, k, v, o, lse, B, H, Sq, Sk, scale, causal, st);          \
-        return launch_tc_pipe<(DD == 256 ? 128 : DD), TT>(q, k, v, o, lse, B, H, Sq, Sk, scale, causal, st); \
+            return launch_tc_basic<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st);          \
+        return launch_tc_pipe<(DD == 256 ? 128 : DD), TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
     }
     ATTN_CASE(64, 0)
     ATTN_CASE(64, 1)
@@ -259,12 +265,17 @@ extern "C" {
 
 int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk, int D,
              float scale, int causal, int dtype, void* stream) {
-    return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, Sq, Sk, D, scale, causal, dtype, stream);
+    return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, H, Sq, Sk, D, scale, causal, dtype, stream);
+}
+
+int attn_fwd_gqa(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
+                 int D, float scale, int causal, int dtype, void* stream) {
+    return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, causal, dtype, stream);
 }
 
 int attn_fwd_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
                   int D, float scale, int causal, int dtype, void* stream) {
-    return dispatch<Impl::Simt>(q, k, v, o, lse, B, H, Sq, Sk, D, scale, causal, dtype, stream);
+    return dispatch<Impl::Simt>(q, k, v, o, lse, B, H, H, Sq, Sk, D, scale, causal, dtype, stream);
 }
 
 size_t attn_fwd_host_workspace_bytes(int B, int H, int Sq, int Sk, int D) {
@@ -277,7 +288,7 @@ size_t attn_fwd_host_workspace_bytes(int B, int H, int Sq, int Sk, int D) {
 int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host, float* lse_host, int B,
                   int H, int Sq, int Sk, int D, float scale, int causal, int dtype, void* workspace,
                   size_t workspace_bytes, void* stream) {
-    int rc = validate(q_host, k_host, v_host, o_host, lse_host, B, H, Sq, Sk, D, scale, dtype, false);
+    int rc = validate(q_host, k_host, v_host, o_host, lse_host, B, H, H, Sq, Sk, D, scale, dtype, false);
     if (rc != ATTN_OK) return rc;
     const size_t bh = static_cast<size_t>(B) * H;
     if (bh * Sq == 0) return ATTN_OK;
@@ -308,7 +319,7 @@ size_t attn_fwd_host_static_capacity(void) { return ATTN_STATIC_WORKSPACE_BYTES;
 
 int attn_fwd_host_static(const void* q_host, const void* k_host, const void* v_host, void* o_host, float* lse_host,
                          int B, int H, int Sq, int Sk, int D, float scale, int causal, int dtype, void* stream) {
-    int rc = validate(q_host, k_host, v_host, o_host, lse_host, B, H, Sq, Sk, D, scale, dtype, false);
+    int rc = validate(q_host, k_host, v_host, o_host, lse_host, B, H, H, Sq, Sk, D, scale, dtype, false);
     if (rc != ATTN_OK) return rc;
     if (static_cast<size_t>(B) * H * Sq == 0) return ATTN_OK;
     const size_t need = attn_fwd_host_workspace_bytes(B, H, Sq, Sk, D);

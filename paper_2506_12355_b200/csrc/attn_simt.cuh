@@ -31,7 +31,7 @@ template <int D, int DTYPE>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 attn_fwd_simt_kernel(const void* __restrict__ q, const void* __restrict__ k,
                      const void* __restrict__ v, void* __restrict__ o, float* __restrict__ lse,
-                     int Sq, int Sk, float scale, int causal) {
+                     int Sq, int Sk, float scale, int causal, int H, int Hkv) {
     constexpr int CPL = D / 32;  // output columns per lane
     __shared__ float qs[kWarpsPerBlock][D];
 
@@ -41,7 +41,8 @@ attn_fwd_simt_kernel(const void* __restrict__ q, const void* __restrict__ k,
     if (i >= Sq) return;
 
     const int64_t qrow = (bh * Sq + i) * D;
-    const int64_t kvbase = bh * static_cast<int64_t>(Sk) * D;
+    const int64_t kv_bh = (bh / H) * Hkv + (bh % H) / (H / Hkv);  // grouped-query attention
+    const int64_t kvbase = kv_bh * static_cast<int64_t>(Sk) * D;
     for (int d = lane; d < D; d += 32) qs[warp][d] = load16<DTYPE>(q, qrow + d);
     __syncwarp();
 

@@ -43,6 +43,7 @@ struct Params {
     float scale_log2;   // scale * log2(e)
     int causal;
     int* status;        // device status word
+    int H, Hkv;         // query heads and key/value heads per batch element (H % Hkv == 0)
 };
 
 template <int D, int DTYPE>
@@ -61,6 +62,7 @@ attn_fwd_tc_basic_kernel(const __grid_constant__ CUtensorMap tmQ,
     const int tid = threadIdx.x, warp = tid >> 5;
     const int q0 = blockIdx.x * BM;
     const int bh = blockIdx.y;
+    const int kv_bh = (bh / prm.H) * prm.Hkv + (bh % prm.H) / (prm.H / prm.Hkv);  // grouped-query attention
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base;
@@ -102,8 +104,8 @@ attn_fwd_tc_basic_kernel(const __grid_constant__ CUtensorMap tmQ,
         const int st = j % C::NSTAGE;
         mbar_arrive_expect_tx(b_kv(st), 2 * C::KV_BYTES);
         for (int bx = 0; bx < NBOX; ++bx) {
-            tma_load_3d(sK(st) + bx * BN * 128, &tmK, b_kv(st), bx * 64, j * BN, bh);
-            tma_load_3d(sV(st) + bx * BN * 128, &tmV, b_kv(st), bx * 64, j * BN, bh);
+            tma_load_3d(sK(st) + bx * BN * 128, &tmK, b_kv(st), bx * 64, j * BN, kv_bh);
+            tma_load_3d(sV(st) + bx * BN * 128, &tmV, b_kv(st), bx * 64, j * BN, kv_bh);
         }
     };
 

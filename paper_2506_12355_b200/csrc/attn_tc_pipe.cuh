@@ -50,6 +50,7 @@ struct PipeParams {
     int n_pairs;          // 256-row Q tile pairs per head
     int BH;               // batch * heads
     int heads_per_group;  // heads whose K/V are walked together (L2 residency)
+    int H, Hkv;           // query heads and key/value heads per batch element (H % Hkv == 0)
 #ifdef ATTN_TC_PROFILE
     long long* prof;      // [grid][32] cycle sums per phase (development builds only)
 #endif
@@ -117,6 +118,8 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         pair = prm.causal ? prm.n_pairs - 1 - pr : pr;  // causal: longest rows first
     }
     const int q0 = pair * 2 * BM;
+    // grouped-query attention: H / Hkv consecutive query heads read the same K/V head
+    const int kv_bh = (bh / prm.H) * prm.Hkv + (bh % prm.H) / (prm.H / prm.Hkv);
 
     // K/V tiles each Q tile needs
     int n_kv[2];
@@ -190,7 +193,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     mbar_arrive_expect_tx(bar(B_KVFULL + slot), C::KV_BYTES);
 #pragma unroll
                     for (int bx = 0; bx < NBOX; ++bx)
-                        tma_load_3d(sKV(slot) + bx * BN * 128, map, bar(B_KVFULL + slot), bx * 64, j * BN, bh);
+                        tma_load_3d(sKV(slot) + bx * BN * 128, map, bar(B_KVFULL + slot), bx * 64, j * BN, kv_bh);
                 }
                 return true;
             };

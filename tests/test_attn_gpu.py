@@ -230,3 +230,31 @@ def test_tensor_core_kernel_agrees_with_cross_check_kernel_everywhere(name):
     o2, l2 = run_gpu(api.attn_fwd_simt, q, k, v, cfg.scale, cfg.causal)
     assert float((o1.float() - o2.float()).abs().max()) <= 2 * O_TOL[cfg.dtype]
     assert float((l1 - l2).abs().max()) <= 2 * LSE_TOL
+
+
+# ------------------------------------------------------------------ grouped-query / multi-query attention
+
+@pytest.mark.parametrize("D,dtype,causal,H,Hkv", [(128, 1, True, 8, 2), (64, 0, False, 6, 1), (256, 0, True, 4, 2),
+                                                  (128, 0, False, 4, 4)])
+def test_gqa_against_oracle(D, dtype, causal, H, Hkv):
+    B, Sq, Sk = 2, 300, 421
+    q = inputs.randn16((B, H, Sq, D), 500, dtype)
+    k = inputs.randn16((B, Hkv, Sk, D), 501, dtype)
+    v = inputs.randn16((B, Hkv, Sk, D), 502, dtype)
+    dev = torch.device("cuda:0")
+    obuf, o = guarded((B, H, Sq, D), q.dtype, dev)
+    lbuf, lse = guarded((B, H, Sq), torch.float32, dev)
+    scale = 1.0 / math.sqrt(D)
+    api.attn_fwd_gqa(q.to(dev), k.to(dev), v.to(dev), scale, causal, out=o, lse=lse)
+    assert api.attn_last_device_status() == 0 and guards_intact(obuf) and guards_intact(lbuf)
+    o_ref, lse_ref = orc.attention_gqa(*(orc.widen(inputs.bits(t), dtype) for t in (q, k, v)), scale, causal)
+    assert np.abs(o.cpu().double().numpy() - o_ref).max() <= O_TOL[dtype]
+    assert np.abs(lse.cpu().double().numpy() - lse_ref).max() <= LSE_TOL
+
+
+def test_gqa_rejects_indivisible_heads():
+    q = torch.zeros(1, 5, 128, 64, dtype=torch.float16, device="cuda:0")
+    kv = torch.zeros(1, 2, 128, 64, dtype=torch.float16, device="cuda:0")
+    with pytest.raises(api.AttnError) as err:
+        api.attn_fwd_gqa(q, kv, kv, 0.1, False)
+    assert err.value.status == 2

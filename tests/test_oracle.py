@@ -269,3 +269,26 @@ def test_input_generator_is_seeded_and_rounded():
     assert a.dtype == torch.bfloat16
     w = orc.widen(inputs.bits(a), inputs.DTYPE_BF16)
     np.testing.assert_array_equal(w, a.to(torch.float64).numpy())
+
+
+# ------------------------------------------------------------------ grouped-query attention
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("H,Hkv", [(6, 2), (4, 1), (3, 3)])
+def test_gqa_equals_mha_with_repeated_kv_heads(H, Hkv, causal):
+    # query head h reads K/V head h // (H // Hkv): the same as plain attention on K/V with every
+    # head repeated H // Hkv times (built here with numpy, not with the oracle's index arithmetic)
+    B, Sq, Sk, D = 2, 9, 14, 8
+    q, k, v = rand((B, H, Sq, D), 40), rand((B, Hkv, Sk, D), 41), rand((B, Hkv, Sk, D), 42)
+    o, lse = orc.attention_gqa(q, k, v, 0.3, causal)
+    o_ref, lse_ref = orc.attention(q, np.repeat(k, H // Hkv, axis=1), np.repeat(v, H // Hkv, axis=1), 0.3, causal)
+    np.testing.assert_array_equal(o, o_ref)
+    np.testing.assert_array_equal(lse, lse_ref)
+    to = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v),
+                                                          is_causal=causal, scale=0.3, enable_gqa=True)
+    np.testing.assert_allclose(o, to.numpy(), atol=1e-10)
+
+
+def test_gqa_rejects_indivisible_heads():
+    with pytest.raises(ValueError):
+        orc.attention_gqa(rand((1, 5, 2, 4), 1), rand((1, 2, 2, 4), 2), rand((1, 2, 2, 4), 3), 1.0, False)

@@ -12,6 +12,7 @@
 #include "../../include/attn_fwd.h"
 #include "attn_simt.cuh"
 #include "attn_tc_basic.cuh"
+#include "attn_tc_d256.cuh"
 #include "attn_tc_pipe.cuh"
 
 // Share of the exponentials evaluated by a polynomial on the FMA pipe instead of the special-function
@@ -191,6 +192,50 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
+// Head dim 256: one Q tile per CTA, Q in tensor memory, double-buffered S.
+template <int DTYPE>
+int launch_tc_d256(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
+                   float scale, int causal, cudaStream_t st) {
+    using C = attn_tc::D256Cfg;
+    auto kern = attn_tc::attn_fwd_tc_d256_kernel<DTYPE>;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    });
+    if (attr_err != cudaSuccess) return ATTN_ERR_CUDA;
+    const int64_t BH = static_cast<int64_t>(B) * H;
+    const int64_t n_qtiles = (static_cast<int64_t>(Sq) + C::BM - 1) / C::BM;
+    if (n_qtiles * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
+    CUtensorMap mk, mv;
+    if (!make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, C::D, C::BN) ||
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, C::D, C::BN))
+        return ATTN_ERR_CUDA;
+    attn_tc::D256Params prm;
+    prm.q = q;
+    prm.o = o;
+    prm.lse = lse;
+    prm.Sq = Sq;
+    prm.Sk = Sk;
+    prm.scale = scale;
+    prm.scale_log2 = scale * 1.4426950408889634f;
+    prm.causal = causal ? 1 : 0;
+    prm.status = device_status_ptr();
+    if (!prm.status) return ATTN_ERR_CUDA;
+    prm.n_qtiles = static_cast<int>(n_qtiles);
+    prm.BH = static_cast<int>(BH);
+    prm.H = H;
+    prm.Hkv = Hkv;
+    const int64_t kv_bytes_per_head = 4LL * Sk * C::D;
+    int64_t hpg = (48LL << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
+    if (hpg < 1) hpg = 1;
+    hpg *= H / Hkv;
+    if (hpg > BH) hpg = BH;
+    prm.heads_per_group = static_cast<int>(hpg);
+    kern<<<static_cast<unsigned>(n_qtiles * BH), C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, prm);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
 template <int D, int DTYPE>
 int launch_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
                 float scale, int causal, cudaStream_t st) {
@@ -219,8 +264,9 @@ int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, i
 #define ATTN_CASE(DD, TT)                                                                              \
     if (D == DD && dtype == TT) {                                                                      \
         if (IMPL == Impl::Simt) return launch_simt<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
-        if (IMPL == Impl::TensorCoreBasic || DD == 256)                                                \
-            return launch_tc_basic<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st);          \
+        if (IMPL == Impl::TensorCoreBasic)                                                             \
+            return launch_tc_basic<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st);     \
+        if (DD == 256) return launch_tc_d256<TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
         return launch_tc_pipe<(DD == 256 ? 128 : DD), TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
     }
     ATTN_CASE(64, 0)

@@ -1,0 +1,363 @@
+// Warp-specialised tcgen05 attention forward kernel for head dim 256.
+//
+// With D = 256 the O accumulator of one 128-row Q tile already takes 256 of the 512 tensor-memory
+// columns, so the two-Q-tile scheme of the D <= 128 kernel does not fit.  Instead one CTA owns ONE
+// Q tile and overlaps the tensor core with the softmax through a double-buffered S:
+//
+//   tensor memory:  O [0,256)   Q [256,384)   S buffer 0 [384,448)   S buffer 1 [448,512)
+//   K/V steps of 64 keys:  S_{j+1} = Q K_{j+1}^T is computed while the softmax works on S_j,
+//   then O += P_j V_j; P_j (16-bit) overwrites the first half of its S buffer.
+//
+// Q is the A operand of the first product FROM TENSOR MEMORY (written there once by the softmax
+// threads), so that product reads only the K tile from shared memory: with both operands in
+// shared memory an N = 64 instruction would be bound by shared-memory bandwidth.
+//
+//   warps 0-3  softmax group (one thread per row): Q -> tensor memory, S -> P, rare O rescale, epilogue
+//   warp  4    MMA issuer
+//   warp  5    TMA producer: 64-key K and V tiles through a ring of shared-memory slots
+//
+// Loop structure as in Appendix C, Listings 1-2 of the paper; online softmax with a lazily advanced
+// reference maximum as in the D <= 128 kernel.
+#pragma once
+#include "attn_tc_basic.cuh"
+
+namespace attn_tc {
+
+struct D256Cfg {
+    static constexpr int D = 256;
+    static constexpr int BM = 128;
+    static constexpr int BN = 64;                         // keys per step
+    static constexpr int NBOX = D / 64;                   // 64-column boxes per tile row
+    static constexpr int KV_BYTES = BN * D * 2;           // 32 KB: one K or V tile of 64 keys
+    static constexpr int NSLOT = 6;
+    static constexpr int TILE_BYTES = NSLOT * KV_BYTES;
+    static constexpr int MISC_BYTES = 512;
+    static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
+    static constexpr int THREADS = 192;
+    static constexpr int O_COL = 0, Q_COL = 256, S_COL = 384;  // S buffer b at S_COL + 64 b
+    static constexpr int TMEM_COLS = 512;
+};
+
+struct D256Params {
+    const void* q;
+    void* o;
+    float* lse;
+    int Sq, Sk;
+    float scale, scale_log2;
+    int causal;
+    int* status;
+    int n_qtiles;         // 128-row Q tiles per head
+    int BH;
+    int heads_per_group;
+    int H, Hkv;
+};
+
+template <int DTYPE>
+__global__ void __launch_bounds__(192, 1)
+attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                        const D256Params prm) {
+    using C = D256Cfg;
+    constexpr int D = C::D, BM = C::BM, BN = C::BN, NBOX = C::NBOX, NSLOT = C::NSLOT;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    auto sKV = [&](int slot) { return smem_base + slot * C::KV_BYTES; };
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
+    const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
+    enum { B_QREADY = 0, B_SFULL = 1, B_PFULL = 3, B_ODONE = 5, B_KVFULL = 6, B_KVEMPTY = 6 + NSLOT,
+           B_COUNT = 6 + 2 * NSLOT };
+    auto bar = [&](int i) { return bars_u32 + i * 8; };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 1;
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+
+    // ---- which work item: heads walked in L2-sized groups, causal: longest rows first ----
+    int qt, bh;
+    {
+        const int lin = blockIdx.x;
+        const int full_group = prm.heads_per_group * prm.n_qtiles;
+        const int g = lin / full_group, r = lin - g * full_group;
+        int hg = prm.BH - g * prm.heads_per_group;
+        if (hg > prm.heads_per_group) hg = prm.heads_per_group;
+        const int pr = r / hg;
+        bh = g * prm.heads_per_group + (r - pr * hg);
+        qt = prm.causal ? prm.n_qtiles - 1 - pr : pr;
+    }
+    const int q0 = qt * BM;
+    const int kv_bh = (bh / prm.H) * prm.Hkv + (bh % prm.H) / (prm.H / prm.Hkv);
+    int last_key = prm.Sk - 1;
+    if (prm.causal && q0 + BM - 1 < last_key) last_key = q0 + BM - 1;
+    const int n = last_key / BN + 1;   // K/V steps
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(B_QREADY), 128);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(B_SFULL + b), 1);
+            mbar_init(bar(B_PFULL + b), 128);
+        }
+        mbar_init(bar(B_ODONE), 1);   // completes once per step: O += P_j V_j has finished
+        for (int s = 0; s < NSLOT; ++s) {
+            mbar_init(bar(B_KVFULL + s), 1);
+            mbar_init(bar(B_KVEMPTY + s), 1);
+        }
+        fence_barrier_init();
+        fence_proxy_async_smem();
+    }
+    if (warp == 4) {
+        tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    if (warp == 5 && elect_one()) {
+        prefetch_tensormap(&tmK);
+        prefetch_tensormap(&tmV);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    // Ring order = consumption order of the MMA warp: K_0, then for every step j: K_{j+1}, V_j.
+    // item index of K_j: j == 0 ? 0 : 2j - 1;  of V_j: 2j + 2 (2j + 1 for the last step, which has no K_{j+1}).
+    auto k_item = [&](int j) { return j == 0 ? 0 : 2 * j - 1; };
+    auto v_item = [&](int j) { return (j + 1 < n) ? 2 * j + 2 : 2 * j + 1; };
+
+    if (warp == 5) {
+        // =========================== TMA producer ===========================
+        const bool leader = elect_one();
+        auto load_kv = [&](const CUtensorMap* map, int item, int j) -> bool {
+            const int slot = item % NSLOT;
+            const uint32_t use = item / NSLOT;
+            if (!mbar_wait(bar(B_KVEMPTY + slot), (use & 1) ^ 1, abort_flag)) return false;
+            if (leader) {
+                mbar_arrive_expect_tx(bar(B_KVFULL + slot), C::KV_BYTES);
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx)
+                    tma_load_3d(sKV(slot) + bx * BN * 128, map, bar(B_KVFULL + slot), bx * 64, j * BN, kv_bh);
+            }
+            return true;
+        };
+        bool ok = load_kv(&tmK, 0, 0);
+        for (int j = 0; j < n && ok; ++j) {
+            if (j + 1 < n) ok = load_kv(&tmK, k_item(j + 1), j + 1);
+            if (ok) ok = load_kv(&tmV, v_item(j), j);
+        }
+    } else if (warp == 4) {
+        // =========================== MMA issuer ===========================
+        const bool leader = elect_one();
+        constexpr uint32_t IDESC_S = make_idesc_f16(BM, BN, DTYPE, 0, 0);   // Q (TMEM) and K both K-major
+        constexpr uint32_t IDESC_O = make_idesc_f16(BM, D, DTYPE, 0, 1);    // P (TMEM) K-major, V MN-major
+        constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
+        const uint32_t k_lo0 = smem_desc_lo(sKV(0), 16);
+        const uint32_t v_lo0 = smem_desc_lo(sKV(0), BN * 128);   // 8 KB between the 64-column boxes
+        auto kv_full_wait = [&](int item) {
+            return mbar_wait(bar(B_KVFULL + item % NSLOT), (item / NSLOT) & 1, abort_flag);
+        };
+        auto issue_s = [&](int j) {   // S_j = Q K_j^T into buffer j & 1 : 16 instructions of K = 16
+            if (leader) {
+                const uint32_t b0 = k_lo0 + (k_item(j) % NSLOT) * (C::KV_BYTES >> 4);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = ((kk >> 2) * BN * 128 + (kk & 3) * 32) >> 4;
+                    mma_f16_ts_lohi(tmem + C::S_COL + (j & 1) * 64, tmem + C::Q_COL + kk * 8, b0 + off, DESC_HI,
+                                    IDESC_S, kk > 0);
+                }
+                mma_commit(bar(B_SFULL + (j & 1)));
+                mma_commit(bar(B_KVEMPTY + k_item(j) % NSLOT));
+            }
+        };
+        bool ok = mbar_wait(bar(B_QREADY), 0, abort_flag) && kv_full_wait(0);
+        if (ok) {
+            tc_fence_after_sync();
+            issue_s(0);
+        }
+        for (int j = 0; j < n && ok; ++j) {
+            if (j + 1 < n) {
+                if (!(ok = kv_full_wait(k_item(j + 1)))) break;
+                tc_fence_after_sync();
+                issue_s(j + 1);
+            }
+            if (!(ok = kv_full_wait(v_item(j)))) break;
+            if (!(ok = mbar_wait(bar(B_PFULL + (j & 1)), (j >> 1) & 1, abort_flag))) break;
+            tc_fence_after_sync();
+            if (leader) {
+                const uint32_t b0 = v_lo0 + (v_item(j) % NSLOT) * (C::KV_BYTES >> 4);
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk)
+                    mma_f16_ts_lohi(tmem + C::O_COL, tmem + C::S_COL + (j & 1) * 64 + kk * 8, b0 + ((kk * 16 * 128) >> 4),
+                                    DESC_HI, IDESC_O, (j > 0 || kk > 0) ? 1u : 0u);
+                mma_commit(bar(B_KVEMPTY + v_item(j) % NSLOT));
+                mma_commit(bar(B_ODONE));
+            }
+        }
+    } else {
+        // =========================== softmax group ===========================
+        const int r = tid;                       // row inside the tile
+        const int row = q0 + r;
+        const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
+        const uint32_t tO = tmem + C::O_COL + lane_off, tQ = tmem + C::Q_COL + lane_off;
+        const float c = prm.scale_log2;
+        const int64_t grow = static_cast<int64_t>(bh) * prm.Sq + row;
+
+        // Q row -> tensor memory (two 16-bit values per column, in memory order)
+        {
+            const uint4* qrow = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(prm.q) + grow * D * 2);
+#pragma unroll
+            for (int ch = 0; ch < D / 64; ++ch) {   // 32 columns = 64 elements = 8 x 16 bytes per chunk
+                uint32_t w[32];
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    uint4 x = make_uint4(0u, 0u, 0u, 0u);
+                    if (row < prm.Sq) x = __ldg(qrow + ch * 8 + g);
+                    w[g * 4 + 0] = x.x;
+                    w[g * 4 + 1] = x.y;
+                    w[g * 4 + 2] = x.z;
+                    w[g * 4 + 3] = x.w;
+                }
+                tmem_st_32x32b_x32(tQ + ch * 32, w);
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(bar(B_QREADY));
+        }
+
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n; ++j) {
+            const uint32_t tS = tmem + C::S_COL + (j & 1) * 64 + lane_off;
+            if (!(ok = mbar_wait(bar(B_SFULL + (j & 1)), (j >> 1) & 1, abort_flag))) break;
+            tc_fence_after_sync();
+            uint32_t sr[BN];
+            tmem_ld_32x32b_x32(tS, sr);
+            tmem_ld_32x32b_x32(tS + 32, sr + 32);
+            tmem_ld_wait();
+
+            const int kv0 = j * BN;
+            const bool need_mask = (kv0 + BN > prm.Sk) || (prm.causal && kv0 + BN - 1 > q0);
+            bool done = false;
+
+            if (j > 0 && !need_mask) {
+                // fast path: exponentials against the reference maximum of the earlier steps, this
+                // step's row maximum computed on the side; redone below if a row ran ahead by > 2^8
+                const float mc = m * c;
+                const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
+                uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+                float mxs[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) mxs[i] = fmaxf(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
+#pragma unroll
+                for (int e = 16; e < BN; e += 16)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        mxs[i] = max3(mxs[i], __uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1]));
+                uint32_t pk[BN / 2];
+#pragma unroll
+                for (int e = 0; e < BN; e += 2) {
+                    const uint64_t s2 = pack_f32x2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1]));
+                    float x0, x1;
+                    unpack_f32x2(fma_f32x2(s2, c2, nmc2), x0, x1);
+                    const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                    acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(p0, p1));
+                    pk[e / 2] = pack2<DTYPE>(p0, p1);
+                }
+                const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                       fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+                if (!__any_sync(0xffffffffu, (mx - m) * c > 8.f)) {
+                    tmem_st_32x32b_x32(tS, pk);   // P overwrites the first half of its S buffer
+                    float a0, a1, a2, a3;
+                    unpack_f32x2(add_f32x2(acc[0], acc[1]), a0, a1);
+                    unpack_f32x2(add_f32x2(acc[2], acc[3]), a2, a3);
+                    l += (a0 + a1) + (a2 + a3);
+                    done = true;
+                }
+            }
+            if (!done) {
+                // general path: first step, diagonal / ragged step, or a row maximum that ran ahead
+                const int lim = !need_mask ? 0x7fffffff : ((prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1);
+                float mx = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < BN; ++e) {
+                    const float sv = (kv0 + e <= lim) ? __uint_as_float(sr[e]) : -INFINITY;
+                    sr[e] = __float_as_uint(sv);
+                    mx = fmaxf(mx, sv);
+                }
+                float alpha = 1.f;
+                if (j == 0) {
+                    m = (mx == -INFINITY) ? 0.f : mx;
+                } else if ((mx - m) * c > 8.f) {
+                    alpha = ex2_approx((m - mx) * c);
+                    m = mx;
+                }
+                if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                    // O += P V of step j-1 must have finished before O is rescaled.  S_j was issued
+                    // before that product, so its barrier does not cover it; B_ODONE does.  Step j-2's
+                    // product IS covered by S_j, hence the barrier is in phase j-1 or j and the parity
+                    // wait below cannot alias.
+                    if (!(ok = mbar_wait(bar(B_ODONE), (j - 1) & 1, abort_flag))) break;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        uint32_t orr[32];
+                        tmem_ld_32x32b_x32(tO + ch * 32, orr);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) orr[e] = __float_as_uint(__uint_as_float(orr[e]) * alpha);
+                        tmem_st_32x32b_x32(tO + ch * 32, orr);
+                    }
+                }
+                const float mc = m * c;
+                float rs = 0.f;
+                uint32_t pk[BN / 2];
+#pragma unroll
+                for (int e = 0; e < BN; e += 2) {
+                    const float s0 = __uint_as_float(sr[e]), s1 = __uint_as_float(sr[e + 1]);
+                    const float p0 = (s0 == -INFINITY) ? 0.f : ex2_approx(fmaf(s0, c, -mc));
+                    const float p1 = (s1 == -INFINITY) ? 0.f : ex2_approx(fmaf(s1, c, -mc));
+                    rs += p0 + p1;
+                    pk[e / 2] = pack2<DTYPE>(p0, p1);
+                }
+                tmem_st_32x32b_x32(tS, pk);
+                l = l * alpha + rs;
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(bar(B_PFULL + (j & 1)));
+        }
+
+        // ---- epilogue: O / l and LSE ----
+        if (ok) ok = mbar_wait(bar(B_ODONE), (n - 1) & 1, abort_flag);
+        if (ok) {
+            tc_fence_after_sync();
+            const float inv = (l > 0.f) ? 1.f / l : 0.f;
+            uint4* orow = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow * D * 2);
+#pragma unroll
+            for (int ch = 0; ch < D / 32; ++ch) {
+                uint32_t orr[32];
+                tmem_ld_32x32b_x32(tO + ch * 32, orr);
+                tmem_ld_wait();
+                if (row < prm.Sq) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint4 w;
+                        w.x = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 0]) * inv, __uint_as_float(orr[g * 8 + 1]) * inv);
+                        w.y = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 2]) * inv, __uint_as_float(orr[g * 8 + 3]) * inv);
+                        w.z = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 4]) * inv, __uint_as_float(orr[g * 8 + 5]) * inv);
+                        w.w = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 6]) * inv, __uint_as_float(orr[g * 8 + 7]) * inv);
+                        orow[ch * 4 + g] = w;
+                    }
+                }
+            }
+            if (row < prm.Sq) prm.lse[grow] = (l > 0.f) ? m * prm.scale + logf(l) : -INFINITY;
+        }
+    }
+
+    // ---- teardown (also reached after a timed-out wait) ----
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && *abort_flag != 0) atomicExch(prm.status, kStatusTimeout);
+    if (warp == 4) tmem_dealloc(tmem, C::TMEM_COLS);
+}
+
+}  // namespace attn_tc

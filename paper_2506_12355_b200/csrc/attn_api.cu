@@ -7,6 +7,7 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "../../include/attn_fwd.h"
@@ -94,6 +95,38 @@ int validate(const void* q, const void* k, const void* v, const void* o, const v
     return ATTN_OK;
 }
 
+// Work counters of the persistent kernel: every launch takes the next slot of this ring and zeroes
+// it on its stream right before the kernel, so launches in flight on different streams do not share
+// a counter (unless more than kCounterSlots launches are in flight at once).
+constexpr int kCounterSlots = 1024;
+__device__ unsigned int g_work_counters[kCounterSlots];
+std::atomic<unsigned int> g_launch_seq{0};
+
+struct DeviceInfo {
+    unsigned int* counters = nullptr;
+    int sm_count = 0;
+};
+
+// Per-device facts resolved on first use (symbol address of the counters, SM count).
+int device_info(DeviceInfo* out) {
+    static std::mutex mu;
+    static DeviceInfo info[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ATTN_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!info[dev].counters) {
+        void* p = nullptr;
+        int sms = 0;
+        if (cudaGetSymbolAddress(&p, g_work_counters) != cudaSuccess || !p) return ATTN_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            return ATTN_ERR_CUDA;
+        info[dev].counters = static_cast<unsigned int*>(p);
+        info[dev].sm_count = sms;
+    }
+    *out = info[dev];
+    return ATTN_OK;
+}
+
 int* device_status_ptr() {
     int* p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_device_status) != cudaSuccess) return nullptr;
@@ -142,7 +175,7 @@ int launch_tc_basic(const void* q, const void* k, const void* v, void* o, float*
 }
 
 #ifdef ATTN_TC_PROFILE
-long long* g_prof_buffer = nullptr;  // development builds: per-CTA cycle sums, [grid][32]
+long long* g_prof_buffer = nullptr;  // development builds only
 #endif
 
 // Pipelined, warp-specialised kernel (head dims 64 and 128): one CTA per pair of 128-row Q tiles.
@@ -185,10 +218,18 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     hpg *= H / Hkv;  // the query heads of one K/V head share its footprint
     if (hpg > BH) hpg = BH;
     prm.heads_per_group = static_cast<int>(hpg);
+    prm.n_items = static_cast<int>(n_pairs * BH);
 #ifdef ATTN_TC_PROFILE
     prm.prof = g_prof_buffer;
 #endif
-    kern<<<static_cast<unsigned>(n_pairs * BH), C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, prm);
+    // persistent grid: one CTA per SM; the first item of a CTA is its block index, the rest come from
+    // a device counter that is zeroed on the stream right before the launch
+    DeviceInfo di;
+    if (device_info(&di) != ATTN_OK) return ATTN_ERR_CUDA;
+    prm.counter = di.counters + (g_launch_seq.fetch_add(1) % kCounterSlots);
+    if (cudaMemsetAsync(prm.counter, 0, sizeof(unsigned int), st) != cudaSuccess) return ATTN_ERR_CUDA;
+    const unsigned grid = static_cast<unsigned>(prm.n_items < di.sm_count ? prm.n_items : di.sm_count);
+    kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, prm);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
@@ -309,6 +350,10 @@ int static_workspace_ptr(void** out) {
 
 extern "C" {
 
+#ifdef ATTN_TC_PROFILE
+void attn_debug_set_profile_buffer(long long* p) { g_prof_buffer = p; }
+#endif
+
 int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk, int D,
              float scale, int causal, int dtype, void* stream) {
     return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, H, Sq, Sk, D, scale, causal, dtype, stream);
@@ -396,10 +441,6 @@ int attn_last_device_status(void* stream) {
     }
     return h == 0 ? ATTN_OK : ATTN_ERR_DEVICE_TIMEOUT;
 }
-
-#ifdef ATTN_TC_PROFILE
-void attn_debug_set_profile_buffer(long long* device_buffer) { g_prof_buffer = device_buffer; }
-#endif
 
 const char* attn_status_string(int status) {
     switch (status) {

@@ -1,23 +1,29 @@
-// Warp-specialised, pipelined tcgen05 attention forward kernel for head dims 64 and 128.
+// Warp-specialised, pipelined, persistent tcgen05 attention forward kernel for head dims 64 and 128.
 //
-// One CTA owns TWO 128-row Q tiles of one (batch, head) and walks the K/V tiles of that head
-// (the loop of Appendix C, Listings 1-2, with the prefetch of Listing 1 generalised to a
-// multi-stage ring):
+// A work item is one (batch, head) and a PAIR of 128-row Q tiles; a CTA walks the K/V tiles of
+// that head for both Q tiles (the loop of Appendix C, Listings 1-2 of the paper, with the prefetch
+// of Listing 1 generalised to a multi-stage ring) and then takes the next item:
 //
 //   warps 0-3   softmax group of Q tile 0: S -> P (online softmax, exp2), rare O rescale, epilogue
 //   warps 4-7   softmax group of Q tile 1
 //   warp  8     MMA issuer: S_t = Q_t K_j^T and O_t += P_t V_j, accumulators in tensor memory
-//   warp  9     TMA producer: Q tiles once, K_j / V_j tiles through a ring of shared-memory slots
+//   warp  9     scheduler + TMA producer: draws work items, loads Q tiles and the K_j / V_j ring
 //   warps 10-11 idle (they complete the third warpgroup so that registers can be re-balanced)
 //
 // While one softmax group turns S_t into P_t, the tensor core works on the other tile, so the
-// exponentials and the MMAs overlap.  P_t is written back into the tensor-memory columns of
-// S_t as 16-bit values and is the A operand of the second product, which is this
-// architecture's form of the register-level fusion of the two GEMMs in Section 3.2.2.
+// exponentials and the MMAs overlap.  P_t is written back into the tensor-memory columns of S_t as
+// 16-bit values and is the A operand of the second product, which is this architecture's form of
+// the register-level fusion of the two GEMMs in Section 3.2.2.
 //
-// Running maximum: the reference maximum m of a row is only advanced when the true maximum
-// has grown by more than 2^8; otherwise the stale m is kept (P values up to 256, exact after
-// the final division by l), so the O accumulator rarely needs rescaling.
+// Persistence: the grid has one CTA per SM.  Items are ordered longest-first (causal) inside
+// L2-sized groups of heads; the first item of a CTA is its block index, later ones come from a
+// global counter (zeroed by the host before the launch).  Barriers, tensor memory and the K/V ring
+// live across items, so the producer already loads the next item's Q/K/V and the MMA warp already
+// issues its first S while the softmax groups still write the previous item's O.
+//
+// Running maximum: the reference maximum m of a row is only advanced when the true maximum has
+// grown by more than 2^8; otherwise the stale m is kept (P values up to 256, exact after the final
+// division by l), so the O accumulator rarely needs rescaling.
 #pragma once
 #include "attn_tc_basic.cuh"
 
@@ -32,7 +38,7 @@ struct PipeCfg {
     static constexpr int KV_BYTES = BN * D * 2;
     static constexpr int NSLOT = (D == 128) ? 5 : 8;     // ring slots (each holds one K or V tile)
     static constexpr int TILE_BYTES = 2 * Q_BYTES + NSLOT * KV_BYTES;
-    static constexpr int MISC_BYTES = 512;               // barriers, TMEM slot, abort flag
+    static constexpr int MISC_BYTES = 512;               // barriers, scheduler slots, TMEM slot, abort flag
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
     static constexpr int TMEM_COLS = 512;
     static constexpr int THREADS = 384;
@@ -47,39 +53,55 @@ struct PipeParams {
     float scale, scale_log2;
     int causal;
     int* status;
-    int n_pairs;          // 256-row Q tile pairs per head
-    int BH;               // batch * heads
-    int heads_per_group;  // heads whose K/V are walked together (L2 residency)
-    int H, Hkv;           // query heads and key/value heads per batch element (H % Hkv == 0)
+    int n_pairs;            // 256-row Q tile pairs per head
+    int BH;                 // batch * query heads
+    int heads_per_group;    // heads whose K/V are walked together (L2 residency)
+    int H, Hkv;             // query heads and key/value heads per batch element (H % Hkv == 0)
+    int n_items;            // n_pairs * BH
+    unsigned int* counter;  // work counter, zero at launch: item = gridDim.x + atomicAdd(counter, 1)
 #ifdef ATTN_TC_PROFILE
-    long long* prof;      // [grid][32] cycle sums per phase (development builds only)
+    long long* prof;        // development builds: [grid][16] cycle sums of softmax group 1, row 0
 #endif
 };
 
-#ifndef ATTN_SUM_MODE
-#define ATTN_SUM_MODE 0
-#endif
-#ifndef ATTN_MAX3
-#define ATTN_MAX3 0
-#endif
+// Register re-balancing: 384 threads start with 168 registers each (64512 of the SM's 65536); the
+// service warpgroup drops to 64 (frees 13312) and the two softmax warpgroups rise to 216 (need 12288).
+__device__ __forceinline__ void reg_inc_softmax() { asm volatile("setmaxnreg.inc.sync.aligned.u32 216;"); }
+__device__ __forceinline__ void reg_dec_service() { asm volatile("setmaxnreg.dec.sync.aligned.u32 64;"); }
 
-#ifndef ATTN_PROF_ROW
-#define ATTN_PROF_ROW 0
-#endif
-#ifdef ATTN_TC_PROFILE
-#define PROF_DECL(n) long long prof_t0 = clock64(), prof_acc[n] = {}
-#define PROF_LAP(i) do { const long long prof_t1 = clock64(); prof_acc[i] += prof_t1 - prof_t0; prof_t0 = prof_t1; } while (0)
-#define PROF_STAMP(cond, slot) do { if (cond) prm.prof[blockIdx.x * 32 + (slot)] = clock64(); } while (0)
-#define PROF_FLUSH(base, n) do { for (int i_ = 0; i_ < (n); ++i_) prm.prof[blockIdx.x * 32 + (base) + i_] = prof_acc[i_]; } while (0)
-#else
-#define PROF_DECL(n)
-#define PROF_LAP(i)
-#define PROF_STAMP(cond, slot)
-#define PROF_FLUSH(base, n)
-#endif
+// One work item, decoded identically by every role.
+struct PipeItem {
+    int bh, kv_bh, q0;
+    int n_kv[2];   // K/V tiles each Q tile needs (0: tile beyond Sq)
+    int n_max;
+};
 
-__device__ __forceinline__ void reg_inc_224() { asm volatile("setmaxnreg.inc.sync.aligned.u32 224;"); }
-__device__ __forceinline__ void reg_dec_56() { asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); }
+__device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int lin, int BM, int BN) {
+    PipeItem it;
+    const int full_group = prm.heads_per_group * prm.n_pairs;
+    const int g = lin / full_group, r = lin - g * full_group;
+    int hg = prm.BH - g * prm.heads_per_group;
+    if (hg > prm.heads_per_group) hg = prm.heads_per_group;
+    const int pr = r / hg;
+    it.bh = g * prm.heads_per_group + (r - pr * hg);
+    const int pair = prm.causal ? prm.n_pairs - 1 - pr : pr;   // causal: longest rows first
+    it.q0 = pair * 2 * BM;
+    // grouped-query attention: H / Hkv consecutive query heads read the same K/V head
+    it.kv_bh = (it.bh / prm.H) * prm.Hkv + (it.bh % prm.H) / (prm.H / prm.Hkv);
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int qs = it.q0 + t * BM;
+        if (qs >= prm.Sq) {
+            it.n_kv[t] = 0;
+        } else {
+            int last_key = prm.Sk - 1;
+            if (prm.causal && qs + BM - 1 < last_key) last_key = qs + BM - 1;
+            it.n_kv[t] = last_key / BN + 1;
+        }
+    }
+    it.n_max = it.n_kv[0] > it.n_kv[1] ? it.n_kv[0] : it.n_kv[1];
+    return it;
+}
 
 template <int D, int DTYPE, int POLY_NUM, int POLY_DEN>
 __global__ void __launch_bounds__(384, 1)
@@ -94,57 +116,42 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     auto sQ = [&](int t) { return smem_base + t * C::Q_BYTES; };
     auto sKV = [&](int slot) { return smem_base + 2 * C::Q_BYTES + slot * C::KV_BYTES; };
 
-    // misc area: barriers
+    // misc area: barriers, then scheduler slots, TMEM base, abort flag
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
     const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
-    enum { B_Q = 0, B_SFULL = 2, B_PFULL = 4, B_PFULL2 = 6, B_OFINAL = 8, B_KVFULL = 10, B_KVEMPTY = 10 + NSLOT,
-           B_COUNT = 10 + 2 * NSLOT };
+    enum {
+        B_QFULL = 0,      // [2] Q tile t loaded (TMA bytes)
+        B_QEMPTY = 2,     // [2] every S MMA of tile t of the current item has finished: Q_t may be overwritten
+        B_SFULL = 4,      // [2] S_t ready (MMA commit)
+        B_PFULL = 6,      // [2] first three quarters of P_t written (128 softmax threads)
+        B_PFULL2 = 8,     // [2] rest of P_t written
+        B_OFINAL = 10,    // [2] last O_t += P_t V of the item has finished
+        B_OFREE = 12,     // [2] the epilogue has read O_t out of tensor memory (128 softmax threads)
+        B_SCHEDFULL = 14, // [2] scheduler slot holds the next item
+        B_SCHEDEMPTY = 16,// [2] slot read by the MMA warp and the 8 softmax warps
+        B_KVFULL = 18,
+        B_KVEMPTY = 18 + NSLOT,
+        B_COUNT = 18 + 2 * NSLOT
+    };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 1;
+    volatile int* sched_item = reinterpret_cast<volatile int*>(bars + B_COUNT);       // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT) + 2;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 3;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // ---- which work item ----
-    int pair, bh;
-    {
-        const int lin = blockIdx.x;
-        const int full_group = prm.heads_per_group * prm.n_pairs;
-        const int g = lin / full_group, r = lin - g * full_group;
-        int hg = prm.BH - g * prm.heads_per_group;
-        if (hg > prm.heads_per_group) hg = prm.heads_per_group;
-        const int pr = r / hg;
-        bh = g * prm.heads_per_group + (r - pr * hg);
-        pair = prm.causal ? prm.n_pairs - 1 - pr : pr;  // causal: longest rows first
-    }
-    const int q0 = pair * 2 * BM;
-    // grouped-query attention: H / Hkv consecutive query heads read the same K/V head
-    const int kv_bh = (bh / prm.H) * prm.Hkv + (bh % prm.H) / (prm.H / prm.Hkv);
-
-    // K/V tiles each Q tile needs
-    int n_kv[2];
-#pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        const int qs = q0 + t * BM;
-        if (qs >= prm.Sq) {
-            n_kv[t] = 0;
-        } else {
-            int last_key = prm.Sk - 1;
-            if (prm.causal && qs + BM - 1 < last_key) last_key = qs + BM - 1;
-            n_kv[t] = last_key / BN + 1;
-        }
-    }
-    const int n_max = n_kv[0] > n_kv[1] ? n_kv[0] : n_kv[1];
-
     if (tid == 0) {
         *abort_flag = 0;
-        mbar_init(bar(B_Q + 0), 1);
-        mbar_init(bar(B_Q + 1), 1);
         for (int t = 0; t < 2; ++t) {
+            mbar_init(bar(B_QFULL + t), 1);
+            mbar_init(bar(B_QEMPTY + t), 1);
             mbar_init(bar(B_SFULL + t), 1);
-            mbar_init(bar(B_PFULL + t), 128);    // first three quarters of P_t written
-            mbar_init(bar(B_PFULL2 + t), 128);   // rest of P_t written
+            mbar_init(bar(B_PFULL + t), 128);
+            mbar_init(bar(B_PFULL2 + t), 128);
             mbar_init(bar(B_OFINAL + t), 1);
+            mbar_init(bar(B_OFREE + t), 128);
+            mbar_init(bar(B_SCHEDFULL + t), 1);
+            mbar_init(bar(B_SCHEDEMPTY + t), 9);
         }
         for (int s = 0; s < NSLOT; ++s) {
             mbar_init(bar(B_KVFULL + s), 1);
@@ -167,46 +174,74 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
+    // Consumers of the scheduler: wait for the k-th item of this CTA, read it, hand the slot back.
+    auto next_item = [&](int k, bool hand_back) -> int {
+        const int slot = k & 1;
+        if (!mbar_wait(bar(B_SCHEDFULL + slot), (k >> 1) & 1, abort_flag)) return -1;
+        const int item = sched_item[slot];
+        if (hand_back) mbar_arrive(bar(B_SCHEDEMPTY + slot));
+        return item;
+    };
+
     if (warp >= 8) {
-        reg_dec_56();
+        reg_dec_service();
         // Both service warps run their loops with all 32 lanes (uniform control flow keeps the
         // address arithmetic on the uniform datapath); one elected lane issues the TMA / MMA
         // instructions.
         if (warp == 9) {
-            // =========================== TMA producer ===========================
+            // =========================== scheduler + TMA producer ===========================
             const bool leader = elect_one();
-            PROF_DECL(2);
-            auto load_q = [&](int t) {
+            int kv_base = 0;            // ring items issued for earlier work items
+            int q_uses[2] = {0, 0};     // work items that loaded Q tile t so far
+            for (int k = 0;; ++k) {
+                // ---- draw the next work item and publish it ----
+                const int slot = k & 1;
+                if (!mbar_wait(bar(B_SCHEDEMPTY + slot), ((k >> 1) & 1) ^ 1, abort_flag)) break;
                 if (leader) {
-                    mbar_arrive_expect_tx(bar(B_Q + t), C::Q_BYTES);
-#pragma unroll
-                    for (int bx = 0; bx < NBOX; ++bx)
-                        tma_load_3d(sQ(t) + bx * BM * 128, &tmQ, bar(B_Q + t), bx * 64, q0 + t * BM, bh);
+                    int next = (k == 0) ? static_cast<int>(blockIdx.x)
+                                        : static_cast<int>(gridDim.x + atomicAdd(prm.counter, 1u));
+                    if (next >= prm.n_items) next = -1;
+                    sched_item[slot] = next;
+                    mbar_arrive(bar(B_SCHEDFULL + slot));
                 }
-            };
-            auto load_kv = [&](const CUtensorMap* map, int item, int j) -> bool {
-                const int slot = item % NSLOT;
-                const uint32_t use = item / NSLOT;
-                if (!mbar_wait(bar(B_KVEMPTY + slot), (use & 1) ^ 1, abort_flag)) return false;
-                PROF_LAP(0);
-                if (leader) {
-                    mbar_arrive_expect_tx(bar(B_KVFULL + slot), C::KV_BYTES);
+                const int item = next_item(k, false);
+                if (item < 0) break;
+                const PipeItem it = pipe_decode_item(prm, item, BM, BN);
+
+                auto load_q = [&](int t) -> bool {
+                    // the previous item's S MMAs on this Q buffer must have finished
+                    if (!mbar_wait(bar(B_QEMPTY + t), (q_uses[t] & 1) ^ 1, abort_flag)) return false;
+                    if (leader) {
+                        mbar_arrive_expect_tx(bar(B_QFULL + t), C::Q_BYTES);
 #pragma unroll
-                    for (int bx = 0; bx < NBOX; ++bx)
-                        tma_load_3d(sKV(slot) + bx * BN * 128, map, bar(B_KVFULL + slot), bx * 64, j * BN, kv_bh);
+                        for (int bx = 0; bx < NBOX; ++bx)
+                            tma_load_3d(sQ(t) + bx * BM * 128, &tmQ, bar(B_QFULL + t), bx * 64, it.q0 + t * BM, it.bh);
+                    }
+                    ++q_uses[t];
+                    return true;
+                };
+                auto load_kv = [&](const CUtensorMap* map, int ring_item, int j) -> bool {
+                    const int s = ring_item % NSLOT;
+                    const uint32_t use = ring_item / NSLOT;
+                    if (!mbar_wait(bar(B_KVEMPTY + s), (use & 1) ^ 1, abort_flag)) return false;
+                    if (leader) {
+                        mbar_arrive_expect_tx(bar(B_KVFULL + s), C::KV_BYTES);
+#pragma unroll
+                        for (int bx = 0; bx < NBOX; ++bx)
+                            tma_load_3d(sKV(s) + bx * BN * 128, map, bar(B_KVFULL + s), bx * 64, j * BN, it.kv_bh);
+                    }
+                    return true;
+                };
+                bool ok = true;
+                if (it.n_kv[0] > 0) ok = load_q(0);
+                for (int j = 0; j < it.n_max && ok; ++j) {
+                    ok = load_kv(&tmK, kv_base + 2 * j, j);
+                    if (ok && j == 0 && it.n_kv[1] > 0) ok = load_q(1);
+                    if (ok) ok = load_kv(&tmV, kv_base + 2 * j + 1, j);
                 }
-                return true;
-            };
-            if (n_kv[0] > 0) load_q(0);
-            for (int j = 0; j < n_max; ++j) {
-                if (!load_kv(&tmK, 2 * j, j)) break;
-                if (j == 0 && n_kv[1] > 0) load_q(1);
-                if (!load_kv(&tmV, 2 * j + 1, j)) break;
-                PROF_LAP(1);
+                if (!ok) break;
+                kv_base += 2 * it.n_max;
             }
-#ifdef ATTN_TC_PROFILE
-            if (leader) PROF_FLUSH(24, 2);
-#endif
         } else if (warp == 8) {
             // =========================== MMA issuer ===========================
             const bool leader = elect_one();
@@ -216,9 +251,9 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             const uint32_t q_lo[2] = {smem_desc_lo(sQ(0), 16), smem_desc_lo(sQ(1), 16)};
             const uint32_t k_lo0 = smem_desc_lo(sKV(0), 16);          // K tile in slot 0 (K-major)
             const uint32_t v_lo0 = smem_desc_lo(sKV(0), BN * 128);    // V tile in slot 0 (MN-major)
-            auto issue_s = [&](int t, int slot) {   // S_t = Q_t K^T : D/16 instructions of K = 16
+            auto issue_s = [&](int t, int s) {   // S_t = Q_t K^T : D/16 instructions of K = 16
                 if (leader) {
-                    const uint32_t a0 = q_lo[t], b0 = k_lo0 + slot * (C::KV_BYTES >> 4);
+                    const uint32_t a0 = q_lo[t], b0 = k_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
                         const uint32_t off = ((kk >> 2) * 128 * 128 + (kk & 3) * 32) >> 4;
@@ -226,9 +261,9 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     }
                 }
             };
-            auto issue_pv = [&](int t, int slot, bool accumulate, int kk_begin, int kk_end) {
-                if (leader) {                       // O_t += P_t V : K = 16 keys per instruction
-                    const uint32_t b0 = v_lo0 + slot * (C::KV_BYTES >> 4);
+            auto issue_pv = [&](int t, int s, bool accumulate, int kk_begin, int kk_end) {
+                if (leader) {                    // O_t += P_t V : K = 16 keys per instruction
+                    const uint32_t b0 = v_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
                     for (int kk = kk_begin; kk < kk_end; ++kk)
                         mma_f16_ts_lohi(tmem + C::o_col(t), tmem + C::s_col(t) + kk * 8, b0 + ((kk * 16 * 128) >> 4),
@@ -238,254 +273,329 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             auto commit = [&](int b) {
                 if (leader) mma_commit(bar(b));
             };
-            auto kv_full_wait = [&](int item) {
-                return mbar_wait(bar(B_KVFULL + item % NSLOT), (item / NSLOT) & 1, abort_flag);
+            auto kv_full_wait = [&](int ring_item) {
+                return mbar_wait(bar(B_KVFULL + ring_item % NSLOT), (ring_item / NSLOT) & 1, abort_flag);
             };
+            int kv_base = 0;
+            int it_base[2] = {0, 0};   // K/V steps tile t has gone through in earlier work items
+            int uses[2] = {0, 0};      // work items in which tile t took part
             bool ok = true;
-            if (n_max > 0) {
-                if (n_kv[0] > 0) ok = mbar_wait(bar(B_Q + 0), 0, abort_flag);
-                ok = ok && kv_full_wait(0);
-                if (ok && n_kv[0] > 0) {
-                    tc_fence_after_sync();
-                    issue_s(0, 0);
-                    commit(B_SFULL + 0);
-                }
-                if (ok && n_kv[1] > 0) {
-                    ok = mbar_wait(bar(B_Q + 1), 0, abort_flag);
-                    if (ok) {
-                        tc_fence_after_sync();
-                        issue_s(1, 0);
-                        commit(B_SFULL + 1);
-                    }
-                }
-                if (ok) commit(B_KVEMPTY + 0);
-            }
-            PROF_DECL(12);
-            for (int j = 0; j < n_max && ok; ++j) {
-                const int vitem = 2 * j + 1, kitem = 2 * j + 2;
-                const int vslot = vitem % NSLOT, kslot = kitem % NSLOT;
-                const uint32_t par = j & 1;
-                // both tiles of this step are normally long loaded: check them off the P -> S critical path
-                if (!(ok = kv_full_wait(vitem))) break;
-                bool k_ready = false;
-                if (j + 1 < n_max) {
-                    if (!(ok = kv_full_wait(kitem))) break;
-                    k_ready = true;
-                }
-                PROF_LAP(0);
+            for (int k = 0; ok; ++k) {
+                const int item = next_item(k, leader);
+                if (item < 0) break;
+                const PipeItem it = pipe_decode_item(prm, item, BM, BN);
+                // ---- first S of both tiles ----
+                ok = kv_full_wait(kv_base);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
-                    if (j < n_kv[t]) {
-                        if (!(ok = mbar_wait(bar(B_PFULL + t), par, abort_flag))) break;
-                        PROF_LAP(1 + 5 * t);
-                        tc_fence_after_sync();
-                        issue_pv(t, vslot, j > 0, 0, 3 * BN / 64);
-                        if (!(ok = mbar_wait(bar(B_PFULL2 + t), par, abort_flag))) break;
-                        PROF_STAMP(leader && t == 0 && j == 64, 27);
-                        PROF_LAP(2 + 5 * t);
-                        tc_fence_after_sync();
-                        issue_pv(t, vslot, true, 3 * BN / 64, BN / 16);
-                        if (j + 1 == n_kv[t]) commit(B_OFINAL + t);
-                    }
-                    if (t == 1) commit(B_KVEMPTY + vslot);
-                    PROF_LAP(3 + 5 * t);
-                    if (j + 1 < n_kv[t]) {
-                        if (!k_ready) {
-                            if (!(ok = kv_full_wait(kitem))) break;
-                            k_ready = true;
+                    if (ok && it.n_kv[t] > 0) {
+                        ok = mbar_wait(bar(B_QFULL + t), uses[t] & 1, abort_flag);
+                        if (ok) {
+                            tc_fence_after_sync();
+                            issue_s(t, kv_base % NSLOT);
+                            commit(B_SFULL + t);
+                            if (it.n_kv[t] == 1) commit(B_QEMPTY + t);
                         }
-                        PROF_LAP(4 + 5 * t);
-                        tc_fence_after_sync();
-                        issue_s(t, kslot);
-                        commit(B_SFULL + t);
-                        PROF_STAMP(leader && t == 0 && j == 64, 28);
                     }
-                    PROF_LAP(5 + 5 * t);
                 }
-                if (ok && j + 1 < n_max) commit(B_KVEMPTY + kslot);
+                if (ok && it.n_max > 0) commit(B_KVEMPTY + kv_base % NSLOT);
+                for (int j = 0; j < it.n_max && ok; ++j) {
+                    const int vitem = kv_base + 2 * j + 1, kitem = kv_base + 2 * j + 2;
+                    const int vslot = vitem % NSLOT, kslot = kitem % NSLOT;
+                    // both tiles of this step are normally long loaded: check them off the P -> S critical path
+                    if (!(ok = kv_full_wait(vitem))) break;
+                    if (j + 1 < it.n_max && !(ok = kv_full_wait(kitem))) break;
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (j < it.n_kv[t]) {
+                            const uint32_t par = (it_base[t] + j) & 1;
+                            if (!(ok = mbar_wait(bar(B_PFULL + t), par, abort_flag))) break;
+                            // the epilogue of the previous item must have read O_t before it is overwritten
+                            if (j == 0 && uses[t] > 0 && !(ok = mbar_wait(bar(B_OFREE + t), (uses[t] - 1) & 1, abort_flag))) break;
+                            tc_fence_after_sync();
+                            issue_pv(t, vslot, j > 0, 0, 3 * BN / 64);
+                            if (!(ok = mbar_wait(bar(B_PFULL2 + t), par, abort_flag))) break;
+                            tc_fence_after_sync();
+                            issue_pv(t, vslot, true, 3 * BN / 64, BN / 16);
+                            if (j + 1 == it.n_kv[t]) commit(B_OFINAL + t);
+                        }
+                        if (t == 1) commit(B_KVEMPTY + vslot);
+                        if (j + 1 < it.n_kv[t]) {
+                            tc_fence_after_sync();
+                            issue_s(t, kslot);
+                            commit(B_SFULL + t);
+                            if (j + 2 == it.n_kv[t]) commit(B_QEMPTY + t);   // that was the last S of this item
+                        }
+                    }
+                    if (ok && j + 1 < it.n_max) commit(B_KVEMPTY + kslot);
+                }
+                kv_base += 2 * it.n_max;
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    it_base[t] += it.n_kv[t];
+                    uses[t] += it.n_kv[t] > 0 ? 1 : 0;
+                }
             }
-#ifdef ATTN_TC_PROFILE
-            if (leader) PROF_FLUSH(0, 12);
-#endif
         }
     } else {
         // =========================== softmax groups ===========================
-        reg_inc_224();
+        reg_inc_softmax();
         const int t = warp >> 2;                       // Q tile of this group
         const int r = tid & 127;                       // row inside the tile
-        const int row = q0 + t * BM + r;
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + C::s_col(t) + lane_off, tO = tmem + C::o_col(t) + lane_off;
         const float c = prm.scale_log2;
-        const int n = n_kv[t];
-        float m = -INFINITY, l = 0.f;
+        int it_base = 0, uses = 0;
         bool ok = true;
-
-        PROF_DECL(6);
-        for (int j = 0; j < n; ++j) {
-            if (!(ok = mbar_wait(bar(B_SFULL + t), j & 1, abort_flag))) break;
-            PROF_STAMP(t == 0 && r == 0 && j == 65, 29);
-            PROF_LAP(0);
-            tc_fence_after_sync();
-            uint32_t sr[BN];
-#pragma unroll
-            for (int ch = 0; ch < BN / 32; ++ch) tmem_ld_32x32b_x32(tS + ch * 32, sr + ch * 32);
-            tmem_ld_wait();
-            PROF_LAP(1);
-
-            const int kv0 = j * BN;
-            const bool need_mask = (kv0 + BN > prm.Sk) || (prm.causal && kv0 + BN - 1 > q0 + t * BM);
-            bool done = false;
-
-            if (j > 0 && !need_mask) {
-                // ---- fast path: exponentials against the reference maximum of the previous tiles,
-                // the row maximum of this tile computed on the side.  Valid when no row of the warp
-                // has grown by more than 2^8; otherwise everything is redone by the general path.
-                const float mc = m * c;
-                const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
-#if ATTN_SUM_MODE == 0
-                uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // 8 partial row sums
+#ifdef ATTN_TC_PROFILE
+        long long pacc[8] = {}, pt0 = clock64();
+#define PLAP(i) do { long long t1_ = clock64(); pacc[i] += t1_ - pt0; pt0 = t1_; } while (0)
 #else
-                float accs[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#define PLAP(i)
 #endif
-                float mxs[8];
+
+        for (int k = 0; ok; ++k) {
+            const int item = next_item(k, lane == 0);
+            PLAP(0);
+            if (item < 0) break;
+            const PipeItem it = pipe_decode_item(prm, item, BM, BN);
+            const int n = it.n_kv[t];
+            if (n == 0) continue;
+            const int q0 = it.q0;
+            const int row = q0 + t * BM + r;
+            const int row_w0 = q0 + t * BM + (warp & 3) * 32;   // first row of this warp
+            float m = -INFINITY, l = 0.f;
+
+            for (int j = 0; j < n; ++j) {
+                if (!(ok = mbar_wait(bar(B_SFULL + t), (it_base + j) & 1, abort_flag))) break;
+                PLAP(j == 0 ? 1 : (j == n - 1 ? 5 : 3));
+                tc_fence_after_sync();
+                // Visibility of this K/V tile, per warp (rows 32 w .. 32 w + 31 of the Q tile): a chunk of
+                // 32 keys is FULL (every row sees all of it), EMPTY (no row sees any of it) or PARTIAL.
+                const int kv0 = j * BN;
+                const int lim = (prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1;   // last visible key of this row
+                const int lim_lo = (prm.causal && row_w0 < prm.Sk - 1) ? row_w0 : prm.Sk - 1;
+                const int lim_hi = (prm.causal && row_w0 + 31 < prm.Sk - 1) ? row_w0 + 31 : prm.Sk - 1;
+                auto chunk_full = [&](int ch) { return kv0 + 32 * ch + 31 <= lim_lo; };
+                auto chunk_empty = [&](int ch) { return kv0 + 32 * ch > lim_hi; };
+                const bool all_full = chunk_full(BN / 32 - 1);
+
+                // Masked (diagonal / ragged) tiles are brought into the form the fast path expects, so that
+                // they run the same (instruction-cache resident) code as every other tile: hidden scores are
+                // overwritten with -inf in tensor memory (their exponential is 0) before the row is loaded.
+                // A zero scale cannot use -inf (-inf * 0 is NaN): it takes the general path instead.
+                if (c > 0.f && !all_full) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) mxs[i] = fmaxf(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
-                auto exp_chunk = [&](int ch) {
-                    uint32_t pk[16];
+                    for (int ch = 0; ch < BN / 32; ++ch) {
+                        if (chunk_full(ch)) continue;
+                        uint32_t tmp[32];
+                        if (chunk_empty(ch)) {
 #pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const uint64_t s2 = pack_f32x2(__uint_as_float(sr[ch * 32 + e]), __uint_as_float(sr[ch * 32 + e + 1]));
-                        const uint64_t x2 = fma_f32x2(s2, c2, nmc2);
-                        float x0, x1, p0, p1;
-                        unpack_f32x2(x2, x0, x1);
-                        if (((ch * 16 + e / 2) % POLY_DEN) < POLY_NUM) {   // this pair: polynomial on the FMA pipe
-                            ex2_poly_f32x2(pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f)), p0, p1);
-                        } else {                                           // this pair: special-function unit
-                            p0 = ex2_approx(x0);
-                            p1 = ex2_approx(x1);
+                            for (int e = 0; e < 32; ++e) tmp[e] = 0xff800000u;   // -inf
+                        } else {
+                            tmem_ld_32x32b_x32(tS + ch * 32, tmp);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (kv0 + ch * 32 + e > lim) tmp[e] = 0xff800000u;
                         }
-#if ATTN_SUM_MODE == 0
-                        acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(p0, p1));
-#else
-                        accs[e & 7] += p0;
-                        accs[(e & 7) + 1] += p1;
-#endif
-                        pk[e / 2] = pack2<DTYPE>(p0, p1);
+                        tmem_st_32x32b_x32(tS + ch * 32, tmp);
                     }
-                    tmem_st_32x32b_x16(tS + ch * 16, pk);   // P overwrites the S columns already in registers
-                };
+                    tmem_st_wait();
+                }
+                uint32_t sr[BN];
 #pragma unroll
-                for (int ch = 0; ch < BN / 32 - 1; ++ch) {
-                    exp_chunk(ch);
-                    // a third of the row maximum per chunk, off the critical path of the exponentials
+                for (int ch = 0; ch < BN / 32; ++ch) tmem_ld_32x32b_x32(tS + ch * 32, sr + ch * 32);
+                tmem_ld_wait();
+
+
+                bool done = false;
+                // With a positive scale every tile takes the fast path: masked tiles were pre-masked above,
+                // and the first tile takes its exact row maximum as the reference first.
+                bool use_fast = j > 0 && all_full;
+                if (c > 0.f && !use_fast) {
+                    if (j == 0) {
+                        float mx0[8];
 #pragma unroll
-                    for (int g = 0; g < 7; ++g) {
-                        const int e = 16 + (ch * 7 + g) * 16;
-                        if (e < BN) {
+                        for (int i = 0; i < 8; ++i) mx0[i] = fmaxf(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
+#pragma unroll
+                        for (int e = 16; e < BN; e += 16)
 #pragma unroll
                             for (int i = 0; i < 8; ++i)
-                                mxs[i] = max3(mxs[i], __uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1]));
+                                mx0[i] = max3(mx0[i], __uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1]));
+                        const float mxf = fmaxf(fmaxf(fmaxf(mx0[0], mx0[1]), fmaxf(mx0[2], mx0[3])),
+                                                fmaxf(fmaxf(mx0[4], mx0[5]), fmaxf(mx0[6], mx0[7])));
+                        m = (mxf == -INFINITY) ? 0.f : mxf;
+                    }
+                    use_fast = true;
+                }
+                if (use_fast) {
+                    // ---- fast path: exponentials against the reference maximum of the previous tiles,
+                    // the row maximum of this tile computed on the side.  Valid when no row of the warp
+                    // has grown by more than 2^8; otherwise everything is redone by the general path.
+                    const float mc = m * c;
+                    const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
+                    uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // 8 partial row sums
+                    float mxs[8];
+    #pragma unroll
+                    for (int i = 0; i < 8; ++i) mxs[i] = fmaxf(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
+                    auto exp_chunk = [&](int ch) {
+                        uint32_t pk[16];
+    #pragma unroll
+                        for (int e = 0; e < 32; e += 2) {
+                            const uint64_t s2 = pack_f32x2(__uint_as_float(sr[ch * 32 + e]), __uint_as_float(sr[ch * 32 + e + 1]));
+                            const uint64_t x2 = fma_f32x2(s2, c2, nmc2);
+                            float x0, x1, p0, p1;
+                            unpack_f32x2(x2, x0, x1);
+                            if (((ch * 16 + e / 2) % POLY_DEN) < POLY_NUM) {   // this pair: polynomial on the FMA pipe
+                                ex2_poly_f32x2(pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f)), p0, p1);
+                            } else {                                           // this pair: special-function unit
+                                p0 = ex2_approx(x0);
+                                p1 = ex2_approx(x1);
+                            }
+                            acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(p0, p1));
+                            pk[e / 2] = pack2<DTYPE>(p0, p1);
+                        }
+                        tmem_st_32x32b_x16(tS + ch * 16, pk);   // P overwrites the S columns already in registers
+                    };
+    #pragma unroll
+                    for (int ch = 0; ch < BN / 32 - 1; ++ch) {
+                        exp_chunk(ch);
+                        // a third of the row maximum per chunk, off the critical path of the exponentials
+    #pragma unroll
+                        for (int g = 0; g < 7; ++g) {
+                            const int e = 16 + (ch * 7 + g) * 16;
+                            if (e < BN) {
+    #pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    mxs[i] = max3(mxs[i], __uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1]));
+                            }
                         }
                     }
+                    const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                           fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+                    if (!__any_sync(0xffffffffu, (mx - m) * c > 8.f)) {
+                        tmem_st_wait();
+                        tc_fence_before_sync();
+                        mbar_arrive(bar(B_PFULL + t));          // first three quarters of P are in place
+                        exp_chunk(BN / 32 - 1);
+                        float a0, a1, a2, a3;
+                        unpack_f32x2(add_f32x2(acc[0], acc[1]), a0, a1);
+                        unpack_f32x2(add_f32x2(acc[2], acc[3]), a2, a3);
+                        l += (a0 + a1) + (a2 + a3);
+                        done = true;
+                    }
                 }
-                const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
-                                       fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
-                if (!__any_sync(0xffffffffu, (mx - m) * c > 8.f)) {
-                    tmem_st_wait();
-                    tc_fence_before_sync();
-                    mbar_arrive(bar(B_PFULL + t));          // first three quarters of P are in place
-                    PROF_LAP(2);
-                    exp_chunk(BN / 32 - 1);
-#if ATTN_SUM_MODE == 0
+
+                if (!done) {
+                    // ---- general path: first tile, masked tile, or a row maximum that ran ahead.
+                    // Exact row maximum over the visible keys first, then the exponentials chunk by chunk.
+                    float alpha = 1.f;
+                    {
+                        float mxs[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) mxs[i] = -INFINITY;
+#pragma unroll
+                        for (int ch = 0; ch < BN / 32; ++ch) {
+                            if (chunk_full(ch)) {
+#pragma unroll
+                                for (int e = 0; e < 32; e += 16)
+#pragma unroll
+                                    for (int i = 0; i < 8; ++i)
+                                        mxs[i] = max3(mxs[i], __uint_as_float(sr[ch * 32 + e + 2 * i]),
+                                                      __uint_as_float(sr[ch * 32 + e + 2 * i + 1]));
+                            } else if (!chunk_empty(ch)) {
+#pragma unroll
+                                for (int e = 0; e < 32; ++e)
+                                    mxs[e & 7] = fmaxf(mxs[e & 7], (kv0 + ch * 32 + e <= lim) ? __uint_as_float(sr[ch * 32 + e]) : -INFINITY);
+                            }
+                        }
+                        const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                               fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+                        // advance the reference maximum only when the true one ran ahead by more than 2^8
+                        if (j == 0) {
+                            m = (mx == -INFINITY) ? 0.f : mx;
+                        } else if ((mx - m) * c > 8.f) {
+                            alpha = ex2_approx((m - mx) * c);
+                            m = mx;
+                        }
+                    }
+                    // rare: rescale the running O (its last update finished before S_j was produced)
+                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+                        for (int ch = 0; ch < D / 32; ++ch) {
+                            uint32_t orr[32];
+                            tmem_ld_32x32b_x32(tO + ch * 32, orr);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) orr[e] = __float_as_uint(__uint_as_float(orr[e]) * alpha);
+                            tmem_st_32x32b_x32(tO + ch * 32, orr);
+                        }
+                    }
+                    const float mc = m * c;
+                    const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
+                    uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // 8 partial row sums (FULL chunks)
+                    float rs = 0.f;                                // row sum of PARTIAL chunks
+#pragma unroll
+                    for (int ch = 0; ch < BN / 32; ++ch) {
+                        uint32_t pk[16];
+                        if (chunk_full(ch)) {
+#pragma unroll
+                            for (int e = 0; e < 32; e += 2) {
+                                const uint64_t s2 = pack_f32x2(__uint_as_float(sr[ch * 32 + e]), __uint_as_float(sr[ch * 32 + e + 1]));
+                                float x0, x1;
+                                unpack_f32x2(fma_f32x2(s2, c2, nmc2), x0, x1);
+                                const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                                acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(p0, p1));
+                                pk[e / 2] = pack2<DTYPE>(p0, p1);
+                            }
+                        } else if (!chunk_empty(ch)) {
+#pragma unroll
+                            for (int e = 0; e < 32; e += 2) {
+                                const int key = kv0 + ch * 32 + e;
+                                const float p0 = (key <= lim) ? ex2_approx(fmaf(__uint_as_float(sr[ch * 32 + e]), c, -mc)) : 0.f;
+                                const float p1 = (key + 1 <= lim) ? ex2_approx(fmaf(__uint_as_float(sr[ch * 32 + e + 1]), c, -mc)) : 0.f;
+                                rs += p0 + p1;
+                                pk[e / 2] = pack2<DTYPE>(p0, p1);
+                            }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) pk[e] = 0u;
+                        }
+                        tmem_st_32x32b_x16(tS + ch * 16, pk);   // P overwrites the S columns already in registers
+                        if (ch == BN / 32 - 2) {
+                            tmem_st_wait();
+                            tc_fence_before_sync();
+                            mbar_arrive(bar(B_PFULL + t));          // first three quarters of P are in place
+                        }
+                    }
                     float a0, a1, a2, a3;
                     unpack_f32x2(add_f32x2(acc[0], acc[1]), a0, a1);
                     unpack_f32x2(add_f32x2(acc[2], acc[3]), a2, a3);
-                    l += (a0 + a1) + (a2 + a3);
-#else
-                    l += ((accs[0] + accs[1]) + (accs[2] + accs[3])) + ((accs[4] + accs[5]) + (accs[6] + accs[7]));
-#endif
-                    done = true;
+                    l = l * alpha + (((a0 + a1) + (a2 + a3)) + rs);
                 }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(bar(B_PFULL2 + t));
+                PLAP(j == 0 ? 2 : (j == n - 1 ? 6 : 4));
             }
+            if (!ok) break;
 
-            if (!done) {
-                // ---- general path: first tile, diagonal / ragged tile, or a row maximum that ran ahead
-                const int lim = !need_mask ? 0x7fffffff
-                                           : ((prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1);  // last visible key
-                float mx = -INFINITY;
-#pragma unroll
-                for (int e = 0; e < BN; ++e) {
-                    const float sv = (kv0 + e <= lim) ? __uint_as_float(sr[e]) : -INFINITY;
-                    sr[e] = __float_as_uint(sv);
-                    mx = fmaxf(mx, sv);
-                }
-                // advance the reference maximum only when the true one ran ahead by more than 2^8
-                float alpha = 1.f;
-                if (j == 0) {
-                    m = (mx == -INFINITY) ? 0.f : mx;
-                } else if ((mx - m) * c > 8.f) {
-                    alpha = ex2_approx((m - mx) * c);
-                    m = mx;
-                }
-                // rescale the running O (its last update finished before S_j was produced)
-                if (__any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll
-                    for (int ch = 0; ch < D / 32; ++ch) {
-                        uint32_t orr[32];
-                        tmem_ld_32x32b_x32(tO + ch * 32, orr);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) orr[e] = __float_as_uint(__uint_as_float(orr[e]) * alpha);
-                        tmem_st_32x32b_x32(tO + ch * 32, orr);
-                    }
-                }
-                const float mc = m * c;
-                float rs = 0.f;
-#pragma unroll
-                for (int ch = 0; ch < BN / 32; ++ch) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const float s0 = __uint_as_float(sr[ch * 32 + e]), s1 = __uint_as_float(sr[ch * 32 + e + 1]);
-                        // masked entries are -inf; keep them 0 also for a zero scale (-inf * 0 = NaN)
-                        const float p0 = (s0 == -INFINITY) ? 0.f : ex2_approx(fmaf(s0, c, -mc));
-                        const float p1 = (s1 == -INFINITY) ? 0.f : ex2_approx(fmaf(s1, c, -mc));
-                        rs += p0 + p1;
-                        pk[e / 2] = pack2<DTYPE>(p0, p1);
-                    }
-                    tmem_st_32x32b_x16(tS + ch * 16, pk);
-                    if (ch == BN / 32 - 2) {
-                        tmem_st_wait();
-                        tc_fence_before_sync();
-                        mbar_arrive(bar(B_PFULL + t));
-                    }
-                }
-                l = l * alpha + rs;
-            }
-            PROF_LAP(3);
-            tmem_st_wait();
-            tc_fence_before_sync();
-            mbar_arrive(bar(B_PFULL2 + t));
-            PROF_STAMP(t == 0 && r == 0 && j == 64, 26);
-            PROF_LAP(4);
-        }
-#ifdef ATTN_TC_PROFILE
-        if (r == ATTN_PROF_ROW) PROF_FLUSH(12 + 6 * t, 6);
-#endif
-
-        // ---- epilogue: O / l and LSE ----
-        if (ok && n > 0) ok = mbar_wait(bar(B_OFINAL + t), 0, abort_flag);
-        if (ok && n > 0) {
+            // ---- epilogue: O / l and LSE ----
+            if (!(ok = mbar_wait(bar(B_OFINAL + t), uses & 1, abort_flag))) break;
             tc_fence_after_sync();
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
-            const int64_t grow = static_cast<int64_t>(bh) * prm.Sq + row;
+            const int64_t grow = static_cast<int64_t>(it.bh) * prm.Sq + row;
             uint4* orow = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow * D * 2);
 #pragma unroll
             for (int ch = 0; ch < D / 32; ++ch) {
                 uint32_t orr[32];
                 tmem_ld_32x32b_x32(tO + ch * 32, orr);
                 tmem_ld_wait();
+                if (ch == D / 32 - 1) {   // O_t is in registers: the next item may overwrite it
+                    tc_fence_before_sync();
+                    mbar_arrive(bar(B_OFREE + t));
+                }
                 if (row < prm.Sq) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
@@ -499,7 +609,13 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 }
             }
             if (row < prm.Sq) prm.lse[grow] = (l > 0.f) ? m * prm.scale + logf(l) : -INFINITY;
+            it_base += n;
+            ++uses;
+            PLAP(7);
         }
+#ifdef ATTN_TC_PROFILE
+        if (t == 1 && r == 0) { for (int i = 0; i < 8; ++i) prm.prof[blockIdx.x * 16 + i] = pacc[i]; prm.prof[blockIdx.x * 16 + 8] = uses; prm.prof[blockIdx.x * 16 + 9] = it_base; }
+#endif
     }
 
     // ---- teardown (also reached after a timed-out wait) ----

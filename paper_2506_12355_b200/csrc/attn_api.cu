@@ -193,9 +193,9 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     const int64_t BH = static_cast<int64_t>(B) * H;
     const int64_t n_pairs = (static_cast<int64_t>(Sq) + 2 * C::BM - 1) / (2 * C::BM);
     if (n_pairs * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mo;
     if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) ||
-        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN))
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) || !make_map(&mo, o, DTYPE, BH, Sq, D, C::BM))
         return ATTN_ERR_CUDA;
     attn_tc::PipeParams prm;
     prm.o = o;
@@ -229,7 +229,7 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     prm.counter = di.counters + (g_launch_seq.fetch_add(1) % kCounterSlots);
     if (cudaMemsetAsync(prm.counter, 0, sizeof(unsigned int), st) != cudaSuccess) return ATTN_ERR_CUDA;
     const unsigned grid = static_cast<unsigned>(prm.n_items < di.sm_count ? prm.n_items : di.sm_count);
-    kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, prm);
+    kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, mo, prm);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 

@@ -36,8 +36,9 @@ struct PipeCfg {
     static constexpr int NBOX = D / 64;
     static constexpr int Q_BYTES = BM * D * 2;
     static constexpr int KV_BYTES = BN * D * 2;
-    static constexpr int NSLOT = (D == 128) ? 5 : 8;     // ring slots (each holds one K or V tile)
-    static constexpr int TILE_BYTES = 2 * Q_BYTES + NSLOT * KV_BYTES;
+    static constexpr int NSLOT = (D == 128) ? 4 : 8;     // ring slots (each holds one K or V tile)
+    static constexpr int OST_BYTES = BM * 128;           // epilogue staging per Q tile: 128 rows x 64 columns
+    static constexpr int TILE_BYTES = 2 * Q_BYTES + NSLOT * KV_BYTES + 2 * OST_BYTES;
     static constexpr int MISC_BYTES = 512;               // barriers, scheduler slots, TMEM slot, abort flag
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
     static constexpr int TMEM_COLS = 512;
@@ -106,7 +107,8 @@ __device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int 
 template <int D, int DTYPE, int POLY_NUM, int POLY_DEN>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                        const __grid_constant__ CUtensorMap tmV, const PipeParams prm) {
+                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                        const PipeParams prm) {
     using C = PipeCfg<D>;
     constexpr int BM = C::BM, BN = C::BN, NBOX = C::NBOX, NSLOT = C::NSLOT;
 
@@ -115,6 +117,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     auto sQ = [&](int t) { return smem_base + t * C::Q_BYTES; };
     auto sKV = [&](int slot) { return smem_base + 2 * C::Q_BYTES + slot * C::KV_BYTES; };
+    auto sOst = [&](int t) { return smem_base + 2 * C::Q_BYTES + NSLOT * C::KV_BYTES + t * C::OST_BYTES; };
 
     // misc area: barriers, then scheduler slots, TMEM base, abort flag
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
@@ -168,6 +171,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         prefetch_tensormap(&tmQ);
         prefetch_tensormap(&tmK);
         prefetch_tensormap(&tmV);
+        prefetch_tensormap(&tmO);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -586,26 +590,35 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             tc_fence_after_sync();
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
             const int64_t grow = static_cast<int64_t>(it.bh) * prm.Sq + row;
-            uint4* orow = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow * D * 2);
+            // O leaves through a swizzled staging tile in shared memory and a TMA store (full-line writes;
+            // rows beyond Sq are clipped by the tensor map), 64 columns at a time.
+            const uint32_t ost = sOst(t);
 #pragma unroll
-            for (int ch = 0; ch < D / 32; ++ch) {
-                uint32_t orr[32];
-                tmem_ld_32x32b_x32(tO + ch * 32, orr);
+            for (int h = 0; h < D / 64; ++h) {
+                uint32_t orr[64];
+                tmem_ld_32x32b_x32(tO + h * 64, orr);
+                tmem_ld_32x32b_x32(tO + h * 64 + 32, orr + 32);
                 tmem_ld_wait();
-                if (ch == D / 32 - 1) {   // O_t is in registers: the next item may overwrite it
+                if (h == D / 64 - 1) {   // O_t is in registers: the next item may overwrite it
                     tc_fence_before_sync();
                     mbar_arrive(bar(B_OFREE + t));
                 }
-                if (row < prm.Sq) {
+                if (r == 0) tma_store_wait_read<0>();          // the previous store has read the staging tile
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint4 w;
-                        w.x = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 0]) * inv, __uint_as_float(orr[g * 8 + 1]) * inv);
-                        w.y = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 2]) * inv, __uint_as_float(orr[g * 8 + 3]) * inv);
-                        w.z = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 4]) * inv, __uint_as_float(orr[g * 8 + 5]) * inv);
-                        w.w = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 6]) * inv, __uint_as_float(orr[g * 8 + 7]) * inv);
-                        orow[ch * 4 + g] = w;
-                    }
+                for (int g = 0; g < 8; ++g) {
+                    const uint32_t w0 = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 0]) * inv, __uint_as_float(orr[g * 8 + 1]) * inv);
+                    const uint32_t w1 = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 2]) * inv, __uint_as_float(orr[g * 8 + 3]) * inv);
+                    const uint32_t w2 = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 4]) * inv, __uint_as_float(orr[g * 8 + 5]) * inv);
+                    const uint32_t w3 = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 6]) * inv, __uint_as_float(orr[g * 8 + 7]) * inv);
+                    const uint32_t dst = ost + r * 128 + ((g ^ (r & 7)) << 4);   // 128-byte swizzle
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+                }
+                fence_proxy_async_smem();
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
+                if (r == 0) {
+                    tma_store_3d(&tmO, ost, h * 64, q0 + t * BM, it.bh);
+                    tma_store_commit();
                 }
             }
             if (row < prm.Sq) prm.lse[grow] = (l > 0.f) ? m * prm.scale + logf(l) : -INFINITY;
@@ -613,6 +626,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             ++uses;
             PLAP(7);
         }
+        if (r == 0) tma_store_wait_all<0>();   // the staging tile must outlive its last store
 #ifdef ATTN_TC_PROFILE
         if (t == 1 && r == 0) { for (int i = 0; i < 8; ++i) prm.prof[blockIdx.x * 16 + i] = pacc[i]; prm.prof[blockIdx.x * 16 + 8] = uses; prm.prof[blockIdx.x * 16 + 9] = it_base; }
 #endif

@@ -87,6 +87,17 @@ int attn_fwd_gqa(const void* q, const void* k, const void* v, void* o, float* ls
                  int Sq, int Sk, int D, float scale, int causal, int dtype, void* stream);
 
 /*
+ * attn_fwd_qkv_dims -- attention whose Q/K head dim differs from its V/O head dim: the MLA head
+ * shape of Section 4.1 / Table 2 (embedding dimension 128 plus RoPE dimension 64 for Q and K,
+ * 128 for V).  q: [B,H,Sq,Dqk], k: [B,Hkv,Sk,Dqk], v: [B,Hkv,Sk,Dv], o: [B,H,Sq,Dv], lse: [B,H,Sq].
+ * Supported: (Dqk, Dv) = (192, 128), and Dqk == Dv in {64, 128, 256} (then identical to
+ * attn_fwd_gqa); anything else returns ATTN_ERR_UNSUPPORTED_HEAD_DIM.  Grouped K/V heads, mask,
+ * scale, errors and asynchrony as for attn_fwd_gqa.
+ */
+int attn_fwd_qkv_dims(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv,
+                      int Sq, int Sk, int Dqk, int Dv, float scale, int causal, int dtype, void* stream);
+
+/*
  * attn_fwd_simt -- same operator, same arguments, same conventions, computed by a plain
  * CUDA-core kernel (one warp per query row, fp32 arithmetic, online softmax).  It is one to
  * two orders of magnitude slower than attn_fwd and exists as an on-device cross-check that

@@ -81,13 +81,24 @@ void oracle_widen(const uint16_t *src, double *dst, int64_t n, int dtype)
 /* q: [D]; k, v: [Sk, D] of the row's (batch, head); s: scratch of Sk doubles.
  * n_vis = number of visible keys (keys 0 .. n_vis-1).  Writes o[D], *lse and,
  * when prowsum != NULL, the sum of the row's probabilities. */
+static void attn_row_dv(const double *q, const double *k, const double *v, double *s, double *o,
+                        double *lse, double *prowsum, int64_t n_vis, int D, int Dv, double scale);
+
 static void attn_row(const double *q, const double *k, const double *v, double *s, double *o,
                      double *lse, double *prowsum, int64_t n_vis, int D, double scale)
+{
+    attn_row_dv(q, k, v, s, o, lse, prowsum, n_vis, D, D, scale);
+}
+
+/* q: [D]; k: [Sk, D]; v: [Sk, Dv] -- Q/K and V may have different head dims (the MLA head shape
+ * of Section 4.1: 192 for Q/K, 128 for V); o: [Dv]. */
+static void attn_row_dv(const double *q, const double *k, const double *v, double *s, double *o,
+                        double *lse, double *prowsum, int64_t n_vis, int D, int Dv, double scale)
 {
     int64_t j;
     int d;
     if (n_vis <= 0) {
-        for (d = 0; d < D; ++d)
+        for (d = 0; d < Dv; ++d)
             o[d] = 0.0;
         *lse = -INFINITY;
         if (prowsum)
@@ -111,14 +122,14 @@ static void attn_row(const double *q, const double *k, const double *v, double *
         l += s[j];
     }
     /* p_j = e_j / l,  o = sum_j p_j v_j */
-    for (d = 0; d < D; ++d)
+    for (d = 0; d < Dv; ++d)
         o[d] = 0.0;
     double psum = 0.0;
     for (j = 0; j < n_vis; ++j) {
         double p = s[j] / l;
         psum += p;
-        for (d = 0; d < D; ++d)
-            o[d] += p * v[j * D + d];
+        for (d = 0; d < Dv; ++d)
+            o[d] += p * v[j * Dv + d];
     }
     *lse = m + log(l);
     if (prowsum)
@@ -189,6 +200,37 @@ int attn_oracle_gqa_f64(const double *q, const double *k, const double *v, doubl
             int64_t kvh = b * Hkv + h / (H / Hkv);
             attn_row(q + r * D, k + kvh * Sk * D, v + kvh * Sk * D, s, o + r * D, lse + r, NULL,
                      visible_keys(i, Sk, causal), D, scale);
+        }
+        free(s);
+    }
+    return failed ? -1 : 0;
+}
+
+/* Grouped-query attention with separate head dims: q, k: D; v, o: Dv. */
+int attn_oracle_gqa_dv_f64(const double *q, const double *k, const double *v, double *o, double *lse,
+                           int B, int H, int Hkv, int Sq, int Sk, int D, int Dv, double scale, int causal)
+{
+    int64_t rows = (int64_t)B * H * Sq;
+    int failed = 0;
+    if (Hkv <= 0 || H % Hkv != 0)
+        return -2;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(Sk > 0 ? Sk : 1));
+        if (!s) {
+#pragma omp atomic write
+            failed = 1;
+        }
+        int64_t r;
+#pragma omp for schedule(dynamic, 16)
+        for (r = 0; r < rows; ++r) {
+            if (!s)
+                continue;
+            int64_t bh = r / Sq, i = r % Sq;
+            int64_t b = bh / H, h = bh % H;
+            int64_t kvh = b * Hkv + h / (H / Hkv);
+            attn_row_dv(q + r * D, k + kvh * Sk * D, v + kvh * Sk * Dv, s, o + r * Dv, lse + r, NULL,
+                        visible_keys(i, Sk, causal), D, Dv, scale);
         }
         free(s);
     }

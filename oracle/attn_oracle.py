@@ -53,6 +53,8 @@ def _load():
                                                                             ctypes.c_int]
         lib.attn_oracle_gqa_f64.restype = ctypes.c_int
         lib.attn_oracle_gqa_f64.argtypes = [dp, dp, dp, dp, dp] + [ctypes.c_int] * 6 + [ctypes.c_double, ctypes.c_int]
+        lib.attn_oracle_gqa_dv_f64.restype = ctypes.c_int
+        lib.attn_oracle_gqa_dv_f64.argtypes = [dp, dp, dp, dp, dp] + [ctypes.c_int] * 7 + [ctypes.c_double, ctypes.c_int]
         lib.oracle_widen.restype = None
         lib.oracle_widen.argtypes = [u16p, dp, ctypes.c_int64, ctypes.c_int]
         lib.oracle_num_threads.restype = ctypes.c_int
@@ -114,6 +116,26 @@ def attention_gqa(q, k, v, scale: float, causal: bool):
     lse = np.empty((B, H, Sq), dtype=np.float64)
     rc = _load().attn_oracle_gqa_f64(_dptr(q), _dptr(k), _dptr(v), _dptr(o), _dptr(lse), B, H, Hkv, Sq, Sk, D,
                                      float(scale), int(bool(causal)))
+    if rc == -2:
+        raise ValueError("H must be a multiple of Hkv")
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return o, lse
+
+
+def attention_gqa_dv(q, k, v, scale: float, causal: bool):
+    """Attention whose V (and O) head dim differs from the Q/K head dim: q [B,H,Sq,D]; k [B,Hkv,Sk,D];
+    v [B,Hkv,Sk,Dv]; returns o [B,H,Sq,Dv], lse [B,H,Sq]."""
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    k = np.ascontiguousarray(k, dtype=np.float64)
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    B, H, Sq, D = q.shape
+    Hkv, Sk, Dv = k.shape[1], k.shape[2], v.shape[3]
+    assert k.shape == (B, Hkv, Sk, D) and v.shape == (B, Hkv, Sk, Dv)
+    o = np.empty((B, H, Sq, Dv), dtype=np.float64)
+    lse = np.empty((B, H, Sq), dtype=np.float64)
+    rc = _load().attn_oracle_gqa_dv_f64(_dptr(q), _dptr(k), _dptr(v), _dptr(o), _dptr(lse), B, H, Hkv, Sq, Sk, D, Dv,
+                                        float(scale), int(bool(causal)))
     if rc == -2:
         raise ValueError("H must be a multiple of Hkv")
     if rc != 0:

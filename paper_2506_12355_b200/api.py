@@ -24,7 +24,7 @@ STATUS_NAMES = {
 }
 
 # every symbol include/attn_fwd.h declares
-EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
+EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_qkv_dims", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
            "attn_fwd_host_static", "attn_fwd_host_static_capacity",
            "attn_query_support", "attn_last_device_status", "attn_status_string"]
 
@@ -57,6 +57,8 @@ def load() -> ctypes.CDLL:
     lib.attn_fwd.argtypes = sig
     lib.attn_fwd_gqa.restype = i
     lib.attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, vp]
+    lib.attn_fwd_qkv_dims.restype = i
+    lib.attn_fwd_qkv_dims.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, vp]
     lib.attn_fwd_simt.restype = i
     lib.attn_fwd_simt.argtypes = sig
     lib.attn_fwd_host.restype = i
@@ -153,6 +155,31 @@ def attn_fwd_gqa(q, k, v, scale: float, causal: bool = False, out=None, lse=None
                                  B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)), dt, _stream_ptr(stream))
     if rc != 0:
         raise AttnError(rc, "attn_fwd_gqa")
+    return out, lse
+
+
+def attn_fwd_qkv_dims(q, k, v, scale: float, causal: bool = False, out=None, lse=None, stream=None):
+    """Attention with separate Q/K and V head dims (the 192/128 MLA head shape): q [B,H,Sq,Dqk],
+    k [B,Hkv,Sk,Dqk], v [B,Hkv,Sk,Dv]; returns o [B,H,Sq,Dv] and lse [B,H,Sq]."""
+    B, H, Sq, Dqk = q.shape
+    Hkv, Sk, Dv = k.shape[1], k.shape[2], v.shape[3]
+    if tuple(k.shape) != (B, Hkv, Sk, Dqk) or tuple(v.shape) != (B, Hkv, Sk, Dv):
+        raise ValueError("k must be [B,Hkv,Sk,Dqk] and v [B,Hkv,Sk,Dv]")
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+        raise ValueError("q, k, v must be contiguous")
+    if not (q.is_cuda and k.is_cuda and v.is_cuda) or not (q.dtype == k.dtype == v.dtype):
+        raise ValueError("q, k, v must be CUDA tensors of one dtype")
+    dt = _dtype_code(q)
+    if out is None:
+        out = torch.empty((B, H, Sq, Dv), dtype=q.dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(q.device):
+        rc = load().attn_fwd_qkv_dims(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                      B, H, Hkv, Sq, Sk, Dqk, Dv, float(scale), int(bool(causal)), dt,
+                                      _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_fwd_qkv_dims")
     return out, lse
 
 

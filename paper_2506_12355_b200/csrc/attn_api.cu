@@ -13,7 +13,7 @@
 #include "../../include/attn_fwd.h"
 #include "attn_simt.cuh"
 #include "attn_tc_basic.cuh"
-#include "attn_tc_d256.cuh"
+#include "attn_tc_qtmem.cuh"
 #include "attn_tc_pipe.cuh"
 
 // Share of the exponentials evaluated by a polynomial on the FMA pipe instead of the special-function
@@ -233,12 +233,12 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
-// Head dim 256: one Q tile per CTA, Q in tensor memory, double-buffered S.
-template <int DTYPE>
-int launch_tc_d256(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                   float scale, int causal, cudaStream_t st) {
-    using C = attn_tc::D256Cfg;
-    auto kern = attn_tc::attn_fwd_tc_d256_kernel<DTYPE>;
+// One Q tile per CTA, Q in tensor memory, double-buffered S: head dim 256 and the 192/128 head shape.
+template <int DQK, int DV, int BN, int DTYPE>
+int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
+                    float scale, int causal, cudaStream_t st) {
+    using C = attn_tc::QTmemCfg<DQK, DV, BN>;
+    auto kern = attn_tc::attn_fwd_tc_qtmem_kernel<DQK, DV, BN, DTYPE>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -249,10 +249,10 @@ int launch_tc_d256(const void* q, const void* k, const void* v, void* o, float* 
     const int64_t n_qtiles = (static_cast<int64_t>(Sq) + C::BM - 1) / C::BM;
     if (n_qtiles * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
     CUtensorMap mk, mv;
-    if (!make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, C::D, C::BN) ||
-        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, C::D, C::BN))
+    if (!make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, DQK, C::BN) ||
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, DV, C::BN))
         return ATTN_ERR_CUDA;
-    attn_tc::D256Params prm;
+    attn_tc::QTmemParams prm;
     prm.q = q;
     prm.o = o;
     prm.lse = lse;
@@ -267,7 +267,7 @@ int launch_tc_d256(const void* q, const void* k, const void* v, void* o, float* 
     prm.BH = static_cast<int>(BH);
     prm.H = H;
     prm.Hkv = Hkv;
-    const int64_t kv_bytes_per_head = 4LL * Sk * C::D;
+    const int64_t kv_bytes_per_head = 2LL * Sk * (DQK + DV);
     int64_t hpg = (48LL << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
     if (hpg < 1) hpg = 1;
     hpg *= H / Hkv;
@@ -307,7 +307,7 @@ int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, i
         if (IMPL == Impl::Simt) return launch_simt<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
         if (IMPL == Impl::TensorCoreBasic)                                                             \
             return launch_tc_basic<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st);     \
-        if (DD == 256) return launch_tc_d256<TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
+        if (DD == 256) return launch_tc_qtmem<256, 256, 64, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
         return launch_tc_pipe<(DD == 256 ? 128 : DD), TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
     }
     ATTN_CASE(64, 0)
@@ -362,6 +362,24 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, i
 int attn_fwd_gqa(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
                  int D, float scale, int causal, int dtype, void* stream) {
     return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, causal, dtype, stream);
+}
+
+int attn_fwd_qkv_dims(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq,
+                      int Sk, int Dqk, int Dv, float scale, int causal, int dtype, void* stream) {
+    if (Dqk == Dv) return attn_fwd_gqa(q, k, v, o, lse, B, H, Hkv, Sq, Sk, Dqk, scale, causal, dtype, stream);
+    if (Dqk != 192 || Dv != 128) return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
+    // validate with a supported single head dim (the checks do not depend on its value)
+    int rc = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, 128, scale, dtype, true);
+    if (rc != ATTN_OK) return rc;
+    if (static_cast<int64_t>(B) * H * Sq == 0) return ATTN_OK;
+    rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (Sk == 0)
+        return fill_empty(o, lse, static_cast<int64_t>(B) * H * Sq * Dv, static_cast<int64_t>(B) * H * Sq, st);
+    if (dtype == ATTN_DTYPE_FP16)
+        return launch_tc_qtmem<192, 128, 128, 0>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st);
+    return launch_tc_qtmem<192, 128, 128, 1>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st);
 }
 
 int attn_fwd_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,

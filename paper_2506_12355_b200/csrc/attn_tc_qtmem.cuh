@@ -1,11 +1,12 @@
-// Warp-specialised tcgen05 attention forward kernel for head dim 256.
+// Warp-specialised tcgen05 attention forward kernel with Q in tensor memory and a double-buffered S:
+// head dim 256, and heads whose Q/K dim differs from their V dim (192/128).
 //
 // With D = 256 the O accumulator of one 128-row Q tile already takes 256 of the 512 tensor-memory
-// columns, so the two-Q-tile scheme of the D <= 128 kernel does not fit.  Instead one CTA owns ONE
-// Q tile and overlaps the tensor core with the softmax through a double-buffered S:
+// columns, so the two-Q-tile scheme of the D <= 128 kernel does not fit.  Here one CTA owns ONE Q
+// tile and overlaps the tensor core with the softmax through two S buffers:
 //
-//   tensor memory:  O [0,256)   Q [256,384)   S buffer 0 [384,448)   S buffer 1 [448,512)
-//   K/V steps of 64 keys:  S_{j+1} = Q K_{j+1}^T is computed while the softmax works on S_j,
+//   tensor memory:  O [0, DV)   Q [DV, DV + DQK/2)   S buffer 0 and 1: the last 2 * BN columns
+//   steps of BN keys:  S_{j+1} = Q K_{j+1}^T is computed while the softmax works on S_j,
 //   then O += P_j V_j; P_j (16-bit) overwrites the first half of its S buffer.
 //
 // Q is the A operand of the first product FROM TENSOR MEMORY (written there once by the softmax
@@ -14,31 +15,36 @@
 //
 //   warps 0-3  softmax group (one thread per row): Q -> tensor memory, S -> P, rare O rescale, epilogue
 //   warp  4    MMA issuer
-//   warp  5    TMA producer: 64-key K and V tiles through a ring of shared-memory slots
+//   warp  5    TMA producer: BN-key K and V tiles through a ring of shared-memory slots
 //
 // Loop structure as in Appendix C, Listings 1-2 of the paper; online softmax with a lazily advanced
-// reference maximum as in the D <= 128 kernel.
+// reference maximum as in the D <= 128 kernel.  The (192, 128) instance is the head shape of the
+// MLA variant of Section 4.1 (128-dim embedding plus 64-dim RoPE part for Q/K, 128-dim V).
 #pragma once
 #include "attn_tc_basic.cuh"
 
 namespace attn_tc {
 
-struct D256Cfg {
-    static constexpr int D = 256;
+template <int DQK, int DV, int BN_>
+struct QTmemCfg {
     static constexpr int BM = 128;
-    static constexpr int BN = 64;                         // keys per step
-    static constexpr int NBOX = D / 64;                   // 64-column boxes per tile row
-    static constexpr int KV_BYTES = BN * D * 2;           // 32 KB: one K or V tile of 64 keys
-    static constexpr int NSLOT = 6;
-    static constexpr int TILE_BYTES = NSLOT * KV_BYTES;
+    static constexpr int BN = BN_;                              // keys per step
+    static constexpr int K_BYTES = BN * DQK * 2;                // one K tile
+    static constexpr int V_BYTES = BN * DV * 2;                 // one V tile
+    static constexpr int SLOT_BYTES = K_BYTES > V_BYTES ? K_BYTES : V_BYTES;
+    static constexpr int NSLOT = (224 * 1024) / SLOT_BYTES > 7 ? 7 : (224 * 1024) / SLOT_BYTES;
+    static constexpr int TILE_BYTES = NSLOT * SLOT_BYTES;
     static constexpr int MISC_BYTES = 512;
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
     static constexpr int THREADS = 192;
-    static constexpr int O_COL = 0, Q_COL = 256, S_COL = 384;  // S buffer b at S_COL + 64 b
+    static constexpr int O_COL = 0, Q_COL = DV, S_COL = 512 - 2 * BN;   // S buffer b at S_COL + BN * b
     static constexpr int TMEM_COLS = 512;
+    static_assert(DV + DQK / 2 <= S_COL, "tensor memory budget");
+    static_assert(DQK % 64 == 0 && DV % 64 == 0 && (BN == 64 || BN == 128), "tile shapes");
+    static_assert(NSLOT >= 4, "K/V ring too shallow");
 };
 
-struct D256Params {
+struct QTmemParams {
     const void* q;
     void* o;
     float* lse;
@@ -52,17 +58,17 @@ struct D256Params {
     int H, Hkv;
 };
 
-template <int DTYPE>
+template <int DQK, int DV, int BN_, int DTYPE>
 __global__ void __launch_bounds__(192, 1)
-attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                        const D256Params prm) {
-    using C = D256Cfg;
-    constexpr int D = C::D, BM = C::BM, BN = C::BN, NBOX = C::NBOX, NSLOT = C::NSLOT;
+attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                         const QTmemParams prm) {
+    using C = QTmemCfg<DQK, DV, BN_>;
+    constexpr int BM = C::BM, BN = C::BN, NSLOT = C::NSLOT;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    auto sKV = [&](int slot) { return smem_base + slot * C::KV_BYTES; };
+    auto sKV = [&](int slot) { return smem_base + slot * C::SLOT_BYTES; };
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
     const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
     enum { B_QREADY = 0, B_SFULL = 1, B_PFULL = 3, B_ODONE = 5, B_KVFULL = 6, B_KVEMPTY = 6 + NSLOT,
@@ -127,41 +133,40 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     if (warp == 5) {
         // =========================== TMA producer ===========================
         const bool leader = elect_one();
-        auto load_kv = [&](const CUtensorMap* map, int item, int j) -> bool {
+        auto load_kv = [&](const CUtensorMap* map, int nbox, int item, int j) -> bool {
             const int slot = item % NSLOT;
             const uint32_t use = item / NSLOT;
             if (!mbar_wait(bar(B_KVEMPTY + slot), (use & 1) ^ 1, abort_flag)) return false;
             if (leader) {
-                mbar_arrive_expect_tx(bar(B_KVFULL + slot), C::KV_BYTES);
-#pragma unroll
-                for (int bx = 0; bx < NBOX; ++bx)
+                mbar_arrive_expect_tx(bar(B_KVFULL + slot), nbox * BN * 128);
+                for (int bx = 0; bx < nbox; ++bx)
                     tma_load_3d(sKV(slot) + bx * BN * 128, map, bar(B_KVFULL + slot), bx * 64, j * BN, kv_bh);
             }
             return true;
         };
-        bool ok = load_kv(&tmK, 0, 0);
+        bool ok = load_kv(&tmK, DQK / 64, 0, 0);
         for (int j = 0; j < n && ok; ++j) {
-            if (j + 1 < n) ok = load_kv(&tmK, k_item(j + 1), j + 1);
-            if (ok) ok = load_kv(&tmV, v_item(j), j);
+            if (j + 1 < n) ok = load_kv(&tmK, DQK / 64, k_item(j + 1), j + 1);
+            if (ok) ok = load_kv(&tmV, DV / 64, v_item(j), j);
         }
     } else if (warp == 4) {
         // =========================== MMA issuer ===========================
         const bool leader = elect_one();
         constexpr uint32_t IDESC_S = make_idesc_f16(BM, BN, DTYPE, 0, 0);   // Q (TMEM) and K both K-major
-        constexpr uint32_t IDESC_O = make_idesc_f16(BM, D, DTYPE, 0, 1);    // P (TMEM) K-major, V MN-major
+        constexpr uint32_t IDESC_O = make_idesc_f16(BM, DV, DTYPE, 0, 1);    // P (TMEM) K-major, V MN-major
         constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
         const uint32_t k_lo0 = smem_desc_lo(sKV(0), 16);
-        const uint32_t v_lo0 = smem_desc_lo(sKV(0), BN * 128);   // 8 KB between the 64-column boxes
+        const uint32_t v_lo0 = smem_desc_lo(sKV(0), BN * 128);   // distance between the 64-column boxes
         auto kv_full_wait = [&](int item) {
             return mbar_wait(bar(B_KVFULL + item % NSLOT), (item / NSLOT) & 1, abort_flag);
         };
-        auto issue_s = [&](int j) {   // S_j = Q K_j^T into buffer j & 1 : 16 instructions of K = 16
+        auto issue_s = [&](int j) {   // S_j = Q K_j^T into buffer j & 1 : DQK/16 instructions of K = 16
             if (leader) {
-                const uint32_t b0 = k_lo0 + (k_item(j) % NSLOT) * (C::KV_BYTES >> 4);
+                const uint32_t b0 = k_lo0 + (k_item(j) % NSLOT) * (C::SLOT_BYTES >> 4);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
+                for (int kk = 0; kk < DQK / 16; ++kk) {
                     const uint32_t off = ((kk >> 2) * BN * 128 + (kk & 3) * 32) >> 4;
-                    mma_f16_ts_lohi(tmem + C::S_COL + (j & 1) * 64, tmem + C::Q_COL + kk * 8, b0 + off, DESC_HI,
+                    mma_f16_ts_lohi(tmem + C::S_COL + (j & 1) * BN, tmem + C::Q_COL + kk * 8, b0 + off, DESC_HI,
                                     IDESC_S, kk > 0);
                 }
                 mma_commit(bar(B_SFULL + (j & 1)));
@@ -183,10 +188,10 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
             if (!(ok = mbar_wait(bar(B_PFULL + (j & 1)), (j >> 1) & 1, abort_flag))) break;
             tc_fence_after_sync();
             if (leader) {
-                const uint32_t b0 = v_lo0 + (v_item(j) % NSLOT) * (C::KV_BYTES >> 4);
+                const uint32_t b0 = v_lo0 + (v_item(j) % NSLOT) * (C::SLOT_BYTES >> 4);
 #pragma unroll
                 for (int kk = 0; kk < BN / 16; ++kk)
-                    mma_f16_ts_lohi(tmem + C::O_COL, tmem + C::S_COL + (j & 1) * 64 + kk * 8, b0 + ((kk * 16 * 128) >> 4),
+                    mma_f16_ts_lohi(tmem + C::O_COL, tmem + C::S_COL + (j & 1) * BN + kk * 8, b0 + ((kk * 16 * 128) >> 4),
                                     DESC_HI, IDESC_O, (j > 0 || kk > 0) ? 1u : 0u);
                 mma_commit(bar(B_KVEMPTY + v_item(j) % NSLOT));
                 mma_commit(bar(B_ODONE));
@@ -196,6 +201,7 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         // =========================== softmax group ===========================
         const int r = tid;                       // row inside the tile
         const int row = q0 + r;
+        const int row_w0 = q0 + warp * 32;       // first row of this warp
         const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
         const uint32_t tO = tmem + C::O_COL + lane_off, tQ = tmem + C::Q_COL + lane_off;
         const float c = prm.scale_log2;
@@ -203,9 +209,9 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
 
         // Q row -> tensor memory (two 16-bit values per column, in memory order)
         {
-            const uint4* qrow = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(prm.q) + grow * D * 2);
+            const uint4* qrow = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(prm.q) + grow * DQK * 2);
 #pragma unroll
-            for (int ch = 0; ch < D / 64; ++ch) {   // 32 columns = 64 elements = 8 x 16 bytes per chunk
+            for (int ch = 0; ch < DQK / 64; ++ch) {   // 32 columns = 64 elements = 8 x 16 bytes per chunk
                 uint32_t w[32];
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
@@ -226,19 +232,66 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         for (int j = 0; j < n; ++j) {
-            const uint32_t tS = tmem + C::S_COL + (j & 1) * 64 + lane_off;
+            const uint32_t tS = tmem + C::S_COL + (j & 1) * BN + lane_off;
             if (!(ok = mbar_wait(bar(B_SFULL + (j & 1)), (j >> 1) & 1, abort_flag))) break;
             tc_fence_after_sync();
+
+            // Visibility of this step's keys, per warp: a chunk of 32 keys is FULL (every row of the warp
+            // sees all of it), EMPTY (no row sees any of it) or PARTIAL.
+            const int kv0 = j * BN;
+            const int lim = (prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1;   // last visible key of this row
+            const int lim_lo = (prm.causal && row_w0 < prm.Sk - 1) ? row_w0 : prm.Sk - 1;
+            const int lim_hi = (prm.causal && row_w0 + 31 < prm.Sk - 1) ? row_w0 + 31 : prm.Sk - 1;
+            auto chunk_full = [&](int ch) { return kv0 + 32 * ch + 31 <= lim_lo; };
+            auto chunk_empty = [&](int ch) { return kv0 + 32 * ch > lim_hi; };
+            const bool all_full = chunk_full(BN / 32 - 1);
+
+            // Masked steps are brought into the form the fast path expects: hidden scores are overwritten
+            // with -inf in tensor memory (their exponential is 0) before the row is loaded.  A zero scale
+            // cannot use -inf (-inf * 0 is NaN) and takes the general path instead.
+            if (c > 0.f && !all_full) {
+#pragma unroll
+                for (int ch = 0; ch < BN / 32; ++ch) {
+                    if (chunk_full(ch)) continue;
+                    uint32_t tmp[32];
+                    if (chunk_empty(ch)) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) tmp[e] = 0xff800000u;   // -inf
+                    } else {
+                        tmem_ld_32x32b_x32(tS + ch * 32, tmp);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (kv0 + ch * 32 + e > lim) tmp[e] = 0xff800000u;
+                    }
+                    tmem_st_32x32b_x32(tS + ch * 32, tmp);
+                }
+                tmem_st_wait();
+            }
             uint32_t sr[BN];
-            tmem_ld_32x32b_x32(tS, sr);
-            tmem_ld_32x32b_x32(tS + 32, sr + 32);
+#pragma unroll
+            for (int ch = 0; ch < BN / 32; ++ch) tmem_ld_32x32b_x32(tS + ch * 32, sr + ch * 32);
             tmem_ld_wait();
 
-            const int kv0 = j * BN;
-            const bool need_mask = (kv0 + BN > prm.Sk) || (prm.causal && kv0 + BN - 1 > q0);
             bool done = false;
-
-            if (j > 0 && !need_mask) {
+            bool use_fast = j > 0 && all_full;
+            if (c > 0.f && !use_fast) {
+                if (j == 0) {   // the first step takes its exact row maximum as the reference
+                    float mx0[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) mx0[i] = fmaxf(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
+#pragma unroll
+                    for (int e = 16; e < BN; e += 16)
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            mx0[i] = max3(mx0[i], __uint_as_float(sr[e + 2 * i]), __uint_as_float(sr[e + 2 * i + 1]));
+                    const float mxf = fmaxf(fmaxf(fmaxf(mx0[0], mx0[1]), fmaxf(mx0[2], mx0[3])),
+                                            fmaxf(fmaxf(mx0[4], mx0[5]), fmaxf(mx0[6], mx0[7])));
+                    m = (mxf == -INFINITY) ? 0.f : mxf;
+                }
+                use_fast = true;
+            }
+            if (use_fast) {
                 // fast path: exponentials against the reference maximum of the earlier steps, this
                 // step's row maximum computed on the side; redone below if a row ran ahead by > 2^8
                 const float mc = m * c;
@@ -265,7 +318,9 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
                 const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
                                        fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
                 if (!__any_sync(0xffffffffu, (mx - m) * c > 8.f)) {
-                    tmem_st_32x32b_x32(tS, pk);   // P overwrites the first half of its S buffer
+#pragma unroll
+                    for (int ch = 0; ch < BN / 64; ++ch)
+                        tmem_st_32x32b_x32(tS + ch * 32, pk + ch * 32);   // P overwrites the first half of its S buffer
                     float a0, a1, a2, a3;
                     unpack_f32x2(add_f32x2(acc[0], acc[1]), a0, a1);
                     unpack_f32x2(add_f32x2(acc[2], acc[3]), a2, a3);
@@ -274,8 +329,7 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
                 }
             }
             if (!done) {
-                // general path: first step, diagonal / ragged step, or a row maximum that ran ahead
-                const int lim = !need_mask ? 0x7fffffff : ((prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1);
+                // general path: a row maximum that ran ahead, or a zero scale
                 float mx = -INFINITY;
 #pragma unroll
                 for (int e = 0; e < BN; ++e) {
@@ -298,7 +352,7 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
                     if (!(ok = mbar_wait(bar(B_ODONE), (j - 1) & 1, abort_flag))) break;
                     tc_fence_after_sync();
 #pragma unroll
-                    for (int ch = 0; ch < D / 32; ++ch) {
+                    for (int ch = 0; ch < DV / 32; ++ch) {
                         uint32_t orr[32];
                         tmem_ld_32x32b_x32(tO + ch * 32, orr);
                         tmem_ld_wait();
@@ -318,7 +372,8 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
                     rs += p0 + p1;
                     pk[e / 2] = pack2<DTYPE>(p0, p1);
                 }
-                tmem_st_32x32b_x32(tS, pk);
+#pragma unroll
+                for (int ch = 0; ch < BN / 64; ++ch) tmem_st_32x32b_x32(tS + ch * 32, pk + ch * 32);
                 l = l * alpha + rs;
             }
             tmem_st_wait();
@@ -331,9 +386,9 @@ attn_fwd_tc_d256_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         if (ok) {
             tc_fence_after_sync();
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
-            uint4* orow = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow * D * 2);
+            uint4* orow = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow * DV * 2);
 #pragma unroll
-            for (int ch = 0; ch < D / 32; ++ch) {
+            for (int ch = 0; ch < DV / 32; ++ch) {
                 uint32_t orr[32];
                 tmem_ld_32x32b_x32(tO + ch * 32, orr);
                 tmem_ld_wait();

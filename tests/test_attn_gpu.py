@@ -258,3 +258,31 @@ def test_gqa_rejects_indivisible_heads():
     with pytest.raises(api.AttnError) as err:
         api.attn_fwd_gqa(q, kv, kv, 0.1, False)
     assert err.value.status == 2
+
+
+# ------------------------------------------------------------------ separate Q/K and V head dims (192 / 128)
+
+@pytest.mark.parametrize("dtype,causal,H,Hkv,Sq,Sk", [(1, True, 4, 4, 300, 300), (0, False, 4, 2, 257, 515),
+                                                      (1, True, 2, 1, 640, 640)])
+def test_qk192_v128_against_oracle(dtype, causal, H, Hkv, Sq, Sk):
+    B = 2
+    q = inputs.randn16((B, H, Sq, 192), 600, dtype)
+    k = inputs.randn16((B, Hkv, Sk, 192), 601, dtype)
+    v = inputs.randn16((B, Hkv, Sk, 128), 602, dtype)
+    dev = torch.device("cuda:0")
+    obuf, o = guarded((B, H, Sq, 128), q.dtype, dev)
+    lbuf, lse = guarded((B, H, Sq), torch.float32, dev)
+    scale = 1.0 / math.sqrt(192)
+    api.attn_fwd_qkv_dims(q.to(dev), k.to(dev), v.to(dev), scale, causal, out=o, lse=lse)
+    assert api.attn_last_device_status() == 0 and guards_intact(obuf) and guards_intact(lbuf)
+    o_ref, lse_ref = orc.attention_gqa_dv(*(orc.widen(inputs.bits(t), dtype) for t in (q, k, v)), scale, causal)
+    assert np.abs(o.cpu().double().numpy() - o_ref).max() <= O_TOL[dtype]
+    assert np.abs(lse.cpu().double().numpy() - lse_ref).max() <= LSE_TOL
+
+
+def test_qkv_dims_rejects_unsupported_pairs():
+    q = torch.zeros(1, 1, 128, 96, dtype=torch.float16, device="cuda:0")
+    v = torch.zeros(1, 1, 128, 64, dtype=torch.float16, device="cuda:0")
+    with pytest.raises(api.AttnError) as err:
+        api.attn_fwd_qkv_dims(q, q, v, 0.1, False)
+    assert err.value.status == 3

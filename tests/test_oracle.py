@@ -292,3 +292,21 @@ def test_gqa_equals_mha_with_repeated_kv_heads(H, Hkv, causal):
 def test_gqa_rejects_indivisible_heads():
     with pytest.raises(ValueError):
         orc.attention_gqa(rand((1, 5, 2, 4), 1), rand((1, 2, 2, 4), 2), rand((1, 2, 2, 4), 3), 1.0, False)
+
+
+# ------------------------------------------------------------------ separate Q/K and V head dims
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_separate_v_dim_equals_zero_padded_v(causal):
+    # O with a narrower V equals the leading columns of plain attention on V padded with zero columns
+    B, H, Hkv, Sq, Sk, D, Dv = 2, 4, 2, 7, 11, 12, 8
+    q, k, v = rand((B, H, Sq, D), 50), rand((B, Hkv, Sk, D), 51), rand((B, Hkv, Sk, Dv), 52)
+    o, lse = orc.attention_gqa_dv(q, k, v, 0.2, causal)
+    vpad = np.concatenate([v, np.zeros((B, Hkv, Sk, D - Dv))], axis=3)
+    o_ref, lse_ref = orc.attention_gqa(q, k, vpad, 0.2, causal)
+    np.testing.assert_array_equal(o, o_ref[..., :Dv])
+    assert np.all(o_ref[..., Dv:] == 0.0)
+    np.testing.assert_array_equal(lse, lse_ref)
+    to = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v),
+                                                          is_causal=causal, scale=0.2, enable_gqa=True)
+    np.testing.assert_allclose(o, to.numpy(), atol=1e-10)

@@ -87,6 +87,29 @@ int attn_fwd_gqa(const void* q, const void* k, const void* v, void* o, float* ls
                  int Sq, int Sk, int D, float scale, int causal, int dtype, void* stream);
 
 /*
+ * attn_fwd_partial -- attention of all queries over ONE SHARD of the keys and values (split-KV
+ * decoding in the manner of FlashDecoding, which the paper cites in its related work, and key/value
+ * sharding across GPUs).  k, v: [B, Hkv, Sk, D] hold the keys with GLOBAL indices
+ * k_offset .. k_offset + Sk - 1; with the causal mask key (k_offset + j) is visible to query i iff
+ * k_offset + j <= i.  o: [B,H,Sq,D] and lse: [B,H,Sq] receive the shard's own normalised result
+ * O_r and LSE_r; rows that see no key of the shard get O_r = 0 and LSE_r = -inf.  k_offset >= 0.
+ * With k_offset == 0 and the whole key range this is attn_fwd_gqa.  Merge shards with attn_combine.
+ */
+int attn_fwd_partial(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv,
+                     int Sq, int Sk, int D, float scale, int causal, int k_offset, int dtype, void* stream);
+
+/*
+ * attn_combine -- merges the partial results of n_parts disjoint K/V shards (1 <= n_parts <= 1024):
+ *     LSE = ln sum_r exp(LSE_r),    O = sum_r exp(LSE_r - LSE) O_r,
+ * the rescaling identity of the online softmax applied across shards.
+ * o_parts: device, [n_parts, B, H, Sq, D] (16-bit, `dtype`), 16-byte aligned; lse_parts: device,
+ * [n_parts, B, H, Sq] fp32; o: [B,H,Sq,D]; lse: [B,H,Sq].  D must be a multiple of 8.  Rows for which
+ * every shard reports -inf give O = 0, LSE = -inf.  Memory-bound; enqueued on `stream`.
+ */
+int attn_combine(const void* o_parts, const float* lse_parts, int n_parts, void* o, float* lse, int B, int H,
+                 int Sq, int D, int dtype, void* stream);
+
+/*
  * attn_fwd_qkv_dims -- attention whose Q/K head dim differs from its V/O head dim: the MLA head
  * shape of Section 4.1 / Table 2 (embedding dimension 128 plus RoPE dimension 64 for Q and K,
  * 128 for V).  q: [B,H,Sq,Dqk], k: [B,Hkv,Sk,Dqk], v: [B,Hkv,Sk,Dv], o: [B,H,Sq,Dv], lse: [B,H,Sq].

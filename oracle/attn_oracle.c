@@ -206,6 +206,78 @@ int attn_oracle_gqa_f64(const double *q, const double *k, const double *v, doubl
     return failed ? -1 : 0;
 }
 
+/* One K/V shard (split-KV decoding / key-value sharding): k, v hold the keys with global indices
+ * k_offset .. k_offset + Sk - 1; with the causal mask key k_offset + j is visible to query i iff
+ * k_offset + j <= i.  Rows that see no key of the shard get O = 0, LSE = -inf. */
+int attn_oracle_shard_f64(const double *q, const double *k, const double *v, double *o, double *lse,
+                          int B, int H, int Hkv, int Sq, int Sk, int D, double scale, int causal,
+                          int k_offset)
+{
+    int64_t rows = (int64_t)B * H * Sq;
+    int failed = 0;
+    if (Hkv <= 0 || H % Hkv != 0)
+        return -2;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(Sk > 0 ? Sk : 1));
+        if (!s) {
+#pragma omp atomic write
+            failed = 1;
+        }
+        int64_t r;
+#pragma omp for schedule(dynamic, 16)
+        for (r = 0; r < rows; ++r) {
+            if (!s)
+                continue;
+            int64_t bh = r / Sq, i = r % Sq;
+            int64_t b = bh / H, h = bh % H;
+            int64_t kvh = b * Hkv + h / (H / Hkv);
+            int64_t n_vis = Sk;
+            if (causal) {
+                n_vis = i + 1 - k_offset;
+                if (n_vis < 0)
+                    n_vis = 0;
+                if (n_vis > Sk)
+                    n_vis = Sk;
+            }
+            attn_row(q + r * D, k + kvh * Sk * D, v + kvh * Sk * D, s, o + r * D, lse + r, NULL, n_vis,
+                     D, scale);
+        }
+        free(s);
+    }
+    return failed ? -1 : 0;
+}
+
+/* Merge of n_parts shard results (definition): LSE = ln sum_r exp(LSE_r), O = sum_r exp(LSE_r - LSE) O_r.
+ * o_parts: [n_parts, rows, D], lse_parts: [n_parts, rows]. */
+void attn_oracle_combine_f64(const double *o_parts, const double *lse_parts, int n_parts, double *o,
+                             double *lse, int64_t rows, int D)
+{
+    int64_t row;
+#pragma omp parallel for schedule(static)
+    for (row = 0; row < rows; ++row) {
+        int r, d;
+        double mx = -INFINITY, sum = 0.0;
+        for (r = 0; r < n_parts; ++r)
+            if (lse_parts[r * rows + row] > mx)
+                mx = lse_parts[r * rows + row];
+        for (d = 0; d < D; ++d)
+            o[row * D + d] = 0.0;
+        if (mx == -INFINITY) {
+            lse[row] = -INFINITY;
+            continue;
+        }
+        for (r = 0; r < n_parts; ++r)
+            sum += exp(lse_parts[r * rows + row] - mx);
+        lse[row] = mx + log(sum);
+        for (r = 0; r < n_parts; ++r) {
+            double w = exp(lse_parts[r * rows + row] - lse[row]);
+            for (d = 0; d < D; ++d)
+                o[row * D + d] += w * o_parts[(r * rows + row) * D + d];
+        }
+    }
+}
+
 /* Grouped-query attention with separate head dims: q, k: D; v, o: Dv. */
 int attn_oracle_gqa_dv_f64(const double *q, const double *k, const double *v, double *o, double *lse,
                            int B, int H, int Hkv, int Sq, int Sk, int D, int Dv, double scale, int causal)

@@ -55,6 +55,10 @@ def _load():
         lib.attn_oracle_gqa_f64.argtypes = [dp, dp, dp, dp, dp] + [ctypes.c_int] * 6 + [ctypes.c_double, ctypes.c_int]
         lib.attn_oracle_gqa_dv_f64.restype = ctypes.c_int
         lib.attn_oracle_gqa_dv_f64.argtypes = [dp, dp, dp, dp, dp] + [ctypes.c_int] * 7 + [ctypes.c_double, ctypes.c_int]
+        lib.attn_oracle_shard_f64.restype = ctypes.c_int
+        lib.attn_oracle_shard_f64.argtypes = [dp, dp, dp, dp, dp] + [ctypes.c_int] * 6 + [ctypes.c_double, ctypes.c_int, ctypes.c_int]
+        lib.attn_oracle_combine_f64.restype = None
+        lib.attn_oracle_combine_f64.argtypes = [dp, dp, ctypes.c_int, dp, dp, ctypes.c_int64, ctypes.c_int]
         lib.oracle_widen.restype = None
         lib.oracle_widen.argtypes = [u16p, dp, ctypes.c_int64, ctypes.c_int]
         lib.oracle_num_threads.restype = ctypes.c_int
@@ -140,6 +144,35 @@ def attention_gqa_dv(q, k, v, scale: float, causal: bool):
         raise ValueError("H must be a multiple of Hkv")
     if rc != 0:
         raise MemoryError("oracle scratch allocation failed")
+    return o, lse
+
+
+def attention_shard(q, k, v, scale: float, causal: bool, k_offset: int):
+    """One K/V shard whose first key has global index k_offset: q [B,H,Sq,D]; k, v [B,Hkv,Sk,D]."""
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    k = np.ascontiguousarray(k, dtype=np.float64)
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    B, H, Sq, D = q.shape
+    Hkv, Sk = k.shape[1], k.shape[2]
+    assert k.shape == (B, Hkv, Sk, D) and v.shape == (B, Hkv, Sk, D)
+    o = np.empty((B, H, Sq, D), dtype=np.float64)
+    lse = np.empty((B, H, Sq), dtype=np.float64)
+    rc = _load().attn_oracle_shard_f64(_dptr(q), _dptr(k), _dptr(v), _dptr(o), _dptr(lse), B, H, Hkv, Sq, Sk, D,
+                                       float(scale), int(bool(causal)), int(k_offset))
+    if rc != 0:
+        raise ValueError("bad head counts" if rc == -2 else "oracle scratch allocation failed")
+    return o, lse
+
+
+def combine(o_parts, lse_parts):
+    """Merge of shard results: o_parts [n, ..., D], lse_parts [n, ...] -> o [..., D], lse [...]."""
+    o_parts = np.ascontiguousarray(o_parts, dtype=np.float64)
+    lse_parts = np.ascontiguousarray(lse_parts, dtype=np.float64)
+    n, D = o_parts.shape[0], o_parts.shape[-1]
+    rows = int(np.prod(lse_parts.shape[1:]))
+    o = np.empty(o_parts.shape[1:], dtype=np.float64)
+    lse = np.empty(lse_parts.shape[1:], dtype=np.float64)
+    _load().attn_oracle_combine_f64(_dptr(o_parts), _dptr(lse_parts), n, _dptr(o), _dptr(lse), rows, D)
     return o, lse
 
 

@@ -24,7 +24,7 @@ STATUS_NAMES = {
 }
 
 # every symbol include/attn_fwd.h declares
-EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_qkv_dims", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
+EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_partial", "attn_combine", "attn_fwd_qkv_dims", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
            "attn_fwd_host_static", "attn_fwd_host_static_capacity",
            "attn_query_support", "attn_last_device_status", "attn_status_string"]
 
@@ -57,6 +57,10 @@ def load() -> ctypes.CDLL:
     lib.attn_fwd.argtypes = sig
     lib.attn_fwd_gqa.restype = i
     lib.attn_fwd_gqa.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, vp]
+    lib.attn_fwd_partial.restype = i
+    lib.attn_fwd_partial.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, i, vp]
+    lib.attn_combine.restype = i
+    lib.attn_combine.argtypes = [vp, vp, i, vp, vp, i, i, i, i, i, vp]
     lib.attn_fwd_qkv_dims.restype = i
     lib.attn_fwd_qkv_dims.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, vp]
     lib.attn_fwd_simt.restype = i
@@ -155,6 +159,51 @@ def attn_fwd_gqa(q, k, v, scale: float, causal: bool = False, out=None, lse=None
                                  B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)), dt, _stream_ptr(stream))
     if rc != 0:
         raise AttnError(rc, "attn_fwd_gqa")
+    return out, lse
+
+
+def attn_fwd_partial(q, k, v, scale: float, causal: bool, k_offset: int, out=None, lse=None, stream=None):
+    """Attention over one K/V shard whose first key has global index k_offset: q [B,H,Sq,D],
+    k, v [B,Hkv,Sk_shard,D].  Returns the shard's normalised O_r and LSE_r (merge with attn_combine)."""
+    B, H, Sq, D = q.shape
+    Hkv, Sk = k.shape[1], k.shape[2]
+    if tuple(k.shape) != (B, Hkv, Sk, D) or tuple(v.shape) != tuple(k.shape):
+        raise ValueError("k, v must be [B,Hkv,Sk,D]")
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+        raise ValueError("q, k, v must be contiguous")
+    if not (q.is_cuda and k.is_cuda and v.is_cuda) or not (q.dtype == k.dtype == v.dtype):
+        raise ValueError("q, k, v must be CUDA tensors of one dtype")
+    dt = _dtype_code(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(q.device):
+        rc = load().attn_fwd_partial(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                     B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)), int(k_offset), dt,
+                                     _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_fwd_partial")
+    return out, lse
+
+
+def attn_combine(o_parts, lse_parts, out=None, lse=None, stream=None):
+    """Merges partial results: o_parts [n,B,H,Sq,D] (16-bit), lse_parts [n,B,H,Sq] (fp32)."""
+    n, B, H, Sq, D = o_parts.shape
+    if tuple(lse_parts.shape) != (n, B, H, Sq) or lse_parts.dtype != torch.float32:
+        raise ValueError("lse_parts must be fp32 [n,B,H,Sq]")
+    if not (o_parts.is_contiguous() and lse_parts.is_contiguous() and o_parts.is_cuda and lse_parts.is_cuda):
+        raise ValueError("o_parts, lse_parts must be contiguous CUDA tensors")
+    dt = _dtype_code(o_parts)
+    if out is None:
+        out = torch.empty((B, H, Sq, D), dtype=o_parts.dtype, device=o_parts.device)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=o_parts.device)
+    with torch.cuda.device(o_parts.device):
+        rc = load().attn_combine(o_parts.data_ptr(), lse_parts.data_ptr(), n, out.data_ptr(), lse.data_ptr(),
+                                 B, H, Sq, D, dt, _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_combine")
     return out, lse
 
 

@@ -11,8 +11,8 @@
 #include <mutex>
 
 #include "../../include/attn_fwd.h"
+#include "attn_combine.cuh"
 #include "attn_simt.cuh"
-#include "attn_tc_basic.cuh"
 #include "attn_tc_qtmem.cuh"
 #include "attn_tc_pipe.cuh"
 
@@ -138,42 +138,6 @@ int fill_empty(void* o, float* lse, int64_t n_o, int64_t n_lse, cudaStream_t st)
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
-template <int D, int DTYPE>
-int launch_tc_basic(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                    float scale, int causal, cudaStream_t st) {
-    using C = attn_tc::BasicCfg<D>;
-    auto kern = attn_tc::attn_fwd_tc_basic_kernel<D, DTYPE>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-    });
-    if (attr_err != cudaSuccess) return ATTN_ERR_CUDA;
-    const int64_t BH = static_cast<int64_t>(B) * H;
-    CUtensorMap mq, mk, mv;
-    if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) ||
-        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN))
-        return ATTN_ERR_CUDA;
-    attn_tc::Params prm;
-    prm.o = o;
-    prm.lse = lse;
-    prm.Sq = Sq;
-    prm.Sk = Sk;
-    prm.scale = scale;
-    prm.scale_log2 = scale * 1.4426950408889634f;
-    prm.causal = causal ? 1 : 0;
-    prm.status = device_status_ptr();
-    if (!prm.status) return ATTN_ERR_CUDA;
-    prm.H = H;
-    prm.Hkv = Hkv;
-    const int64_t q_tiles = (static_cast<int64_t>(Sq) + C::BM - 1) / C::BM;
-    // grid.y is limited to 65535: fold the heads into grid.x when there are more
-    if (BH > 65535) return ATTN_ERR_BAD_SHAPE;
-    dim3 grid(static_cast<unsigned>(q_tiles), static_cast<unsigned>(BH));
-    kern<<<grid, 128, C::SMEM_BYTES, st>>>(mq, mk, mv, prm);
-    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
-}
-
 #ifdef ATTN_TC_PROFILE
 long long* g_prof_buffer = nullptr;  // development builds only
 #endif
@@ -181,7 +145,7 @@ long long* g_prof_buffer = nullptr;  // development builds only
 // Pipelined, warp-specialised kernel (head dims 64 and 128): one CTA per pair of 128-row Q tiles.
 template <int D, int DTYPE>
 int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                   float scale, int causal, cudaStream_t st) {
+                   float scale, int causal, int k_offset, cudaStream_t st) {
     using C = attn_tc::PipeCfg<D>;
     auto kern = attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE, ATTN_POLY_NUM, ATTN_POLY_DEN>;
     static std::once_flag once;
@@ -209,6 +173,7 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     if (!prm.status) return ATTN_ERR_CUDA;
     prm.H = H;
     prm.Hkv = Hkv;
+    prm.k_offset = k_offset;
     prm.n_pairs = static_cast<int>(n_pairs);
     prm.BH = static_cast<int>(BH);
     // walk together as many heads as keep their K and V (2 * Sk * D * 2 bytes each) inside ~48 MB of L2
@@ -236,7 +201,7 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
 // One Q tile per CTA, Q in tensor memory, double-buffered S: head dim 256 and the 192/128 head shape.
 template <int DQK, int DV, int BN, int DTYPE>
 int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                    float scale, int causal, cudaStream_t st) {
+                    float scale, int causal, int k_offset, cudaStream_t st) {
     using C = attn_tc::QTmemCfg<DQK, DV, BN>;
     auto kern = attn_tc::attn_fwd_tc_qtmem_kernel<DQK, DV, BN, DTYPE>;
     static std::once_flag once;
@@ -267,6 +232,7 @@ int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float*
     prm.BH = static_cast<int>(BH);
     prm.H = H;
     prm.Hkv = Hkv;
+    prm.k_offset = k_offset;
     const int64_t kv_bytes_per_head = 2LL * Sk * (DQK + DV);
     int64_t hpg = (48LL << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
     if (hpg < 1) hpg = 1;
@@ -279,23 +245,24 @@ int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float*
 
 template <int D, int DTYPE>
 int launch_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                float scale, int causal, cudaStream_t st) {
+                float scale, int causal, int k_offset, cudaStream_t st) {
     const int64_t BH = static_cast<int64_t>(B) * H;
     if (BH > 65535) return ATTN_ERR_BAD_SHAPE;
     dim3 grid(static_cast<unsigned>((static_cast<int64_t>(Sq) + attn_simt::kWarpsPerBlock - 1) / attn_simt::kWarpsPerBlock),
               static_cast<unsigned>(BH));
     attn_simt::attn_fwd_simt_kernel<D, DTYPE><<<grid, attn_simt::kWarpsPerBlock * 32, 0, st>>>(q, k, v, o, lse, Sq, Sk,
-                                                                                              scale, causal ? 1 : 0, H, Hkv);
+                                                                                              scale, causal ? 1 : 0, H, Hkv, k_offset);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
-enum class Impl { TensorCore, TensorCoreBasic, Simt };
+enum class Impl { TensorCore, Simt };
 
 template <Impl IMPL>
 int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk, int D,
-             float scale, int causal, int dtype, void* stream) {
+             float scale, int causal, int k_offset, int dtype, void* stream) {
     int rc = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, dtype, true);
     if (rc != ATTN_OK) return rc;
+    if (k_offset < 0 || static_cast<int64_t>(k_offset) + Sk > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
     if (static_cast<int64_t>(B) * H * Sq == 0) return ATTN_OK;
     rc = check_arch();
     if (rc != ATTN_OK) return rc;
@@ -304,11 +271,9 @@ int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, i
         return fill_empty(o, lse, static_cast<int64_t>(B) * H * Sq * D, static_cast<int64_t>(B) * H * Sq, st);
 #define ATTN_CASE(DD, TT)                                                                              \
     if (D == DD && dtype == TT) {                                                                      \
-        if (IMPL == Impl::Simt) return launch_simt<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
-        if (IMPL == Impl::TensorCoreBasic)                                                             \
-            return launch_tc_basic<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st);     \
-        if (DD == 256) return launch_tc_qtmem<256, 256, 64, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
-        return launch_tc_pipe<(DD == 256 ? 128 : DD), TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st); \
+        if (IMPL == Impl::Simt) return launch_simt<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, k_offset, st); \
+        if (DD == 256) return launch_tc_qtmem<256, 256, 64, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, k_offset, st); \
+        return launch_tc_pipe<(DD == 256 ? 128 : DD), TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, k_offset, st); \
     }
     ATTN_CASE(64, 0)
     ATTN_CASE(64, 1)
@@ -356,12 +321,43 @@ void attn_debug_set_profile_buffer(long long* p) { g_prof_buffer = p; }
 
 int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk, int D,
              float scale, int causal, int dtype, void* stream) {
-    return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, H, Sq, Sk, D, scale, causal, dtype, stream);
+    return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, H, Sq, Sk, D, scale, causal, 0, dtype, stream);
 }
 
 int attn_fwd_gqa(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
                  int D, float scale, int causal, int dtype, void* stream) {
-    return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, causal, dtype, stream);
+    return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, causal, 0, dtype, stream);
+}
+
+int attn_fwd_partial(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq,
+                     int Sk, int D, float scale, int causal, int k_offset, int dtype, void* stream) {
+    return dispatch<Impl::TensorCore>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, causal, k_offset, dtype, stream);
+}
+
+int attn_combine(const void* o_parts, const float* lse_parts, int n_parts, void* o, float* lse, int B, int H, int Sq,
+                 int D, int dtype, void* stream) {
+    if (B < 0 || H < 0 || Sq < 0 || n_parts < 1 || n_parts > 1024) return ATTN_ERR_BAD_SHAPE;
+    if (D <= 0 || D % 8 != 0) return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
+    if (dtype != ATTN_DTYPE_FP16 && dtype != ATTN_DTYPE_BF16) return ATTN_ERR_UNSUPPORTED_DTYPE;
+    const int64_t rows = static_cast<int64_t>(B) * H * Sq;
+    if (rows == 0) return ATTN_OK;
+    if (!o_parts || !lse_parts || !o || !lse) return ATTN_ERR_NULL_POINTER;
+    if ((reinterpret_cast<uintptr_t>(o_parts) | reinterpret_cast<uintptr_t>(o)) & 15u) return ATTN_ERR_MISALIGNED;
+    if ((reinterpret_cast<uintptr_t>(lse_parts) | reinterpret_cast<uintptr_t>(lse)) & 3u) return ATTN_ERR_MISALIGNED;
+    int rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+    const int segs = D / 8;
+    const int64_t total = rows * segs;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == ATTN_DTYPE_FP16)
+        attn_merge::attn_combine_kernel<0><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+            static_cast<const uint4*>(o_parts), lse_parts, n_parts, static_cast<uint4*>(o), lse, rows, segs);
+    else
+        attn_merge::attn_combine_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+            static_cast<const uint4*>(o_parts), lse_parts, n_parts, static_cast<uint4*>(o), lse, rows, segs);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
 int attn_fwd_qkv_dims(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq,
@@ -378,13 +374,13 @@ int attn_fwd_qkv_dims(const void* q, const void* k, const void* v, void* o, floa
     if (Sk == 0)
         return fill_empty(o, lse, static_cast<int64_t>(B) * H * Sq * Dv, static_cast<int64_t>(B) * H * Sq, st);
     if (dtype == ATTN_DTYPE_FP16)
-        return launch_tc_qtmem<192, 128, 128, 0>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st);
-    return launch_tc_qtmem<192, 128, 128, 1>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, st);
+        return launch_tc_qtmem<192, 128, 128, 0>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, 0, st);
+    return launch_tc_qtmem<192, 128, 128, 1>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, 0, st);
 }
 
 int attn_fwd_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,
                   int D, float scale, int causal, int dtype, void* stream) {
-    return dispatch<Impl::Simt>(q, k, v, o, lse, B, H, H, Sq, Sk, D, scale, causal, dtype, stream);
+    return dispatch<Impl::Simt>(q, k, v, o, lse, B, H, H, Sq, Sk, D, scale, causal, 0, dtype, stream);
 }
 
 size_t attn_fwd_host_workspace_bytes(int B, int H, int Sq, int Sk, int D) {

@@ -1,0 +1,81 @@
+// Merge of partial attention results computed over disjoint K/V shards.
+//
+// For every query row, shard r delivers a normalised O_r and LSE_r = ln(sum of exponentials over the
+// shard's visible keys).  Softmax over the union of the shards is then exactly
+//     LSE = ln sum_r exp(LSE_r),      O = sum_r exp(LSE_r - LSE) * O_r,
+// the same rescaling identity the online softmax of the attention kernels applies tile by tile.
+// Shards in which a row sees no key carry LSE_r = -inf and drop out.  Memory-bound elementwise work.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+namespace attn_merge {
+
+template <int DTYPE>
+__device__ __forceinline__ void unpack8(const uint4& w, float* f) {
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if constexpr (DTYPE == 0) {
+            const __half2 h = *reinterpret_cast<const __half2*>(&u[i]);
+            f[2 * i] = __low2float(h);
+            f[2 * i + 1] = __high2float(h);
+        } else {
+            const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&u[i]);
+            f[2 * i] = __low2float(h);
+            f[2 * i + 1] = __high2float(h);
+        }
+    }
+}
+
+template <int DTYPE>
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    if constexpr (DTYPE == 0) {
+        __half2 h = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&h);
+    } else {
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&h);
+    }
+}
+
+// o_parts: [n_parts, rows, D] 16-bit; lse_parts: [n_parts, rows] fp32; o: [rows, D]; lse: [rows].
+// One thread per 8 consecutive output elements (16 bytes).
+template <int DTYPE>
+__global__ void __launch_bounds__(256)
+attn_combine_kernel(const uint4* __restrict__ o_parts, const float* __restrict__ lse_parts, int n_parts,
+                    uint4* __restrict__ o, float* __restrict__ lse, int64_t rows, int segs_per_row) {
+    const int64_t total = rows * segs_per_row;
+    for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
+         idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t row = idx / segs_per_row;
+        const int seg = static_cast<int>(idx - row * segs_per_row);
+        float mx = -INFINITY;
+        for (int r = 0; r < n_parts; ++r) mx = fmaxf(mx, lse_parts[r * rows + row]);
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        float total_lse = -INFINITY;
+        if (mx != -INFINITY) {
+            float sum = 0.f;
+            for (int r = 0; r < n_parts; ++r) sum += expf(lse_parts[r * rows + row] - mx);
+            total_lse = mx + logf(sum);
+            for (int r = 0; r < n_parts; ++r) {
+                const float w = expf(lse_parts[r * rows + row] - total_lse);
+                if (w == 0.f) continue;
+                float f[8];
+                unpack8<DTYPE>(o_parts[(r * rows + row) * segs_per_row + seg], f);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, f[i], acc[i]);
+            }
+        }
+        uint4 w;
+        w.x = pack2<DTYPE>(acc[0], acc[1]);
+        w.y = pack2<DTYPE>(acc[2], acc[3]);
+        w.z = pack2<DTYPE>(acc[4], acc[5]);
+        w.w = pack2<DTYPE>(acc[6], acc[7]);
+        o[row * segs_per_row + seg] = w;
+        if (seg == 0) lse[row] = total_lse;
+    }
+}
+
+}  // namespace attn_merge

@@ -31,7 +31,7 @@ template <int D, int DTYPE>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 attn_fwd_simt_kernel(const void* __restrict__ q, const void* __restrict__ k,
                      const void* __restrict__ v, void* __restrict__ o, float* __restrict__ lse,
-                     int Sq, int Sk, float scale, int causal, int H, int Hkv) {
+                     int Sq, int Sk, float scale, int causal, int H, int Hkv, int k_offset) {
     constexpr int CPL = D / 32;  // output columns per lane
     __shared__ float qs[kWarpsPerBlock][D];
 
@@ -46,7 +46,13 @@ attn_fwd_simt_kernel(const void* __restrict__ q, const void* __restrict__ k,
     for (int d = lane; d < D; d += 32) qs[warp][d] = load16<DTYPE>(q, qrow + d);
     __syncwarp();
 
-    const int64_t n_vis = causal ? (i + 1 < Sk ? i + 1 : Sk) : Sk;
+    // visible keys: all, or (causal) those with k_offset + j <= i
+    int64_t n_vis = Sk;
+    if (causal) {
+        n_vis = i + 1 - k_offset;
+        if (n_vis < 0) n_vis = 0;
+        if (n_vis > Sk) n_vis = Sk;
+    }
     float m = -INFINITY, l = 0.f;
     float acc[CPL];
 #pragma unroll

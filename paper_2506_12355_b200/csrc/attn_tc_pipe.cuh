@@ -25,7 +25,7 @@
 // grown by more than 2^8; otherwise the stale m is kept (P values up to 256, exact after the final
 // division by l), so the O accumulator rarely needs rescaling.
 #pragma once
-#include "attn_tc_basic.cuh"
+#include "attn_tc_common.cuh"
 
 namespace attn_tc {
 
@@ -58,6 +58,7 @@ struct PipeParams {
     int BH;                 // batch * query heads
     int heads_per_group;    // heads whose K/V are walked together (L2 residency)
     int H, Hkv;             // query heads and key/value heads per batch element (H % Hkv == 0)
+    int k_offset;           // global index of key 0 of this K/V shard (0 for whole problems); enters the causal mask
     int n_items;            // n_pairs * BH
     unsigned int* counter;  // work counter, zero at launch: item = gridDim.x + atomicAdd(counter, 1)
 #ifdef ATTN_TC_PROFILE
@@ -73,7 +74,7 @@ __device__ __forceinline__ void reg_dec_service() { asm volatile("setmaxnreg.dec
 // One work item, decoded identically by every role.
 struct PipeItem {
     int bh, kv_bh, q0;
-    int n_kv[2];   // K/V tiles each Q tile needs (0: tile beyond Sq)
+    int n_kv[2];   // K/V tiles each Q tile needs (0: tile beyond Sq, or no visible key)
     int n_max;
 };
 
@@ -95,9 +96,8 @@ __device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int 
         if (qs >= prm.Sq) {
             it.n_kv[t] = 0;
         } else {
-            int last_key = prm.Sk - 1;
-            if (prm.causal && qs + BM - 1 < last_key) last_key = qs + BM - 1;
-            it.n_kv[t] = last_key / BN + 1;
+            const int last_key = last_visible_key(qs + BM - 1, prm.Sk, prm.causal, prm.k_offset);
+            it.n_kv[t] = last_key < 0 ? 0 : last_key / BN + 1;   // 0: no row of the tile sees a key of this shard
         }
     }
     it.n_max = it.n_kv[0] > it.n_kv[1] ? it.n_kv[0] : it.n_kv[1];
@@ -289,7 +289,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (item < 0) break;
                 const PipeItem it = pipe_decode_item(prm, item, BM, BN);
                 // ---- first S of both tiles ----
-                ok = kv_full_wait(kv_base);
+                if (it.n_max > 0) ok = kv_full_wait(kv_base);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (ok && it.n_kv[t] > 0) {
@@ -364,9 +364,19 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             if (item < 0) break;
             const PipeItem it = pipe_decode_item(prm, item, BM, BN);
             const int n = it.n_kv[t];
-            if (n == 0) continue;
             const int q0 = it.q0;
             const int row = q0 + t * BM + r;
+            if (n == 0) {
+                // beyond Sq, or (K/V shards under the causal mask) rows that see no key: O = 0, LSE = -inf
+                if (row < prm.Sq) {
+                    const int64_t grow0 = static_cast<int64_t>(it.bh) * prm.Sq + row;
+                    uint4* orow0 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow0 * D * 2);
+#pragma unroll
+                    for (int g = 0; g < D / 8; ++g) orow0[g] = make_uint4(0u, 0u, 0u, 0u);
+                    prm.lse[grow0] = -INFINITY;
+                }
+                continue;
+            }
             const int row_w0 = q0 + t * BM + (warp & 3) * 32;   // first row of this warp
             float m = -INFINITY, l = 0.f;
 
@@ -377,9 +387,9 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 // Visibility of this K/V tile, per warp (rows 32 w .. 32 w + 31 of the Q tile): a chunk of
                 // 32 keys is FULL (every row sees all of it), EMPTY (no row sees any of it) or PARTIAL.
                 const int kv0 = j * BN;
-                const int lim = (prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1;   // last visible key of this row
-                const int lim_lo = (prm.causal && row_w0 < prm.Sk - 1) ? row_w0 : prm.Sk - 1;
-                const int lim_hi = (prm.causal && row_w0 + 31 < prm.Sk - 1) ? row_w0 + 31 : prm.Sk - 1;
+                const int lim = last_visible_key(row, prm.Sk, prm.causal, prm.k_offset);   // of this row
+                const int lim_lo = last_visible_key(row_w0, prm.Sk, prm.causal, prm.k_offset);
+                const int lim_hi = last_visible_key(row_w0 + 31, prm.Sk, prm.causal, prm.k_offset);
                 auto chunk_full = [&](int ch) { return kv0 + 32 * ch + 31 <= lim_lo; };
                 auto chunk_empty = [&](int ch) { return kv0 + 32 * ch > lim_hi; };
                 const bool all_full = chunk_full(BN / 32 - 1);
@@ -588,7 +598,11 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             // ---- epilogue: O / l and LSE ----
             if (!(ok = mbar_wait(bar(B_OFINAL + t), uses & 1, abort_flag))) break;
             tc_fence_after_sync();
-            const float inv = (l > 0.f) ? 1.f / l : 0.f;
+            // A row that saw at least one key has l >= 2^-8 (its maximum contributed 1 when it was taken as the
+            // reference).  Rows that saw none (possible for K/V shards under the causal mask) only collected
+            // the 2^-126 floor of the polynomial exponential: they give O = 0, LSE = -inf.
+            const bool seen = l > 1e-30f;
+            const float inv = seen ? 1.f / l : 0.f;
             const int64_t grow = static_cast<int64_t>(it.bh) * prm.Sq + row;
             // O leaves through a swizzled staging tile in shared memory and a TMA store (full-line writes;
             // rows beyond Sq are clipped by the tensor map), 64 columns at a time.
@@ -621,7 +635,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     tma_store_commit();
                 }
             }
-            if (row < prm.Sq) prm.lse[grow] = (l > 0.f) ? m * prm.scale + logf(l) : -INFINITY;
+            if (row < prm.Sq) prm.lse[grow] = seen ? m * prm.scale + logf(l) : -INFINITY;
             it_base += n;
             ++uses;
             PLAP(7);

@@ -21,7 +21,7 @@
 // reference maximum as in the D <= 128 kernel.  The (192, 128) instance is the head shape of the
 // MLA variant of Section 4.1 (128-dim embedding plus 64-dim RoPE part for Q/K, 128-dim V).
 #pragma once
-#include "attn_tc_basic.cuh"
+#include "attn_tc_common.cuh"
 
 namespace attn_tc {
 
@@ -56,6 +56,7 @@ struct QTmemParams {
     int BH;
     int heads_per_group;
     int H, Hkv;
+    int k_offset;         // global index of key 0 of this K/V shard; enters the causal mask
 };
 
 template <int DQK, int DV, int BN_, int DTYPE>
@@ -93,9 +94,8 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     }
     const int q0 = qt * BM;
     const int kv_bh = (bh / prm.H) * prm.Hkv + (bh % prm.H) / (prm.H / prm.Hkv);
-    int last_key = prm.Sk - 1;
-    if (prm.causal && q0 + BM - 1 < last_key) last_key = q0 + BM - 1;
-    const int n = last_key / BN + 1;   // K/V steps
+    const int last_key = last_visible_key(q0 + BM - 1, prm.Sk, prm.causal, prm.k_offset);
+    const int n = last_key < 0 ? 0 : last_key / BN + 1;   // K/V steps (0: no row of the tile sees a key of this shard)
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -144,7 +144,7 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
             }
             return true;
         };
-        bool ok = load_kv(&tmK, DQK / 64, 0, 0);
+        bool ok = n > 0 && load_kv(&tmK, DQK / 64, 0, 0);
         for (int j = 0; j < n && ok; ++j) {
             if (j + 1 < n) ok = load_kv(&tmK, DQK / 64, k_item(j + 1), j + 1);
             if (ok) ok = load_kv(&tmV, DV / 64, v_item(j), j);
@@ -173,7 +173,7 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
                 mma_commit(bar(B_KVEMPTY + k_item(j) % NSLOT));
             }
         };
-        bool ok = mbar_wait(bar(B_QREADY), 0, abort_flag) && kv_full_wait(0);
+        bool ok = n > 0 && mbar_wait(bar(B_QREADY), 0, abort_flag) && kv_full_wait(0);
         if (ok) {
             tc_fence_after_sync();
             issue_s(0);
@@ -207,8 +207,17 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         const float c = prm.scale_log2;
         const int64_t grow = static_cast<int64_t>(bh) * prm.Sq + row;
 
+        if (n == 0) {
+            // (K/V shards under the causal mask) no row of this tile sees a key: O = 0, LSE = -inf
+            if (row < prm.Sq) {
+                uint4* orow0 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow * DV * 2);
+#pragma unroll
+                for (int g = 0; g < DV / 8; ++g) orow0[g] = make_uint4(0u, 0u, 0u, 0u);
+                prm.lse[grow] = -INFINITY;
+            }
+        }
         // Q row -> tensor memory (two 16-bit values per column, in memory order)
-        {
+        if (n > 0) {
             const uint4* qrow = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(prm.q) + grow * DQK * 2);
 #pragma unroll
             for (int ch = 0; ch < DQK / 64; ++ch) {   // 32 columns = 64 elements = 8 x 16 bytes per chunk
@@ -239,9 +248,9 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
             // Visibility of this step's keys, per warp: a chunk of 32 keys is FULL (every row of the warp
             // sees all of it), EMPTY (no row sees any of it) or PARTIAL.
             const int kv0 = j * BN;
-            const int lim = (prm.causal && row < prm.Sk - 1) ? row : prm.Sk - 1;   // last visible key of this row
-            const int lim_lo = (prm.causal && row_w0 < prm.Sk - 1) ? row_w0 : prm.Sk - 1;
-            const int lim_hi = (prm.causal && row_w0 + 31 < prm.Sk - 1) ? row_w0 + 31 : prm.Sk - 1;
+            const int lim = last_visible_key(row, prm.Sk, prm.causal, prm.k_offset);   // of this row
+            const int lim_lo = last_visible_key(row_w0, prm.Sk, prm.causal, prm.k_offset);
+            const int lim_hi = last_visible_key(row_w0 + 31, prm.Sk, prm.causal, prm.k_offset);
             auto chunk_full = [&](int ch) { return kv0 + 32 * ch + 31 <= lim_lo; };
             auto chunk_empty = [&](int ch) { return kv0 + 32 * ch > lim_hi; };
             const bool all_full = chunk_full(BN / 32 - 1);
@@ -382,8 +391,8 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         }
 
         // ---- epilogue: O / l and LSE ----
-        if (ok) ok = mbar_wait(bar(B_ODONE), (n - 1) & 1, abort_flag);
-        if (ok) {
+        if (ok && n > 0) ok = mbar_wait(bar(B_ODONE), (n - 1) & 1, abort_flag);
+        if (ok && n > 0) {
             tc_fence_after_sync();
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
             uint4* orow = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow * DV * 2);

@@ -286,3 +286,55 @@ def test_qkv_dims_rejects_unsupported_pairs():
     with pytest.raises(api.AttnError) as err:
         api.attn_fwd_qkv_dims(q, q, v, 0.1, False)
     assert err.value.status == 3
+
+
+# ------------------------------------------------------------------ K/V shards (partial results) and their merge
+
+@pytest.mark.parametrize("D,dtype,causal,Hkv", [(128, 1, True, 2), (64, 0, False, 4), (256, 1, True, 4), (128, 0, True, 1)])
+def test_kv_shards_and_combine_against_oracle(D, dtype, causal, Hkv):
+    B, H, Sq, Sk = 1, 4, 600, 700
+    q = inputs.randn16((B, H, Sq, D), 700, dtype)
+    k = inputs.randn16((B, Hkv, Sk, D), 701, dtype)
+    v = inputs.randn16((B, Hkv, Sk, D), 702, dtype)
+    dev = torch.device("cuda:0")
+    qd = q.to(dev)
+    scale = 1.0 / math.sqrt(D)
+    cuts = [0, 130, 384, Sk]        # uneven shards, one boundary off the tile grid
+    n = len(cuts) - 1
+    o_parts = torch.full((n, B, H, Sq, D), float("nan"), dtype=q.dtype, device=dev)
+    l_parts = torch.full((n, B, H, Sq), float("nan"), dtype=torch.float32, device=dev)
+    qf, kf, vf = (orc.widen(inputs.bits(t), dtype) for t in (q, k, v))
+    for r, (a, b) in enumerate(zip(cuts, cuts[1:])):
+        api.attn_fwd_partial(qd, k[:, :, a:b].contiguous().to(dev), v[:, :, a:b].contiguous().to(dev), scale, causal, a,
+                             out=o_parts[r], lse=l_parts[r])
+        # each shard on its own against the oracle's shard entry
+        o_ref_r, l_ref_r = orc.attention_shard(qf, kf[:, :, a:b], vf[:, :, a:b], scale, causal, a)
+        got_l = l_parts[r].cpu().double().numpy()
+        assert np.array_equal(np.isneginf(got_l), np.isneginf(l_ref_r))
+        fin = ~np.isneginf(l_ref_r)
+        assert np.abs(got_l[fin] - l_ref_r[fin]).max() <= LSE_TOL
+        assert np.abs(o_parts[r].cpu().double().numpy() - o_ref_r).max() <= O_TOL[dtype]
+    assert api.attn_last_device_status() == 0
+    o, lse = api.attn_combine(o_parts, l_parts)
+    torch.cuda.synchronize()
+    o_ref, lse_ref = orc.attention_gqa(qf, kf, vf, scale, causal)
+    assert np.abs(o.cpu().double().numpy() - o_ref).max() <= O_TOL[dtype]
+    assert np.abs(lse.cpu().double().numpy() - lse_ref).max() <= LSE_TOL
+
+
+def test_combine_of_all_empty_rows():
+    dev = torch.device("cuda:0")
+    o_parts = torch.randn(3, 1, 2, 40, 64, device=dev).to(torch.float16)
+    l_parts = torch.full((3, 1, 2, 40), float("-inf"), dtype=torch.float32, device=dev)
+    o, lse = api.attn_combine(o_parts, l_parts)
+    assert float(o.abs().max()) == 0.0 and bool(torch.isneginf(lse).all())
+
+
+def test_kv_sharded_attention_single_rank_reduces_to_plain_attention():
+    from paper_2506_12355_b200 import dist as adist
+    q, k, v = inputs.make_qkv(1, 2, 300, 300, 128, inputs.DTYPE_BF16, seed=77)
+    dev = torch.device("cuda:0")
+    o1, l1 = adist.kv_sharded_attention(q.to(dev), k.to(dev), v.to(dev), 0.1, True, 0)
+    o2, l2 = api.attn_fwd(q.to(dev), k.to(dev), v.to(dev), 0.1, True)
+    torch.cuda.synchronize()
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and float((l1 - l2).abs().max()) <= 1e-5

@@ -70,3 +70,40 @@ def test_two_gloo_ranks_shard_by_heads(tmp_path):
     out = str(tmp_path / "result.txt")
     mp.spawn(_worker, args=(2, _free_port(), out), nprocs=2, join=True)
     assert open(out).read() == "ok"
+
+
+def _kv_worker(rank, world, port, out_path):
+    """Key/value sharding on CPU: every rank evaluates its own key slice with the oracle's shard entry
+    (global key offset from shard_keys), the partial (O, LSE) pairs are exchanged, and the merge equals
+    the unsharded result."""
+    from oracle import attn_oracle as orc
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    adist.init("gloo")
+    B, H, Sq, Sk, D = 1, 2, 37, 53, 8
+    q, k, v = inputs.make_qkv(B, H, Sq, Sk, D, inputs.DTYPE_FP16, seed=21)
+    qf, kf, vf = (orc.widen(inputs.bits(t), 0) for t in (q, k, v))
+    b, e = adist.shard_keys(Sk, world, rank)
+    o_r, l_r = orc.attention_shard(qf, kf[:, :, b:e], vf[:, :, b:e], 0.3, True, b)
+    got_o = [torch.zeros(B, H, Sq, D, dtype=torch.float64) for _ in range(world)]
+    got_l = [torch.zeros(B, H, Sq, dtype=torch.float64) for _ in range(world)]
+    dist.all_gather(got_o, torch.from_numpy(o_r))
+    dist.all_gather(got_l, torch.from_numpy(l_r))
+    o, lse = orc.combine(np.stack([t.numpy() for t in got_o]), np.stack([t.numpy() for t in got_l]))
+    o_ref, l_ref = orc.attention(qf, kf, vf, 0.3, True)
+    ok = np.allclose(o, o_ref, atol=1e-12) and np.allclose(lse, l_ref, atol=1e-12)
+    flags = [None] * world
+    dist.all_gather_object(flags, bool(ok))
+    if rank == 0:
+        open(out_path, "w").write("ok" if all(flags) else "mismatch")
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_by_keys_and_merge(tmp_path):
+    out = str(tmp_path / "result_kv.txt")
+    mp.spawn(_kv_worker, args=(2, _free_port(), out), nprocs=2, join=True)
+    assert open(out).read() == "ok"
+
+
+def test_shard_keys_offsets():
+    assert [adist.shard_keys(10, 3, r) for r in range(3)] == [(0, 4), (4, 7), (7, 10)]

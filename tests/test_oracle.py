@@ -310,3 +310,35 @@ def test_separate_v_dim_equals_zero_padded_v(causal):
     to = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v),
                                                           is_causal=causal, scale=0.2, enable_gqa=True)
     np.testing.assert_allclose(o, to.numpy(), atol=1e-10)
+
+
+# ------------------------------------------------------------------ K/V shards and their merge
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_shards_merge_to_the_unsharded_result(causal):
+    # keys cut into three uneven shards; each shard evaluated with its global key offset; the merge
+    # must give the one-shot result (pins the offset convention of the causal mask and the merge)
+    B, H, Hkv, Sq, Sk, D = 1, 4, 2, 23, 31, 8
+    q, k, v = rand((B, H, Sq, D), 60), rand((B, Hkv, Sk, D), 61), rand((B, Hkv, Sk, D), 62)
+    o_ref, lse_ref = orc.attention_gqa(q, k, v, 0.3, causal)
+    cuts = [0, 5, 18, Sk]
+    parts = [orc.attention_shard(q, k[:, :, a:b], v[:, :, a:b], 0.3, causal, a) for a, b in zip(cuts, cuts[1:])]
+    if causal:   # early rows see nothing of the later shards
+        assert np.all(np.isneginf(parts[2][1][:, :, :18])) and np.all(parts[2][0][:, :, :18] == 0.0)
+        assert np.all(np.isfinite(parts[2][1][:, :, 18:]))
+    o, lse = orc.combine(np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]))
+    np.testing.assert_allclose(o, o_ref, atol=1e-12)
+    np.testing.assert_allclose(lse, lse_ref, atol=1e-12)
+    # the merge against numpy's logaddexp written out separately
+    l_np = np.logaddexp.reduce(np.stack([p[1] for p in parts]), axis=0)
+    np.testing.assert_allclose(lse, l_np, atol=1e-12)
+
+
+def test_shard_with_zero_offset_is_plain_attention_and_empty_merge():
+    q, k, v = rand((1, 2, 6, 4), 63), rand((1, 2, 9, 4), 64), rand((1, 2, 9, 4), 65)
+    o, lse = orc.attention_shard(q, k, v, 0.5, True, 0)
+    o_ref, lse_ref = orc.attention(q, k, v, 0.5, True)
+    np.testing.assert_array_equal(o, o_ref)
+    np.testing.assert_array_equal(lse, lse_ref)
+    o2, lse2 = orc.combine(np.zeros((2, 3, 4)), np.full((2, 3), -np.inf))
+    assert np.all(o2 == 0.0) and np.all(np.isneginf(lse2))

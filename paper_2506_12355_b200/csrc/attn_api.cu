@@ -23,6 +23,13 @@
 #define ATTN_POLY_DEN 8
 #endif
 
+#ifndef ATTN_MERGE_LAST
+#define ATTN_MERGE_LAST 3
+#endif
+#ifndef ATTN_L2_MB
+#define ATTN_L2_MB 24
+#endif
+
 namespace {
 
 // Device-side status word: 0, or ATTN_ERR_DEVICE_TIMEOUT once a kernel gave up on a wait.
@@ -176,13 +183,19 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     prm.k_offset = k_offset;
     prm.n_pairs = static_cast<int>(n_pairs);
     prm.BH = static_cast<int>(BH);
-    // walk together as many heads as keep their K and V (2 * Sk * D * 2 bytes each) inside ~48 MB of L2
+    // walk together as many heads as keep their K and V (2 * Sk * D * 2 bytes each) inside ~24 MB of L2 (the L2 is split over two dies)
     const int64_t kv_bytes_per_head = 4LL * Sk * D;
-    int64_t hpg = (48LL << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
+    int64_t hpg = (static_cast<int64_t>(ATTN_L2_MB) << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
     if (hpg < 1) hpg = 1;
     hpg *= H / Hkv;  // the query heads of one K/V head share its footprint
     if (hpg > BH) hpg = BH;
     prm.heads_per_group = static_cast<int>(hpg);
+    // the last three groups are merged into one: its items, ordered longest-first, then end with short ones,
+    // which keeps the tail of the launch short
+    {
+        const int64_t n_groups = (BH + hpg - 1) / hpg;
+        prm.last_group = static_cast<int>(n_groups >= ATTN_MERGE_LAST ? n_groups - ATTN_MERGE_LAST : 0);
+    }
     prm.n_items = static_cast<int>(n_pairs * BH);
 #ifdef ATTN_TC_PROFILE
     prm.prof = g_prof_buffer;
@@ -234,11 +247,17 @@ int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float*
     prm.Hkv = Hkv;
     prm.k_offset = k_offset;
     const int64_t kv_bytes_per_head = 2LL * Sk * (DQK + DV);
-    int64_t hpg = (48LL << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
+    int64_t hpg = (static_cast<int64_t>(ATTN_L2_MB) << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
     if (hpg < 1) hpg = 1;
     hpg *= H / Hkv;
     if (hpg > BH) hpg = BH;
     prm.heads_per_group = static_cast<int>(hpg);
+    // the last three groups are merged into one: its items, ordered longest-first, then end with short ones,
+    // which keeps the tail of the launch short
+    {
+        const int64_t n_groups = (BH + hpg - 1) / hpg;
+        prm.last_group = static_cast<int>(n_groups >= ATTN_MERGE_LAST ? n_groups - ATTN_MERGE_LAST : 0);
+    }
     kern<<<static_cast<unsigned>(n_qtiles * BH), C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, prm);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }

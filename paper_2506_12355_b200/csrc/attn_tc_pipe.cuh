@@ -57,6 +57,7 @@ struct PipeParams {
     int n_pairs;            // 256-row Q tile pairs per head
     int BH;                 // batch * query heads
     int heads_per_group;    // heads whose K/V are walked together (L2 residency)
+    int last_group;         // index of the final group, which takes all remaining heads
     int H, Hkv;             // query heads and key/value heads per batch element (H % Hkv == 0)
     int k_offset;           // global index of key 0 of this K/V shard (0 for whole problems); enters the causal mask
     int n_items;            // n_pairs * BH
@@ -81,9 +82,10 @@ struct PipeItem {
 __device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int lin, int BM, int BN) {
     PipeItem it;
     const int full_group = prm.heads_per_group * prm.n_pairs;
-    const int g = lin / full_group, r = lin - g * full_group;
-    int hg = prm.BH - g * prm.heads_per_group;
-    if (hg > prm.heads_per_group) hg = prm.heads_per_group;
+    int g = lin / full_group;
+    if (g > prm.last_group) g = prm.last_group;
+    const int r = lin - g * full_group;
+    const int hg = (g == prm.last_group) ? prm.BH - g * prm.heads_per_group : prm.heads_per_group;
     const int pr = r / hg;
     it.bh = g * prm.heads_per_group + (r - pr * hg);
     const int pair = prm.causal ? prm.n_pairs - 1 - pr : pr;   // causal: longest rows first

@@ -55,6 +55,7 @@ struct QTmemParams {
     int n_qtiles;         // 128-row Q tiles per head
     int BH;
     int heads_per_group;
+    int last_group;       // index of the final group, which takes all remaining heads
     int H, Hkv;
     int k_offset;         // global index of key 0 of this K/V shard; enters the causal mask
 };
@@ -85,9 +86,10 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     {
         const int lin = blockIdx.x;
         const int full_group = prm.heads_per_group * prm.n_qtiles;
-        const int g = lin / full_group, r = lin - g * full_group;
-        int hg = prm.BH - g * prm.heads_per_group;
-        if (hg > prm.heads_per_group) hg = prm.heads_per_group;
+        int g = lin / full_group;
+        if (g > prm.last_group) g = prm.last_group;
+        const int r = lin - g * full_group;
+        const int hg = (g == prm.last_group) ? prm.BH - g * prm.heads_per_group : prm.heads_per_group;
         const int pr = r / hg;
         bh = g * prm.heads_per_group + (r - pr * hg);
         qt = prm.causal ? prm.n_qtiles - 1 - pr : pr;

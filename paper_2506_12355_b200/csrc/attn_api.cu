@@ -9,6 +9,8 @@
 
 #include <atomic>
 #include <mutex>
+#include <utility>
+#include <vector>
 
 #include "../../include/attn_fwd.h"
 #include "attn_combine.cuh"
@@ -134,6 +136,21 @@ int device_info(DeviceInfo* out) {
     return ATTN_OK;
 }
 
+// Raises a kernel's dynamic shared-memory limit once per (kernel, device): the attribute belongs to
+// the device's context, and one process may drive several GPUs.
+bool allow_dynamic_smem(const void* kern, int bytes) {
+    static std::mutex mu;
+    static std::vector<std::pair<const void*, int>> done;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    for (const auto& d : done)
+        if (d.first == kern && d.second == dev) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    done.emplace_back(kern, dev);
+    return true;
+}
+
 int* device_status_ptr() {
     int* p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_device_status) != cudaSuccess) return nullptr;
@@ -155,12 +172,7 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
                    float scale, int causal, int k_offset, cudaStream_t st) {
     using C = attn_tc::PipeCfg<D>;
     auto kern = attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE, ATTN_POLY_NUM, ATTN_POLY_DEN>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-    });
-    if (attr_err != cudaSuccess) return ATTN_ERR_CUDA;
+    if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), C::SMEM_BYTES)) return ATTN_ERR_CUDA;
     const int64_t BH = static_cast<int64_t>(B) * H;
     const int64_t n_pairs = (static_cast<int64_t>(Sq) + 2 * C::BM - 1) / (2 * C::BM);
     if (n_pairs * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
@@ -204,9 +216,12 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     // a device counter that is zeroed on the stream right before the launch
     DeviceInfo di;
     if (device_info(&di) != ATTN_OK) return ATTN_ERR_CUDA;
-    prm.counter = di.counters + (g_launch_seq.fetch_add(1) % kCounterSlots);
-    if (cudaMemsetAsync(prm.counter, 0, sizeof(unsigned int), st) != cudaSuccess) return ATTN_ERR_CUDA;
     const unsigned grid = static_cast<unsigned>(prm.n_items < di.sm_count ? prm.n_items : di.sm_count);
+    prm.counter = nullptr;   // small problems: every CTA takes exactly one item, no counter and no memset
+    if (prm.n_items > di.sm_count) {
+        prm.counter = di.counters + (g_launch_seq.fetch_add(1) % kCounterSlots);
+        if (cudaMemsetAsync(prm.counter, 0, sizeof(unsigned int), st) != cudaSuccess) return ATTN_ERR_CUDA;
+    }
     kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, mo, prm);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
@@ -217,12 +232,7 @@ int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float*
                     float scale, int causal, int k_offset, cudaStream_t st) {
     using C = attn_tc::QTmemCfg<DQK, DV, BN>;
     auto kern = attn_tc::attn_fwd_tc_qtmem_kernel<DQK, DV, BN, DTYPE>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-    });
-    if (attr_err != cudaSuccess) return ATTN_ERR_CUDA;
+    if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), C::SMEM_BYTES)) return ATTN_ERR_CUDA;
     const int64_t BH = static_cast<int64_t>(B) * H;
     const int64_t n_qtiles = (static_cast<int64_t>(Sq) + C::BM - 1) / C::BM;
     if (n_qtiles * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
@@ -368,14 +378,18 @@ int attn_combine(const void* o_parts, const float* lse_parts, int n_parts, void*
     const int segs = D / 8;
     const int64_t total = rows * segs;
     int64_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 32) blocks = 148 * 32;
+    if (blocks > 148 * 64) blocks = 148 * 64;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (dtype == ATTN_DTYPE_FP16)
-        attn_merge::attn_combine_kernel<0><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
-            static_cast<const uint4*>(o_parts), lse_parts, n_parts, static_cast<uint4*>(o), lse, rows, segs);
-    else
-        attn_merge::attn_combine_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
-            static_cast<const uint4*>(o_parts), lse_parts, n_parts, static_cast<uint4*>(o), lse, rows, segs);
+#define ATTN_COMBINE(TT, BB)                                                                                 \
+    attn_merge::attn_combine_kernel<TT, BB><<<static_cast<unsigned>(blocks), 256, 0, st>>>(                    \
+        static_cast<const uint4*>(o_parts), lse_parts, n_parts, static_cast<uint4*>(o), lse, rows, segs)
+    // shards are read in batches of 4 (2 or 1 when there are fewer) so that a batch's loads overlap
+    if (dtype == ATTN_DTYPE_FP16) {
+        if (n_parts >= 3) ATTN_COMBINE(0, 4); else if (n_parts == 2) ATTN_COMBINE(0, 2); else ATTN_COMBINE(0, 1);
+    } else {
+        if (n_parts >= 3) ATTN_COMBINE(1, 4); else if (n_parts == 2) ATTN_COMBINE(1, 2); else ATTN_COMBINE(1, 1);
+    }
+#undef ATTN_COMBINE
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 

@@ -42,7 +42,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 
 // o_parts: [n_parts, rows, D] 16-bit; lse_parts: [n_parts, rows] fp32; o: [rows, D]; lse: [rows].
 // One thread per 8 consecutive output elements (16 bytes).
-template <int DTYPE>
+template <int DTYPE, int BATCH>
 __global__ void __launch_bounds__(256)
 attn_combine_kernel(const uint4* __restrict__ o_parts, const float* __restrict__ lse_parts, int n_parts,
                     uint4* __restrict__ o, float* __restrict__ lse, int64_t rows, int segs_per_row) {
@@ -59,13 +59,23 @@ attn_combine_kernel(const uint4* __restrict__ o_parts, const float* __restrict__
             float sum = 0.f;
             for (int r = 0; r < n_parts; ++r) sum += expf(lse_parts[r * rows + row] - mx);
             total_lse = mx + logf(sum);
-            for (int r = 0; r < n_parts; ++r) {
-                const float w = expf(lse_parts[r * rows + row] - total_lse);
-                if (w == 0.f) continue;
-                float f[8];
-                unpack8<DTYPE>(o_parts[(r * rows + row) * segs_per_row + seg], f);
+            // BATCH shards at a time: all loads of a batch are issued before their results are used
+            for (int r0 = 0; r0 < n_parts; r0 += BATCH) {
+                uint4 v[BATCH];
+                float w[BATCH];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, f[i], acc[i]);
+                for (int i = 0; i < BATCH; ++i) {
+                    const int r = r0 + i < n_parts ? r0 + i : n_parts - 1;   // tail: re-read the last shard, weight 0
+                    v[i] = __ldg(o_parts + (r * rows + row) * segs_per_row + seg);
+                    w[i] = r0 + i < n_parts ? expf(__ldg(lse_parts + r * rows + row) - total_lse) : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < BATCH; ++i) {
+                    float f[8];
+                    unpack8<DTYPE>(v[i], f);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[e] = fmaf(w[i], f[e], acc[e]);
+                }
             }
         }
         uint4 w;

@@ -61,7 +61,7 @@ struct PipeParams {
     int H, Hkv;             // query heads and key/value heads per batch element (H % Hkv == 0)
     int k_offset;           // global index of key 0 of this K/V shard (0 for whole problems); enters the causal mask
     int n_items;            // n_pairs * BH
-    unsigned int* counter;  // work counter, zero at launch: item = gridDim.x + atomicAdd(counter, 1)
+    unsigned int* counter;  // work counter, zero at launch: item = gridDim.x + atomicAdd(counter, 1); NULL when n_items <= grid
 #ifdef ATTN_TC_PROFILE
     long long* prof;        // development builds: [grid][16] cycle sums of softmax group 1, row 0
 #endif
@@ -204,9 +204,10 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const int slot = k & 1;
                 if (!mbar_wait(bar(B_SCHEDEMPTY + slot), ((k >> 1) & 1) ^ 1, abort_flag)) break;
                 if (leader) {
+                    // no counter: the grid covers every item with the CTAs' first draws
                     int next = (k == 0) ? static_cast<int>(blockIdx.x)
-                                        : static_cast<int>(gridDim.x + atomicAdd(prm.counter, 1u));
-                    if (next >= prm.n_items) next = -1;
+                               : (prm.counter ? static_cast<int>(gridDim.x + atomicAdd(prm.counter, 1u)) : prm.n_items);
+                    if (next < 0 || next >= prm.n_items) next = -1;
                     sched_item[slot] = next;
                     mbar_arrive(bar(B_SCHEDFULL + slot));
                 }

@@ -338,3 +338,55 @@ def test_kv_sharded_attention_single_rank_reduces_to_plain_attention():
     o2, l2 = api.attn_fwd(q.to(dev), k.to(dev), v.to(dev), 0.1, True)
     torch.cuda.synchronize()
     assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and float((l1 - l2).abs().max()) <= 1e-5
+
+
+# ------------------------------------------------------------------ scheduling: many items, streams, graphs
+
+def test_many_short_items_match_cross_check_kernel():
+    # 2048 one-pair work items on 148 persistent CTAs: every item must be drawn exactly once
+    B, H, S, D = 64, 32, 128, 64
+    q, k, v = inputs.make_qkv(B, H, S, S, D, inputs.DTYPE_FP16, seed=88)
+    o1, l1 = run_gpu(api.attn_fwd, q, k, v, 0.125, True)
+    o2, l2 = run_gpu(api.attn_fwd_simt, q, k, v, 0.125, True)
+    assert float((o1.float() - o2.float()).abs().max()) <= 2 * O_TOL[inputs.DTYPE_FP16]
+    assert float((l1 - l2).abs().max()) <= 2 * LSE_TOL
+
+
+def test_launches_on_two_streams_do_not_share_a_work_counter():
+    dev = torch.device("cuda:0")
+    cases = []
+    for i, (D, causal) in enumerate(((128, True), (64, False))):
+        q, k, v = inputs.make_qkv(2, 8, 1024, 1024, D, inputs.DTYPE_BF16, seed=120 + i)
+        qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+        ref_o, ref_l = api.attn_fwd(qd, kd, vd, 0.1, causal)
+        cases.append((qd, kd, vd, causal, ref_o, ref_l))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(device=dev) for _ in cases]
+    outs = []
+    for _ in range(5):
+        for (qd, kd, vd, causal, _, _), st in zip(cases, streams):
+            outs.append((api.attn_fwd(qd, kd, vd, 0.1, causal, stream=st), len(outs) % len(cases)))
+    torch.cuda.synchronize()
+    assert api.attn_last_device_status() == 0
+    for (o, l), idx in outs:
+        assert torch.equal(o.view(torch.int16), cases[idx][4].view(torch.int16)) and torch.equal(l, cases[idx][5])
+
+
+def test_cuda_graph_capture_and_replay():
+    dev = torch.device("cuda:0")
+    cfg = inputs.CONFIGS["C1"]
+    q, k, v = (t.to(dev) for t in inputs.make_config_inputs(cfg))
+    o = torch.empty_like(q)
+    lse = torch.empty(cfg.B, cfg.H, cfg.Sq, dtype=torch.float32, device=dev)
+    ref_o, ref_l = api.attn_fwd(q, k, v, cfg.scale, cfg.causal)      # first call: one-time set-up outside capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    st = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            api.attn_fwd(q, k, v, cfg.scale, cfg.causal, out=o, lse=lse, stream=st)
+    for _ in range(3):
+        o.zero_()
+        g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(o.view(torch.int16), ref_o.view(torch.int16)) and torch.equal(lse, ref_l)

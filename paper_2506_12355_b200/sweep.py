@@ -1,0 +1,78 @@
+"""Throughput sweep over the benchmark grid of the paper's Section 4.1.
+
+    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16] [--gqa Hkv] [--iters N]
+
+Grid: sequence length 512 .. 16k with the batch chosen so that batch x sequence = 16k tokens,
+hidden size 2048 (32 heads of dim 64 or 16 heads of dim 128), with and without the causal mask; in
+addition head dim 256 (8 heads) and the 192/128 MLA head shape (16 heads).  FLOPs are counted as in
+the paper, 4 * seq^2 * head_dim * heads per batch element, halved for the causal rows (for the
+192/128 shape: 2 * seq^2 * (192 + 128) * heads).  Inputs are seeded N(0,1) values; every shape is
+timed with CUDA events over isolated launches with a buffer larger than L2 rewritten in between.
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import api, inputs
+
+
+def time_call(fn, flush, iters):
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for i in range(iters):
+        flush.fill_(i & 0xff)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    ts.sort()
+    return ts[len(ts) // 2]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"])
+    ap.add_argument("--gqa", type=int, default=0, help="number of K/V heads (0: same as query heads)")
+    ap.add_argument("--iters", type=int, default=15)
+    args = ap.parse_args()
+    dt = inputs.DTYPE_BF16 if args.dtype == "bf16" else inputs.DTYPE_FP16
+    dev = torch.device("cuda:0")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    seqs = [512, 1024, 2048, 4096, 8192, 16384]
+    shapes = [("D=64", 32, 64, 64), ("D=128", 16, 128, 128), ("D=256", 8, 256, 256), ("Dqk=192 Dv=128", 16, 192, 128)]
+    print("| heads x dims | mask | " + " | ".join(str(s) for s in seqs) + " |")
+    print("|---|---|" + "---|" * len(seqs))
+    for name, H, Dqk, Dv in shapes:
+        Hkv = args.gqa if args.gqa and H % args.gqa == 0 else H
+        for causal in (True, False):
+            cells = []
+            for S in seqs:
+                B = 16384 // S
+                q = inputs.randn16((B, H, S, Dqk), 1, dt).to(dev)
+                k = inputs.randn16((B, Hkv, S, Dqk), 2, dt).to(dev)
+                v = inputs.randn16((B, Hkv, S, Dv), 3, dt).to(dev)
+                o = torch.empty((B, H, S, Dv), dtype=q.dtype, device=dev)
+                lse = torch.empty((B, H, S), dtype=torch.float32, device=dev)
+                scale = Dqk ** -0.5
+                if Dqk == Dv:
+                    fn = lambda: api.attn_fwd_gqa(q, k, v, scale, causal, out=o, lse=lse)
+                else:
+                    fn = lambda: api.attn_fwd_qkv_dims(q, k, v, scale, causal, out=o, lse=lse)
+                ms = time_call(fn, flush, args.iters)
+                flops = 2.0 * B * H * S * S * (Dqk + Dv) / (2 if causal else 1)
+                cells.append("%.0f" % (flops / ms / 1e9))
+                del q, k, v, o, lse
+            print("| %d x %s%s | %s | %s |" % (H, name, "" if Hkv == H else " (Hkv=%d)" % Hkv,
+                                              "causal" if causal else "none", " | ".join(cells)), flush=True)
+    if api.attn_last_device_status() != 0:
+        raise SystemExit("device timeout status")
+
+
+if __name__ == "__main__":
+    main()

@@ -236,13 +236,13 @@ int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float*
     const int64_t BH = static_cast<int64_t>(B) * H;
     const int64_t n_qtiles = (static_cast<int64_t>(Sq) + C::BM - 1) / C::BM;
     if (n_qtiles * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
-    CUtensorMap mk, mv;
+    CUtensorMap mk, mv, mo;
     if (!make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, DQK, C::BN) ||
-        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, DV, C::BN))
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, DV, C::BN) || !make_map(&mo, o, DTYPE, BH, Sq, DV, C::BM))
         return ATTN_ERR_CUDA;
     attn_tc::QTmemParams prm;
     prm.q = q;
-    prm.o = o;
+    prm.o_plain = o;
     prm.lse = lse;
     prm.Sq = Sq;
     prm.Sk = Sk;
@@ -262,13 +262,20 @@ int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float*
     hpg *= H / Hkv;
     if (hpg > BH) hpg = BH;
     prm.heads_per_group = static_cast<int>(hpg);
-    // the last three groups are merged into one: its items, ordered longest-first, then end with short ones,
-    // which keeps the tail of the launch short
     {
         const int64_t n_groups = (BH + hpg - 1) / hpg;
         prm.last_group = static_cast<int>(n_groups >= ATTN_MERGE_LAST ? n_groups - ATTN_MERGE_LAST : 0);
     }
-    kern<<<static_cast<unsigned>(n_qtiles * BH), C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, prm);
+    prm.n_items = static_cast<int>(n_qtiles * BH);
+    DeviceInfo di;
+    if (device_info(&di) != ATTN_OK) return ATTN_ERR_CUDA;
+    const unsigned grid = static_cast<unsigned>(prm.n_items < di.sm_count ? prm.n_items : di.sm_count);
+    prm.counter = nullptr;   // small problems: every CTA takes exactly one item, no counter and no memset
+    if (prm.n_items > di.sm_count) {
+        prm.counter = di.counters + (g_launch_seq.fetch_add(1) % kCounterSlots);
+        if (cudaMemsetAsync(prm.counter, 0, sizeof(unsigned int), st) != cudaSuccess) return ATTN_ERR_CUDA;
+    }
+    kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mo, prm);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 

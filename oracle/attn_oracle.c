@@ -76,6 +76,37 @@ void oracle_widen(const uint16_t *src, double *dst, int64_t n, int dtype)
         dst[i] = dtype == 0 ? oracle_f16_bits_to_f64(src[i]) : oracle_bf16_bits_to_f64(src[i]);
 }
 
+/* ---- 8-bit storage format -> double (exact widening) -------------------- */
+
+/* OCP 8-bit floating point, E4M3 flavour: 1 sign, 4 exponent (bias 7), 3 fraction bits; no
+ * infinities; exponent 15 with fraction 7 is the only NaN, so the largest finite value is
+ * 1.75 * 2^8 = 448.  (FP8 is the data type of the case study in Section 4.4, Table 6; the paper
+ * does not say which 8-bit format or which scaling it uses: E4M3 with one dequantisation factor
+ * per tensor is this build's reading.) */
+double oracle_e4m3_bits_to_f64(uint8_t b)
+{
+    int sign = (b >> 7) & 1;
+    int e = (b >> 3) & 0xf;
+    int f = b & 7;
+    double mag;
+    if (e == 0)
+        mag = ldexp((double)f, -9); /* subnormal: f * 2^-3 * 2^-6 */
+    else if (e == 15 && f == 7)
+        mag = NAN;
+    else
+        mag = ldexp(1.0 + (double)f / 8.0, e - 7);
+    return sign ? -mag : mag;
+}
+
+/* dst[i] = factor * value(src[i]): the dequantised tensor (factor is the per-tensor scale). */
+void oracle_widen_e4m3(const uint8_t *src, double *dst, int64_t n, double factor)
+{
+    int64_t i;
+#pragma omp parallel for schedule(static)
+    for (i = 0; i < n; ++i)
+        dst[i] = factor * oracle_e4m3_bits_to_f64(src[i]);
+}
+
 /* ---- one query row ------------------------------------------------------ */
 
 /* q: [D]; k, v: [Sk, D] of the row's (batch, head); s: scratch of Sk doubles.
@@ -355,6 +386,63 @@ int attn_oracle_rows_16(const uint16_t *q, const uint16_t *k, const uint16_t *v,
                 for (e = 0; e < D; ++e)
                     qd[e] = dtype == 0 ? oracle_f16_bits_to_f64(q[r * D + e])
                                        : oracle_bf16_bits_to_f64(q[r * D + e]);
+                attn_row(qd, kd, vd, s, o + t * D, lse + t, NULL,
+                         visible_keys(r % Sq, Sk, causal), D, scale);
+            }
+            free(s);
+            free(qd);
+        }
+        t0 = t1;
+    }
+    free(kd);
+    free(vd);
+    return failed ? -1 : 0;
+}
+
+/* FP8 inputs: the same definition on the dequantised tensors q_f * Q, k_f * K, v_f * V (E4M3 bit
+ * patterns, one factor per tensor), for a chosen subset of rows and with grouped K/V heads:
+ * q: [B,H,Sq,D]; k, v: [B,Hkv,Sk,D]; rows ascending as in attn_oracle_rows_16. */
+int attn_oracle_rows_e4m3(const uint8_t *q, const uint8_t *k, const uint8_t *v, double q_f, double k_f,
+                          double v_f, const int64_t *rows, int64_t n_rows, double *o, double *lse,
+                          int B, int H, int Hkv, int Sq, int Sk, int D, double scale, int causal)
+{
+    (void)B;
+    if (Hkv <= 0 || H % Hkv != 0)
+        return -2;
+    size_t nk = (size_t)(Sk > 0 ? Sk : 1);
+    double *kd = (double *)malloc(sizeof(double) * nk * (size_t)D);
+    double *vd = (double *)malloc(sizeof(double) * nk * (size_t)D);
+    int failed = (!kd || !vd);
+    int64_t t0 = 0;
+    while (!failed && t0 < n_rows) {
+        int64_t bh = rows[t0] / Sq, t1 = t0;
+        int64_t need = 0;
+        while (t1 < n_rows && rows[t1] / Sq == bh) {
+            int64_t nv = visible_keys(rows[t1] % Sq, Sk, causal);
+            if (nv > need)
+                need = nv;
+            ++t1;
+        }
+        int64_t kvh = (bh / H) * Hkv + (bh % H) / (H / Hkv);
+        oracle_widen_e4m3(k + kvh * Sk * D, kd, need * D, k_f);
+        oracle_widen_e4m3(v + kvh * Sk * D, vd, need * D, v_f);
+#pragma omp parallel
+        {
+            double *s = (double *)malloc(sizeof(double) * nk);
+            double *qd = (double *)malloc(sizeof(double) * (size_t)D);
+            if (!s || !qd) {
+#pragma omp atomic write
+                failed = 1;
+            }
+            int64_t t;
+#pragma omp for schedule(dynamic, 1)
+            for (t = t0; t < t1; ++t) {
+                if (!s || !qd)
+                    continue;
+                int64_t r = rows[t];
+                int e;
+                for (e = 0; e < D; ++e)
+                    qd[e] = q_f * oracle_e4m3_bits_to_f64(q[r * D + e]);
                 attn_row(qd, kd, vd, s, o + t * D, lse + t, NULL,
                          visible_keys(r % Sq, Sk, causal), D, scale);
             }

@@ -61,6 +61,15 @@ def _load():
         lib.attn_oracle_combine_f64.argtypes = [dp, dp, ctypes.c_int, dp, dp, ctypes.c_int64, ctypes.c_int]
         lib.oracle_widen.restype = None
         lib.oracle_widen.argtypes = [u16p, dp, ctypes.c_int64, ctypes.c_int]
+        u8p = ctypes.POINTER(ctypes.c_uint8)
+        lib.oracle_widen_e4m3.argtypes = [u8p, dp, ctypes.c_int64, ctypes.c_double]
+        lib.oracle_widen_e4m3.restype = None
+        lib.oracle_e4m3_bits_to_f64.argtypes = [ctypes.c_uint8]
+        lib.oracle_e4m3_bits_to_f64.restype = ctypes.c_double
+        lib.attn_oracle_rows_e4m3.argtypes = [u8p, u8p, u8p, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                              i64p, ctypes.c_int64, dp, dp] + [ctypes.c_int] * 6 + [
+                                                  ctypes.c_double, ctypes.c_int]
+        lib.attn_oracle_rows_e4m3.restype = ctypes.c_int
         lib.oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -197,6 +206,49 @@ def attention_rows_16(q_bits, k_bits, v_bits, dtype: int, rows, scale: float, ca
         _u16ptr(q_bits), _u16ptr(k_bits), _u16ptr(v_bits), int(dtype),
         rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), rows.size, _dptr(o), _dptr(lse),
         B, H, Sq, Sk, D, float(scale), int(bool(causal)))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return o, lse
+
+
+def _u8ptr(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8))
+
+
+def widen_e4m3(bits: np.ndarray, factor: float = 1.0) -> np.ndarray:
+    """factor * value of E4M3 bit patterns (uint8), exactly, as float64: the dequantised tensor."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    out = np.empty(bits.shape, dtype=np.float64)
+    _load().oracle_widen_e4m3(_u8ptr(bits), _dptr(out), bits.size, float(factor))
+    return out
+
+
+def attention_fp8(q_bits, k_bits, v_bits, q_f: float, k_f: float, v_f: float, scale: float, causal: bool):
+    """FP8 attention by the definition on the dequantised tensors: q_bits uint8 [B,H,Sq,D];
+    k_bits, v_bits uint8 [B,Hkv,Sk,D]; one dequantisation factor per tensor.  Returns o, lse (float64)."""
+    return attention_gqa(widen_e4m3(q_bits, q_f), widen_e4m3(k_bits, k_f), widen_e4m3(v_bits, v_f), scale, causal)
+
+
+def attention_rows_fp8(q_bits, k_bits, v_bits, q_f: float, k_f: float, v_f: float, rows, scale: float, causal: bool):
+    """Row subset of `attention_fp8` straight from the 8-bit inputs (rows: ascending flat indices
+    (b*H + h)*Sq + i).  Returns o [n,D] and lse [n] in float64."""
+    q_bits = np.ascontiguousarray(q_bits, dtype=np.uint8)
+    k_bits = np.ascontiguousarray(k_bits, dtype=np.uint8)
+    v_bits = np.ascontiguousarray(v_bits, dtype=np.uint8)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    B, H, Sq, D = q_bits.shape
+    Hkv, Sk = k_bits.shape[1], k_bits.shape[2]
+    assert k_bits.shape == (B, Hkv, Sk, D) and v_bits.shape == (B, Hkv, Sk, D)
+    assert rows.size == 0 or (rows.min() >= 0 and rows.max() < B * H * Sq)
+    assert np.all(np.diff(rows) >= 0), "rows must be in ascending order"
+    o = np.empty((rows.size, D), dtype=np.float64)
+    lse = np.empty((rows.size,), dtype=np.float64)
+    rc = _load().attn_oracle_rows_e4m3(
+        _u8ptr(q_bits), _u8ptr(k_bits), _u8ptr(v_bits), float(q_f), float(k_f), float(v_f),
+        rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), rows.size, _dptr(o), _dptr(lse),
+        B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)))
+    if rc == -2:
+        raise ValueError("H must be a multiple of Hkv")
     if rc != 0:
         raise MemoryError("oracle scratch allocation failed")
     return o, lse

@@ -20,6 +20,7 @@ import torch
 
 DTYPE_FP16 = 0
 DTYPE_BF16 = 1
+DTYPE_FP8_E4M3 = 2   # 8-bit inputs (stored as uint8 bit patterns), bf16 output
 
 BASE_SEED = 20250612
 
@@ -88,6 +89,25 @@ def make_qkv(B, H, Sq, Sk, D, dtype, seed, sigma=1.0):
     q = randn16((B, H, Sq, D), seed + 0, dtype, sigma)
     k = randn16((B, H, Sk, D), seed + 1, dtype, sigma)
     v = randn16((B, H, Sk, D), seed + 2, dtype, sigma)
+    return q, k, v
+
+
+def randn8(shape, seed: int, sigma: float = 1.0, factor: float = 1.0) -> torch.Tensor:
+    """E4M3 bit patterns (uint8) of sigma * N(0,1) / factor, drawn in fp32 on the CPU from `seed`,
+    clamped to the format's finite range (+-448) and rounded RN-even: the stored tensor whose
+    dequantised value is factor * e4m3(bits)."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(int(seed))
+    x = torch.randn(tuple(shape), generator=g, dtype=torch.float32) * (sigma / factor)
+    return x.clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8).contiguous()
+
+
+def make_qkv_fp8(B, H, Hkv, Sq, Sk, D, seed, sigma=1.0, factors=(1.0, 1.0, 1.0)):
+    """Q [B,H,Sq,D], K, V [B,Hkv,Sk,D] as uint8 E4M3 bit patterns; seeds seed+0/1/2; one
+    dequantisation factor per tensor."""
+    q = randn8((B, H, Sq, D), seed + 0, sigma, factors[0])
+    k = randn8((B, Hkv, Sk, D), seed + 1, sigma, factors[1])
+    v = randn8((B, Hkv, Sk, D), seed + 2, sigma, factors[2])
     return q, k, v
 
 

@@ -342,3 +342,71 @@ def test_shard_with_zero_offset_is_plain_attention_and_empty_merge():
     np.testing.assert_array_equal(lse, lse_ref)
     o2, lse2 = orc.combine(np.zeros((2, 3, 4)), np.full((2, 3), -np.inf))
     assert np.all(o2 == 0.0) and np.all(np.isneginf(lse2))
+
+
+# ------------------------------------------------------------------ 8-bit (E4M3) inputs, Section 4.4 / Table 6
+
+def test_e4m3_widening_all_patterns():
+    allbits = np.arange(256, dtype=np.uint8)
+    got = orc.widen_e4m3(allbits)
+    want = torch.from_numpy(allbits.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    nan = np.isnan(want)
+    assert nan.sum() == 2 and np.array_equal(nan, np.isnan(got))          # 0x7f and 0xff only
+    np.testing.assert_array_equal(got[~nan], want[~nan])
+    assert np.array_equal(np.signbit(got[~nan]), np.signbit(want[~nan]))
+    # landmarks of the format, from its definition (bias 7, 3 fraction bits, no infinities)
+    for code, val in [(0x38, 1.0), (0x7e, 448.0), (0x01, 2.0 ** -9), (0x07, 7 * 2.0 ** -9), (0x08, 2.0 ** -6),
+                      (0x40, 2.0), (0x3c, 1.5), (0xc5, -3.25), (0x78, 256.0)]:
+        assert got[code] == val
+    assert orc.widen_e4m3(np.array([0x3c], dtype=np.uint8), 0.5)[0] == 0.75   # the factor multiplies the value
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_fp8_attention_is_the_definition_on_dequantised_tensors(causal):
+    B, H, Hkv, Sq, Sk, D = 2, 4, 2, 33, 47, 16
+    fq, fk, fv = 0.5, 2.0, 0.125
+    q, k, v = inputs.make_qkv_fp8(B, H, Hkv, Sq, Sk, D, seed=311, factors=(fq, fk, fv))
+    scale = 0.3
+    o, lse = orc.attention_fp8(q.numpy(), k.numpy(), v.numpy(), fq, fk, fv, scale, causal)
+    # torch's own 8-bit decoding and fp64 library attention on the dequantised tensors
+    tq = q.view(torch.float8_e4m3fn).to(torch.float64) * fq
+    tk = (k.view(torch.float8_e4m3fn).to(torch.float64) * fk).repeat_interleave(H // Hkv, dim=1)
+    tv = (v.view(torch.float8_e4m3fn).to(torch.float64) * fv).repeat_interleave(H // Hkv, dim=1)
+    to = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=causal, scale=scale)
+    np.testing.assert_allclose(o, to.numpy(), atol=1e-12)
+    s = (tq @ tk.transpose(-1, -2)) * scale
+    if causal:
+        s = s.masked_fill(torch.triu(torch.ones(Sq, Sk, dtype=torch.bool), 1), float("-inf"))
+    np.testing.assert_allclose(lse, torch.logsumexp(s, dim=-1).numpy(), atol=1e-12)
+    # the factors act as the definition says: q and k factors only through the scores, v's linearly
+    o2, lse2 = orc.attention_fp8(q.numpy(), k.numpy(), v.numpy(), 1.0, 1.0, 1.0, scale * fq * fk, causal)
+    np.testing.assert_allclose(o2 * fv, o, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(lse2, lse, rtol=1e-13, atol=1e-13)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_fp8_row_subset_entry_matches_full(causal):
+    B, H, Hkv, Sq, Sk, D = 2, 4, 2, 40, 56, 16
+    fq, fk, fv = 0.25, 1.0, 4.0
+    q, k, v = inputs.make_qkv_fp8(B, H, Hkv, Sq, Sk, D, seed=312, factors=(fq, fk, fv))
+    o, lse = orc.attention_fp8(q.numpy(), k.numpy(), v.numpy(), fq, fk, fv, 0.25, causal)
+    rows = np.array([0, 1, 39, 40, 79, 100, 159, 160, 319], dtype=np.int64)
+    orows, lrows = orc.attention_rows_fp8(q.numpy(), k.numpy(), v.numpy(), fq, fk, fv, rows, 0.25, causal)
+    np.testing.assert_array_equal(orows, o.reshape(-1, D)[rows])
+    np.testing.assert_array_equal(lrows, lse.reshape(-1)[rows])
+
+
+def test_fp8_input_generator_is_seeded_clamped_and_rounded():
+    a = inputs.randn8((3, 5, 7), 99, sigma=2.0, factor=0.5)
+    b = inputs.randn8((3, 5, 7), 99, sigma=2.0, factor=0.5)
+    assert a.dtype == torch.uint8 and torch.equal(a, b)
+    g = torch.Generator(device="cpu")
+    g.manual_seed(99)
+    x = torch.randn((3, 5, 7), generator=g, dtype=torch.float32) * 4.0
+    val = orc.widen_e4m3(a.numpy())
+    assert not np.isnan(val).any()
+    # nearest representable value: the error is at most half a unit in the last place (2^-4 relative, 2^-10 absolute)
+    err = np.abs(val - x.numpy().astype(np.float64))
+    assert np.all(err <= np.maximum(np.abs(x.numpy()) * 2.0 ** -4, 2.0 ** -10))
+    big = inputs.randn8((1000,), 5, sigma=1000.0)
+    assert np.nanmax(np.abs(orc.widen_e4m3(big.numpy()))) == 448.0

@@ -41,7 +41,9 @@
 extern "C" {
 #endif
 
-typedef enum { ATTN_DTYPE_FP16 = 0, ATTN_DTYPE_BF16 = 1 } attn_dtype_t;
+/* ATTN_DTYPE_FP8_E4M3 names the 8-bit input format of attn_fwd_fp8 only; every entry point with a
+ * `dtype` argument accepts the two 16-bit types and answers ATTN_ERR_UNSUPPORTED_DTYPE otherwise. */
+typedef enum { ATTN_DTYPE_FP16 = 0, ATTN_DTYPE_BF16 = 1, ATTN_DTYPE_FP8_E4M3 = 2 } attn_dtype_t;
 
 typedef enum {
     ATTN_OK = 0,
@@ -119,6 +121,34 @@ int attn_combine(const void* o_parts, const float* lse_parts, int n_parts, void*
  */
 int attn_fwd_qkv_dims(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv,
                       int Sq, int Sk, int Dqk, int Dv, float scale, int causal, int dtype, void* stream);
+
+/*
+ * attn_fwd_fp8 -- the operator on 8-bit inputs: the FP8 case study of Section 4.4 (Table 6: causal
+ * MHA, head dim 128).  The paper reports throughput only and fixes neither the 8-bit format nor a
+ * scaling scheme; this entry point takes E4M3 (1 sign, 4 exponent bits with bias 7, 3 fraction bits,
+ * no infinities, largest finite value 448) with one positive dequantisation factor per tensor:
+ *
+ *     O = Softmax(Mask(scale * (q_factor Q)(k_factor K)^T)) (v_factor V),
+ *     LSE[i] = ln sum over visible j of exp(scale * q_factor * k_factor * <q_i, k_j>).
+ *
+ * q: device, [B,H,Sq,D] bytes; k, v: device, [B,Hkv,Sk,D] bytes (H % Hkv == 0); o: device,
+ * [B,H,Sq,D] bf16; lse: device, [B,H,Sq] fp32.  D must be 128 (ATTN_ERR_UNSUPPORTED_HEAD_DIM
+ * otherwise).  q, k, v, o 16-byte aligned.  scale finite and >= 0; the factors finite and > 0
+ * (ATTN_ERR_BAD_SCALE otherwise).  Inputs must be finite: the bytes 0x7f and 0xff are NaN in this
+ * format, and a NaN in K or V can reach rows from which the mask hides that key.
+ * impl 0: tensor-core kernel -- both products are 8-bit MMAs with fp32 accumulation; the
+ * probabilities are rounded to E4M3 (with a power-of-two factor that keeps them in the format's
+ * normal range) for the second product, which is the one approximation beyond the 16-bit path:
+ * each probability carries a relative rounding error of at most 2^-4, so
+ * |O - O_exact| <= 2^-4 * sum_j p_j |v_factor v_j| elementwise, and typically ~4 % of O's own
+ * root-mean-square size; LSE is not affected (the row sum is taken in fp32 before rounding).
+ * impl 1: the CUDA-core cross-check kernel of attn_fwd_simt on the same inputs (fp32 throughout,
+ * no rounding of the probabilities).  Other values: ATTN_ERR_UNSUPPORTED_DTYPE.
+ * Mask, empty-row convention, ownership, errors and asynchrony as for attn_fwd_gqa.
+ */
+int attn_fwd_fp8(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq,
+                 int Sk, int D, float scale, float q_factor, float k_factor, float v_factor, int causal, int impl,
+                 void* stream);
 
 /*
  * attn_fwd_simt -- same operator, same arguments, same conventions, computed by a plain

@@ -24,7 +24,7 @@ STATUS_NAMES = {
 }
 
 # every symbol include/attn_fwd.h declares
-EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_partial", "attn_combine", "attn_fwd_qkv_dims", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
+EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_partial", "attn_combine", "attn_fwd_qkv_dims", "attn_fwd_fp8", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
            "attn_fwd_host_static", "attn_fwd_host_static_capacity",
            "attn_query_support", "attn_last_device_status", "attn_status_string"]
 
@@ -63,6 +63,8 @@ def load() -> ctypes.CDLL:
     lib.attn_combine.argtypes = [vp, vp, i, vp, vp, i, i, i, i, i, vp]
     lib.attn_fwd_qkv_dims.restype = i
     lib.attn_fwd_qkv_dims.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, vp]
+    lib.attn_fwd_fp8.restype = i
+    lib.attn_fwd_fp8.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, f, f, f, i, i, vp]
     lib.attn_fwd_simt.restype = i
     lib.attn_fwd_simt.argtypes = sig
     lib.attn_fwd_host.restype = i
@@ -229,6 +231,33 @@ def attn_fwd_qkv_dims(q, k, v, scale: float, causal: bool = False, out=None, lse
                                       _stream_ptr(stream))
     if rc != 0:
         raise AttnError(rc, "attn_fwd_qkv_dims")
+    return out, lse
+
+
+def attn_fwd_fp8(q, k, v, scale: float, q_factor: float = 1.0, k_factor: float = 1.0, v_factor: float = 1.0,
+                 causal: bool = False, out=None, lse=None, stream=None, impl: int = 0):
+    """Attention on E4M3 inputs with one dequantisation factor per tensor: q [B,H,Sq,128],
+    k, v [B,Hkv,Sk,128] as CUDA uint8 (or torch.float8_e4m3fn) tensors; returns o (bf16) and lse (fp32).
+    impl 0: tensor-core kernel; impl 1: CUDA-core cross-check kernel."""
+    if q.dim() != 4 or k.dim() != 4 or v.dim() != 4:
+        raise ValueError("q, k, v must be [B,H,S,D]")
+    for t in (q, k, v):
+        if t.dtype not in (torch.uint8, torch.float8_e4m3fn) or not t.is_cuda or not t.is_contiguous():
+            raise ValueError("q, k, v must be contiguous CUDA tensors of E4M3 bytes")
+    B, H, Sq, D = q.shape
+    Hkv, Sk = k.shape[1], k.shape[2]
+    if tuple(k.shape) != (B, Hkv, Sk, D) or tuple(v.shape) != (B, Hkv, Sk, D):
+        raise ValueError("k, v must be [B,Hkv,Sk,D] matching q's B and D")
+    if out is None:
+        out = torch.empty((B, H, Sq, D), dtype=torch.bfloat16, device=q.device)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(q.device):
+        rc = load().attn_fwd_fp8(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                 B, H, Hkv, Sq, Sk, D, float(scale), float(q_factor), float(k_factor),
+                                 float(v_factor), int(bool(causal)), int(impl), _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_fwd_fp8")
     return out, lse
 
 

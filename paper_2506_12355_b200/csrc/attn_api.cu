@@ -55,16 +55,20 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// Rank-3 map over a [BH, S, D] row-major 16-bit tensor; box = [1, box_rows, 64 columns],
-// 128-byte swizzle, out-of-range rows read as zero.
+// Rank-3 map over a [BH, S, D] row-major tensor of 16-bit (dtype 0 / 1) or 8-bit (dtype 2) elements;
+// box = [1, box_rows, 128 bytes of columns], 128-byte swizzle, out-of-range rows read as zero.
 bool make_map(CUtensorMap* map, const void* base, int dtype, int64_t BH, int64_t S, int D, int box_rows) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
+    const cuuint64_t es = dtype == ATTN_DTYPE_FP8_E4M3 ? 1 : 2;
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S), static_cast<cuuint64_t>(BH)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(S) * D * 2};
-    cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), 1};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * es, static_cast<cuuint64_t>(S) * D * es};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(128 / es), static_cast<cuuint32_t>(box_rows), 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(map, dtype == ATTN_DTYPE_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+    const CUtensorMapDataType type = dtype == ATTN_DTYPE_FP16   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                     : dtype == ATTN_DTYPE_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                                                : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+    CUresult r = enc(map, type,
                      3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -169,8 +173,10 @@ long long* g_prof_buffer = nullptr;  // development builds only
 // Pipelined, warp-specialised kernel (head dims 64 and 128): one CTA per pair of 128-row Q tiles.
 template <int D, int DTYPE>
 int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                   float scale, int causal, int k_offset, cudaStream_t st) {
-    using C = attn_tc::PipeCfg<D>;
+                   float scale, int causal, int k_offset, cudaStream_t st, float o_scale = 1.f) {
+    constexpr int ES = DTYPE == ATTN_DTYPE_FP8_E4M3 ? 1 : 2;                 // bytes per Q/K/V element
+    constexpr int ODT = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_DTYPE_BF16 : DTYPE;   // O storage type
+    using C = attn_tc::PipeCfg<D, ES>;
     auto kern = attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE, ATTN_POLY_NUM, ATTN_POLY_DEN>;
     if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), C::SMEM_BYTES)) return ATTN_ERR_CUDA;
     const int64_t BH = static_cast<int64_t>(B) * H;
@@ -178,7 +184,7 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     if (n_pairs * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
     CUtensorMap mq, mk, mv, mo;
     if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) ||
-        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) || !make_map(&mo, o, DTYPE, BH, Sq, D, C::BM))
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) || !make_map(&mo, o, ODT, BH, Sq, D, C::BM))
         return ATTN_ERR_CUDA;
     attn_tc::PipeParams prm;
     prm.o = o;
@@ -187,6 +193,7 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     prm.Sk = Sk;
     prm.scale = scale;
     prm.scale_log2 = scale * 1.4426950408889634f;
+    prm.o_scale = o_scale;
     prm.causal = causal ? 1 : 0;
     prm.status = device_status_ptr();
     if (!prm.status) return ATTN_ERR_CUDA;
@@ -196,7 +203,7 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     prm.n_pairs = static_cast<int>(n_pairs);
     prm.BH = static_cast<int>(BH);
     // walk together as many heads as keep their K and V (2 * Sk * D * 2 bytes each) inside ~24 MB of L2 (the L2 is split over two dies)
-    const int64_t kv_bytes_per_head = 4LL * Sk * D;
+    const int64_t kv_bytes_per_head = 2LL * ES * Sk * D;
     int64_t hpg = (static_cast<int64_t>(ATTN_L2_MB) << 20) / (kv_bytes_per_head > 0 ? kv_bytes_per_head : 1);
     if (hpg < 1) hpg = 1;
     hpg *= H / Hkv;  // the query heads of one K/V head share its footprint
@@ -281,13 +288,13 @@ int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float*
 
 template <int D, int DTYPE>
 int launch_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                float scale, int causal, int k_offset, cudaStream_t st) {
+                float scale, int causal, int k_offset, cudaStream_t st, float o_scale = 1.f) {
     const int64_t BH = static_cast<int64_t>(B) * H;
     if (BH > 65535) return ATTN_ERR_BAD_SHAPE;
     dim3 grid(static_cast<unsigned>((static_cast<int64_t>(Sq) + attn_simt::kWarpsPerBlock - 1) / attn_simt::kWarpsPerBlock),
               static_cast<unsigned>(BH));
     attn_simt::attn_fwd_simt_kernel<D, DTYPE><<<grid, attn_simt::kWarpsPerBlock * 32, 0, st>>>(q, k, v, o, lse, Sq, Sk,
-                                                                                              scale, causal ? 1 : 0, H, Hkv, k_offset);
+                                                                                              scale, causal ? 1 : 0, H, Hkv, k_offset, o_scale);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
@@ -416,6 +423,32 @@ int attn_fwd_qkv_dims(const void* q, const void* k, const void* v, void* o, floa
     if (dtype == ATTN_DTYPE_FP16)
         return launch_tc_qtmem<192, 128, 128, 0>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, 0, st);
     return launch_tc_qtmem<192, 128, 128, 1>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, 0, st);
+}
+
+int attn_fwd_fp8(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
+                 int D, float scale, float q_factor, float k_factor, float v_factor, int causal, int impl, void* stream) {
+    if (D != 128) {
+        if (B < 0 || H < 0 || Hkv < 0 || Sq < 0 || Sk < 0 || D < 0) return ATTN_ERR_BAD_SHAPE;
+        return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
+    }
+    // the shared checks, with a 16-bit type standing in (they do not depend on the element size)
+    int rc = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, ATTN_DTYPE_BF16, true);
+    if (rc != ATTN_OK) return rc;
+    if (!isfinite(q_factor) || !isfinite(k_factor) || !isfinite(v_factor) || q_factor <= 0.f || k_factor <= 0.f ||
+        v_factor <= 0.f)
+        return ATTN_ERR_BAD_SCALE;
+    const float s_eff = scale * q_factor * k_factor;   // the factors of Q and K act only through the scores
+    if (!isfinite(s_eff)) return ATTN_ERR_BAD_SCALE;
+    if (impl != 0 && impl != 1) return ATTN_ERR_UNSUPPORTED_DTYPE;
+    if (static_cast<int64_t>(B) * H * Sq == 0) return ATTN_OK;
+    rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (Sk == 0)
+        return fill_empty(o, lse, static_cast<int64_t>(B) * H * Sq * D, static_cast<int64_t>(B) * H * Sq, st);
+    if (impl == 1)
+        return launch_simt<128, ATTN_DTYPE_FP8_E4M3>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, s_eff, causal, 0, st, v_factor);
+    return launch_tc_pipe<128, ATTN_DTYPE_FP8_E4M3>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, s_eff, causal, 0, st, v_factor);
 }
 
 int attn_fwd_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,

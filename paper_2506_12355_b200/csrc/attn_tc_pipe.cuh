@@ -151,16 +151,17 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         B_PFULL2 = 8,     // [2] rest of P_t written
         B_OFINAL = 10,    // [2] last O_t += P_t V of the item has finished
         B_OFREE = 12,     // [2] the epilogue has read O_t out of tensor memory (128 softmax threads)
-        B_SCHEDFULL = 14, // [2] scheduler slot holds the next item
-        B_SCHEDEMPTY = 16,// [2] slot read by the MMA warp and the 8 softmax warps
-        B_KVFULL = 18,
-        B_KVEMPTY = 18 + NSLOT,
-        B_COUNT = 18 + 2 * NSLOT
+        B_SCHEDFULL = 14, // [4] scheduler slot holds a decoded item
+        B_SCHEDEMPTY = 18,// [4] slot read by the MMA warp and the 8 softmax warps
+        B_KVFULL = 22,
+        B_KVEMPTY = 22 + NSLOT,
+        B_COUNT = 22 + 2 * NSLOT
     };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
-    volatile int* sched_item = reinterpret_cast<volatile int*>(bars + B_COUNT);       // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT) + 2;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 3;
+    // scheduler slots [4][8]: item index (-1: no more work), bh, kv_bh, q0, n_kv[0], n_kv[1]
+    volatile int* sched_item = reinterpret_cast<volatile int*>(bars + B_COUNT);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT) + 32;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 33;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -175,7 +176,9 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             mbar_init(bar(B_OFINAL + t), 1);
             mbar_init(bar(B_OFREE + t), 128);
             mbar_init(bar(B_SCHEDFULL + t), 1);
+            mbar_init(bar(B_SCHEDFULL + 2 + t), 1);
             mbar_init(bar(B_SCHEDEMPTY + t), 9);
+            mbar_init(bar(B_SCHEDEMPTY + 2 + t), 9);
         }
         for (int s = 0; s < NSLOT; ++s) {
             mbar_init(bar(B_KVFULL + s), 1);
@@ -199,11 +202,19 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
-    // Consumers of the scheduler: wait for the k-th item of this CTA, read it, hand the slot back.
-    auto next_item = [&](int k, bool hand_back) -> int {
-        const int slot = k & 1;
-        if (!mbar_wait(bar(B_SCHEDFULL + slot), (k >> 1) & 1, abort_flag)) return -1;
-        const int item = sched_item[slot];
+    // Consumers of the scheduler: wait for the k-th item of this CTA, read it (the producer has decoded it:
+    // the index arithmetic is done once per item, not once per thread), hand the slot back.
+    auto next_item = [&](int k, bool hand_back, PipeItem& it) -> int {
+        const int slot = k & 3;
+        if (!mbar_wait(bar(B_SCHEDFULL + slot), (k >> 2) & 1, abort_flag)) return -1;
+        volatile int* e = sched_item + slot * 8;
+        const int item = e[0];
+        it.bh = e[1];
+        it.kv_bh = e[2];
+        it.q0 = e[3];
+        it.n_kv[0] = e[4];
+        it.n_kv[1] = e[5];
+        it.n_max = it.n_kv[0] > it.n_kv[1] ? it.n_kv[0] : it.n_kv[1];
         if (hand_back) mbar_arrive(bar(B_SCHEDEMPTY + slot));
         return item;
     };
@@ -218,21 +229,35 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             const bool leader = elect_one();
             int kv_base = 0;            // ring items issued for earlier work items
             int q_uses[2] = {0, 0};     // work items that loaded Q tile t so far
-            for (int k = 0;; ++k) {
-                // ---- draw the next work item and publish it ----
-                const int slot = k & 1;
-                if (!mbar_wait(bar(B_SCHEDEMPTY + slot), ((k >> 1) & 1) ^ 1, abort_flag)) break;
+            // Draws the k-th work item of this CTA, decodes it and publishes it in scheduler slot k & 3.
+            // (Drawing one item ahead was measured and is slower: the CTAs finish less evenly.)
+            auto publish = [&](int k) -> bool {
+                const int slot = k & 3;
+                if (!mbar_wait(bar(B_SCHEDEMPTY + slot), ((k >> 2) & 1) ^ 1, abort_flag)) return false;
                 if (leader) {
                     // no counter: the grid covers every item with the CTAs' first draws
                     int next = (k == 0) ? static_cast<int>(blockIdx.x)
                                : (prm.counter ? static_cast<int>(gridDim.x + atomicAdd(prm.counter, 1u)) : prm.n_items);
                     if (next < 0 || next >= prm.n_items) next = -1;
-                    sched_item[slot] = next;
+                    volatile int* e = sched_item + slot * 8;
+                    if (next >= 0) {
+                        const PipeItem d = pipe_decode_item(prm, next, BM, BN);
+                        e[1] = d.bh;
+                        e[2] = d.kv_bh;
+                        e[3] = d.q0;
+                        e[4] = d.n_kv[0];
+                        e[5] = d.n_kv[1];
+                    }
+                    e[0] = next;
                     mbar_arrive(bar(B_SCHEDFULL + slot));
                 }
-                const int item = next_item(k, false);
+                return true;
+            };
+            for (int k = 0;; ++k) {
+                if (!publish(k)) break;
+                PipeItem it;
+                const int item = next_item(k, false, it);
                 if (item < 0) break;
-                const PipeItem it = pipe_decode_item(prm, item, BM, BN);
 
                 auto load_q = [&](int t) -> bool {
                     // the previous item's S MMAs on this Q buffer must have finished
@@ -315,9 +340,9 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             int uses[2] = {0, 0};      // work items in which tile t took part
             bool ok = true;
             for (int k = 0; ok; ++k) {
-                const int item = next_item(k, leader);
+                PipeItem it;
+                const int item = next_item(k, leader, it);
                 if (item < 0) break;
-                const PipeItem it = pipe_decode_item(prm, item, BM, BN);
                 // ---- first S of both tiles ----
                 if (it.n_max > 0) ok = kv_full_wait(kv_base);
 #pragma unroll
@@ -396,10 +421,10 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 #endif
 
         for (int k = 0; ok; ++k) {
-            const int item = next_item(k, lane == 0);
+            PipeItem it;
+            const int item = next_item(k, lane == 0, it);
             PLAP(0);
             if (item < 0) break;
-            const PipeItem it = pipe_decode_item(prm, item, BM, BN);
             const int n = it.n_kv[t];
             const int q0 = it.q0;
             const int row = q0 + t * BM + r;

@@ -114,16 +114,17 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         B_ODONE = 5,       // completes once per step: O += P_g V_g has finished
         B_OFINAL = 6,      // completes once per item: its last second product has finished
         B_OFREE = 7,       // the epilogue has read O out of tensor memory (128 softmax threads)
-        B_SCHEDFULL = 8,   // [2] scheduler slot holds the next item
+        B_SCHEDFULL = 8,   // [2] scheduler slot holds the next item, decoded
         B_SCHEDEMPTY = 10, // [2] slot read by the MMA warp and the 4 softmax warps
         B_KVFULL = 12,
         B_KVEMPTY = 12 + NSLOT,
         B_COUNT = 12 + 2 * NSLOT
     };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
-    volatile int* sched_item = reinterpret_cast<volatile int*>(bars + B_COUNT);   // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT) + 2;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 3;
+    // scheduler slots [2][8]: item index (-1: no more work), bh, kv_bh, q0, n
+    volatile int* sched_item = reinterpret_cast<volatile int*>(bars + B_COUNT);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT) + 16;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 17;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -161,10 +162,16 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     const uint32_t tmem = *tmem_slot;
 
     // Consumers of the scheduler: wait for the k-th item of this CTA, read it, hand the slot back.
-    auto next_item = [&](int k, bool hand_back) -> int {
+    // (the producer has decoded the item: the index arithmetic is done once per item, not once per thread)
+    auto next_item = [&](int k, bool hand_back, QTmemItem& it) -> int {
         const int slot = k & 1;
         if (!mbar_wait(bar(B_SCHEDFULL + slot), (k >> 1) & 1, abort_flag)) return -1;
-        const int item = sched_item[slot];
+        volatile int* e = sched_item + slot * 8;
+        const int item = e[0];
+        it.bh = e[1];
+        it.kv_bh = e[2];
+        it.q0 = e[3];
+        it.n = e[4];
         if (hand_back) mbar_arrive(bar(B_SCHEDEMPTY + slot));
         return item;
     };
@@ -185,12 +192,20 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
                 int next = (k == 0) ? static_cast<int>(blockIdx.x)
                            : (prm.counter ? static_cast<int>(gridDim.x + atomicAdd(prm.counter, 1u)) : prm.n_items);
                 if (next < 0 || next >= prm.n_items) next = -1;
-                sched_item[slot] = next;
+                volatile int* e = sched_item + slot * 8;
+                if (next >= 0) {
+                    const QTmemItem d = qtmem_decode_item(prm, next, BM, BN);
+                    e[1] = d.bh;
+                    e[2] = d.kv_bh;
+                    e[3] = d.q0;
+                    e[4] = d.n;
+                }
+                e[0] = next;
                 mbar_arrive(bar(B_SCHEDFULL + slot));
             }
-            const int item = next_item(k, false);
+            QTmemItem it;
+            const int item = next_item(k, false, it);
             if (item < 0) break;
-            const QTmemItem it = qtmem_decode_item(prm, item, BM, BN);
             auto load_kv = [&](const CUtensorMap* map, int nbox, int ring_item, int j) -> bool {
                 const int s = ring_item % NSLOT;
                 const uint32_t use = ring_item / NSLOT;
@@ -226,9 +241,9 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         int uses = 0;     // work items with at least one step so far
         bool ok = true;
         for (int k = 0; ok; ++k) {
-            const int item = next_item(k, leader);
+            QTmemItem it;
+            const int item = next_item(k, leader, it);
             if (item < 0) break;
-            const QTmemItem it = qtmem_decode_item(prm, item, BM, BN);
             if (it.n == 0) continue;
             auto issue_s = [&](int j) {   // S = Q K_j^T into buffer (g_base + j) & 1 : DQK/16 instructions of K = 16
                 if (leader) {
@@ -310,8 +325,8 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 
         int g_base = 0, uses = 0;
         bool ok = true;
-        int item = next_item(0, lane == 0);
-        QTmemItem it = qtmem_decode_item(prm, item < 0 ? 0 : item, BM, BN);
+        QTmemItem it;
+        int item = next_item(0, lane == 0, it);
         if (item >= 0 && it.n > 0) load_q(it);
 
         for (int k = 0; ok && item >= 0; ++k) {
@@ -483,8 +498,8 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 
             // ---- the next item: its Q goes into tensor memory while the last second product still runs
             // (every S of the current item has finished: the last one was waited for above) ----
-            const int next = next_item(k + 1, lane == 0);
-            QTmemItem itn = qtmem_decode_item(prm, next < 0 ? 0 : next, BM, BN);
+            QTmemItem itn;
+            const int next = next_item(k + 1, lane == 0, itn);
             if (next >= 0 && itn.n > 0) load_q(itn);
 
             // ---- epilogue of the current item: O / l and LSE ----

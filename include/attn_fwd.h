@@ -165,6 +165,12 @@ int attn_fwd_simt(const void* q, const void* k, const void* v, void* o, float* l
  * least attn_fwd_host_workspace_bytes(...) bytes, 256-byte aligned.  Enqueues on `stream`:
  * three host-to-device copies, the attention kernel, two device-to-host copies.  The results
  * are valid once the caller has synchronised `stream`.
+ * Large problems (at least 16 MiB of Q, K, V and at least 4 heads) are split into up to 8 groups
+ * of heads: the kernels of the groups run on `stream`, the copies on two streams of the library's
+ * own (created with their events on the first such call on a device), so that copies in both
+ * directions overlap the kernels.  Everything is ordered after the work already on `stream`, and
+ * `stream` waits for the last copy back, so the caller sees the same ordering as for the small
+ * case.  Calls from several host threads are serialised while they enqueue.
  * Errors: as attn_fwd, plus ATTN_ERR_WORKSPACE.
  */
 int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,

@@ -363,6 +363,86 @@ int static_workspace_ptr(void** out) {
 
 }  // namespace
 
+namespace {
+
+// ---- attn_fwd_host for large problems: groups of heads pipelined over two internal copy streams ----
+//
+// The caller's stream runs the kernels; one internal stream carries the host-to-device copies, one the
+// device-to-host copies, so that the copies of neighbouring groups overlap the kernels and each other
+// (PCIe is full duplex).  Streams and events are created once per device, on first use.
+constexpr int kHostPipeMaxChunks = 8;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_in[kHostPipeMaxChunks] = {}, ev_k[kHostPipeMaxChunks] = {};
+    std::mutex mu;   // one enqueue sequence at a time: the events are shared by every call on the device
+};
+HostPipe g_host_pipe[64];
+
+// at least 16 MiB to copy in (more than the built-in buffer of attn_fwd_host_static can hold, so that entry point
+// never takes this path and keeps its promise to create nothing) and at least 4 heads to split
+bool host_pipe_wanted(size_t bh, size_t h2d_bytes) { return bh >= 4 && h2d_bytes >= (static_cast<size_t>(16) << 20); }
+
+int host_pipelined(const void* q_host, const void* k_host, const void* v_host, void* o_host, float* lse_host, int BH, int Sq,
+                   int Sk, int D, float scale, int causal, int dtype, uint8_t* dq, uint8_t* dk, uint8_t* dv, uint8_t* d_o,
+                   float* dl, cudaStream_t st) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ATTN_ERR_CUDA;
+    HostPipe& hp = g_host_pipe[dev];
+    std::lock_guard<std::mutex> lock(hp.mu);
+    if (!hp.ready) {
+        bool ok = cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.ev_done, cudaEventDisableTiming) == cudaSuccess;
+        for (int c = 0; ok && c < kHostPipeMaxChunks; ++c)
+            ok = cudaEventCreateWithFlags(&hp.ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.ev_k[c], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return ATTN_ERR_CUDA;
+        hp.ready = true;
+    }
+    const int n_chunks = BH < kHostPipeMaxChunks ? BH : kHostPipeMaxChunks;
+    const size_t q_head = static_cast<size_t>(Sq) * D * 2, kv_head = static_cast<size_t>(Sk) * D * 2, l_head = static_cast<size_t>(Sq) * 4;
+    // everything below is ordered after the work already on the caller's stream
+    if (cudaEventRecord(hp.ev_start, st) != cudaSuccess) return ATTN_ERR_CUDA;
+    if (cudaStreamWaitEvent(hp.s_in, hp.ev_start, 0) != cudaSuccess) return ATTN_ERR_CUDA;
+    if (cudaStreamWaitEvent(hp.s_out, hp.ev_start, 0) != cudaSuccess) return ATTN_ERR_CUDA;
+    for (int c = 0; c < n_chunks; ++c) {
+        const int h0 = static_cast<int>(static_cast<int64_t>(BH) * c / n_chunks);
+        const int h1 = static_cast<int>(static_cast<int64_t>(BH) * (c + 1) / n_chunks);
+        const size_t nh = static_cast<size_t>(h1 - h0);
+        const uint8_t* qh = static_cast<const uint8_t*>(q_host) + h0 * q_head;
+        const uint8_t* kh = static_cast<const uint8_t*>(k_host) + h0 * kv_head;
+        const uint8_t* vh = static_cast<const uint8_t*>(v_host) + h0 * kv_head;
+        if (cudaMemcpyAsync(dq + h0 * q_head, qh, nh * q_head, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess) return ATTN_ERR_CUDA;
+        if (kv_head) {
+            if (cudaMemcpyAsync(dk + h0 * kv_head, kh, nh * kv_head, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess) return ATTN_ERR_CUDA;
+            if (cudaMemcpyAsync(dv + h0 * kv_head, vh, nh * kv_head, cudaMemcpyHostToDevice, hp.s_in) != cudaSuccess) return ATTN_ERR_CUDA;
+        }
+        if (cudaEventRecord(hp.ev_in[c], hp.s_in) != cudaSuccess) return ATTN_ERR_CUDA;
+        if (cudaStreamWaitEvent(st, hp.ev_in[c], 0) != cudaSuccess) return ATTN_ERR_CUDA;
+        // the heads of a group as one batch element: (batch, head) only enters the kernels as one flat index
+        int rc = attn_fwd(dq + h0 * q_head, dk + h0 * kv_head, dv + h0 * kv_head, d_o + h0 * q_head,
+                          reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(dl) + h0 * l_head), 1, static_cast<int>(nh), Sq, Sk, D,
+                          scale, causal, dtype, st);
+        if (rc != ATTN_OK) return rc;
+        if (cudaEventRecord(hp.ev_k[c], st) != cudaSuccess) return ATTN_ERR_CUDA;
+        if (cudaStreamWaitEvent(hp.s_out, hp.ev_k[c], 0) != cudaSuccess) return ATTN_ERR_CUDA;
+        if (cudaMemcpyAsync(static_cast<uint8_t*>(o_host) + h0 * q_head, d_o + h0 * q_head, nh * q_head, cudaMemcpyDeviceToHost,
+                            hp.s_out) != cudaSuccess)
+            return ATTN_ERR_CUDA;
+        if (cudaMemcpyAsync(reinterpret_cast<uint8_t*>(lse_host) + h0 * l_head, reinterpret_cast<uint8_t*>(dl) + h0 * l_head,
+                            nh * l_head, cudaMemcpyDeviceToHost, hp.s_out) != cudaSuccess)
+            return ATTN_ERR_CUDA;
+    }
+    // the caller's stream continues only after the last copy back
+    if (cudaEventRecord(hp.ev_done, hp.s_out) != cudaSuccess) return ATTN_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, hp.ev_done, 0) != cudaSuccess) return ATTN_ERR_CUDA;
+    return ATTN_OK;
+}
+
+}  // namespace
+
 extern "C" {
 
 #ifdef ATTN_TC_PROFILE
@@ -488,6 +568,9 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
     uint8_t* d_o = dv + align256(kv_b);
     float* dl = reinterpret_cast<float*>(d_o + align256(qo_b));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (host_pipe_wanted(bh, qo_b + 2 * kv_b))
+        return host_pipelined(q_host, k_host, v_host, o_host, lse_host, static_cast<int>(bh), Sq, Sk, D, scale, causal, dtype,
+                              dq, dk, dv, d_o, dl, st);
     if (cudaMemcpyAsync(dq, q_host, qo_b, cudaMemcpyHostToDevice, st) != cudaSuccess) return ATTN_ERR_CUDA;
     if (kv_b) {
         if (cudaMemcpyAsync(dk, k_host, kv_b, cudaMemcpyHostToDevice, st) != cudaSuccess) return ATTN_ERR_CUDA;

@@ -197,6 +197,29 @@ def test_host_entry_matches_device_entry():
     assert torch.equal(o.view(torch.int16), o_dev.view(torch.int16)) and torch.equal(lse, lse_dev)
 
 
+@pytest.mark.parametrize("D,dtype,causal,B,H,S", [(128, 1, True, 2, 8, 2048), (64, 0, False, 1, 5, 8192)])
+def test_host_entry_pipelined_over_groups_of_heads(D, dtype, causal, B, H, S):
+    # large enough (>= 16 MiB of Q, K, V, >= 4 heads) for the copies to run on the library's own streams in
+    # groups of heads; two calls in a row on a side stream, the second on other inputs into the same workspace
+    dev = torch.device("cuda:0")
+    ws = torch.empty(api.attn_fwd_host_workspace_bytes(B, H, S, S, D), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    outs, refs = [], []
+    for rep in range(2):
+        q, k, v = inputs.make_qkv(B, H, S, S, D, dtype, seed=4400 + 10 * rep)
+        refs.append(run_gpu(api.attn_fwd, q, k, v, D ** -0.5, causal))
+        o = torch.full((B, H, S, D), float("nan"), dtype=q.dtype).pin_memory()
+        lse = torch.full((B, H, S), float("nan"), dtype=torch.float32).pin_memory()
+        outs.append((q.pin_memory(), k.pin_memory(), v.pin_memory(), o, lse))
+    with torch.cuda.stream(stream):
+        for qp, kp, vp, o, lse in outs:
+            api.attn_fwd_host(qp, kp, vp, D ** -0.5, causal, o, lse, ws, stream=stream)
+    stream.synchronize()
+    assert api.attn_last_device_status() == 0
+    for (qp, kp, vp, o, lse), (o_dev, lse_dev) in zip(outs, refs):
+        assert torch.equal(o.view(torch.int16), o_dev.view(torch.int16)) and torch.equal(lse, lse_dev)
+
+
 # ------------------------------------------------------------------ full-size configurations, sampled rows
 
 @pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5"])

@@ -25,6 +25,10 @@
 #define ATTN_POLY_DEN 8
 #endif
 
+#ifndef ATTN_POLY64_NUM
+#define ATTN_POLY64_NUM 1
+#define ATTN_POLY64_DEN 4
+#endif
 #ifndef ATTN_FP8_POLY_NUM
 #define ATTN_FP8_POLY_NUM 1
 #define ATTN_FP8_POLY_DEN 8
@@ -181,9 +185,10 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     constexpr int ES = DTYPE == ATTN_DTYPE_FP8_E4M3 ? 1 : 2;                 // bytes per Q/K/V element
     constexpr int ODT = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_DTYPE_BF16 : DTYPE;   // O storage type
     using C = attn_tc::PipeCfg<D, ES>;
-    // share of the exponentials evaluated by the polynomial: one pair in ATTN_POLY_DEN / ATTN_FP8_POLY_DEN
-    constexpr int PN = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_FP8_POLY_NUM : ATTN_POLY_NUM;
-    constexpr int PD = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_FP8_POLY_DEN : ATTN_POLY_DEN;
+    // share of the exponentials evaluated by the polynomial (measured best): 1 pair in 8 at head dim 128, 1 in 4 at
+    // head dim 64, where the tensor core leaves more issue slots to the softmax warps
+    constexpr int PN = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_FP8_POLY_NUM : (D == 64 ? ATTN_POLY64_NUM : ATTN_POLY_NUM);
+    constexpr int PD = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_FP8_POLY_DEN : (D == 64 ? ATTN_POLY64_DEN : ATTN_POLY_DEN);
     auto kern = attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE, PN, PD>;
     if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), C::SMEM_BYTES)) return ATTN_ERR_CUDA;
     const int64_t BH = static_cast<int64_t>(B) * H;

@@ -1,6 +1,6 @@
 """Throughput sweep over the benchmark grid of the paper's Section 4.1.
 
-    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16|fp8] [--gqa Hkv] [--iters N] [--seq S]
+    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16|fp8] [--gqa Hkv] [--iters N] [--seq S] [--shards N]
 
 Grid: sequence length 512 .. 16k with the batch chosen so that batch x sequence = 16k tokens,
 hidden size 2048 (32 heads of dim 64 or 16 heads of dim 128), with and without the causal mask; in
@@ -10,6 +10,11 @@ inputs.  FLOPs are counted as in
 the paper, 4 * seq^2 * head_dim * heads per batch element, halved for the causal rows (for the
 192/128 shape: 2 * seq^2 * (192 + 128) * heads).  Inputs are seeded N(0,1) values; every shape is
 timed with CUDA events over isolated launches with a buffer larger than L2 rewritten in between.
+
+`--shards N` times the K/V-sharded path instead (the building block of split-KV decoding and of K/V
+sharding across GPUs): N partial launches over N key ranges of one problem (causal, 32 heads of dim
+128, bf16) and the merge of their results, against the unsharded call; the merge kernel is
+memory-bound and is reported in GB/s of the bytes it must move.
 """
 from __future__ import annotations
 
@@ -37,16 +42,51 @@ def time_call(fn, flush, iters):
     return ts[len(ts) // 2]
 
 
+def shard_table(args, dev, flush):
+    n, H, D, dt = args.shards, 32, 128, inputs.DTYPE_BF16
+    print("| sequence | unsharded ms | %d partial launches ms | merge us | merge GB/s | sharded / unsharded |" % n)
+    print("|---|---|---|---|---|---|")
+    for S in ([args.seq] if args.seq else [4096, 16384]):
+        q = inputs.randn16((1, H, S, D), 1, dt).to(dev)
+        k = inputs.randn16((1, H, S, D), 2, dt).to(dev)
+        v = inputs.randn16((1, H, S, D), 3, dt).to(dev)
+        o = torch.empty_like(q)
+        lse = torch.empty((1, H, S), dtype=torch.float32, device=dev)
+        o_parts = torch.empty((n, 1, H, S, D), dtype=q.dtype, device=dev)
+        l_parts = torch.empty((n, 1, H, S), dtype=torch.float32, device=dev)
+        bounds = [S * i // n // 128 * 128 for i in range(n)] + [S]
+        ks = [k[:, :, bounds[i]:bounds[i + 1]].contiguous() for i in range(n)]
+        vs = [v[:, :, bounds[i]:bounds[i + 1]].contiguous() for i in range(n)]
+        scale = D ** -0.5
+
+        def partials():
+            for i in range(n):
+                api.attn_fwd_partial(q, ks[i], vs[i], scale, True, bounds[i], out=o_parts[i], lse=l_parts[i])
+
+        t_full = time_call(lambda: api.attn_fwd(q, k, v, scale, True, out=o, lse=lse), flush, args.iters)
+        t_part = time_call(partials, flush, args.iters)
+        t_merge = time_call(lambda: api.attn_combine(o_parts, l_parts, out=o, lse=lse), flush, args.iters)
+        moved = (n + 1) * H * S * (D * 2 + 4)
+        print("| %d | %.3f | %.3f | %.1f | %.0f | %.2f |" % (S, t_full, t_part, t_merge * 1e3, moved / t_merge / 1e6,
+                                                       (t_part + t_merge) / t_full), flush=True)
+    if api.attn_last_device_status() != 0:
+        raise SystemExit("device timeout status")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16", "fp8"])
     ap.add_argument("--gqa", type=int, default=0, help="number of K/V heads (0: same as query heads)")
     ap.add_argument("--iters", type=int, default=15)
     ap.add_argument("--seq", type=int, default=0, help="only this sequence length (a power of two, 512..16384)")
+    ap.add_argument("--shards", type=int, default=0, help="time N K/V shards + merge against the unsharded call")
     args = ap.parse_args()
     dt = inputs.DTYPE_BF16 if args.dtype == "bf16" else inputs.DTYPE_FP16
     dev = torch.device("cuda:0")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    if args.shards:
+        shard_table(args, dev, flush)
+        return
     seqs = [512, 1024, 2048, 4096, 8192, 16384]
     if args.seq:
         if args.seq not in seqs:

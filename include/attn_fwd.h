@@ -112,6 +112,29 @@ int attn_combine(const void* o_parts, const float* lse_parts, int n_parts, void*
                  int Sq, int D, int dtype, void* stream);
 
 /*
+ * attn_fwd_splitkv -- attn_fwd_gqa with the keys split into n_splits ranges that run as concurrent
+ * launches, followed by the merge of attn_combine: split-KV decoding in the manner of FlashDecoding,
+ * which the paper cites in its related work.  For problems with few query rows (a handful of heads,
+ * one or a few queries each) and many keys, one launch has too few work items to fill the GPU;
+ * splitting the keys gives every range its own items.  Arguments and conventions as attn_fwd_gqa,
+ * plus: n_splits in 1..64 (clamped to the number of 128-key tiles; 1 is plain attn_fwd_gqa);
+ * workspace: caller-owned DEVICE buffer of at least attn_fwd_splitkv_workspace_bytes(...) bytes,
+ * 256-byte aligned, which receives the ranges' partial results ([n_splits,B,H,Sq,D] in `dtype`, then
+ * [n_splits,B,H,Sq] fp32).  K and V are read in place (no copies).  The launches run on up to 16
+ * streams of the library's own (created with their events on the first such call on a device),
+ * ordered after the work already on `stream`; the merge runs on `stream` after all of them.
+ * The partial outputs are rounded to `dtype` before the merge, so O carries one more 16-bit rounding
+ * than attn_fwd_gqa.  Errors: as attn_fwd_gqa, plus ATTN_ERR_BAD_SHAPE for n_splits outside 1..64
+ * and ATTN_ERR_WORKSPACE.
+ */
+int attn_fwd_splitkv(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv,
+                     int Sq, int Sk, int D, float scale, int causal, int dtype, int n_splits, void* workspace,
+                     size_t workspace_bytes, void* stream);
+
+/* Bytes of device workspace attn_fwd_splitkv needs (0 for an invalid shape). */
+size_t attn_fwd_splitkv_workspace_bytes(int B, int H, int Sq, int D, int n_splits);
+
+/*
  * attn_fwd_qkv_dims -- attention whose Q/K head dim differs from its V/O head dim: the MLA head
  * shape of Section 4.1 / Table 2 (embedding dimension 128 plus RoPE dimension 64 for Q and K,
  * 128 for V).  q: [B,H,Sq,Dqk], k: [B,Hkv,Sk,Dqk], v: [B,Hkv,Sk,Dv], o: [B,H,Sq,Dv], lse: [B,H,Sq].

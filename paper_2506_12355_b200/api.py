@@ -24,7 +24,7 @@ STATUS_NAMES = {
 }
 
 # every symbol include/attn_fwd.h declares
-EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_partial", "attn_combine", "attn_fwd_qkv_dims", "attn_fwd_fp8", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
+EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_partial", "attn_combine", "attn_fwd_qkv_dims", "attn_fwd_splitkv", "attn_fwd_splitkv_workspace_bytes", "attn_fwd_fp8", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
            "attn_fwd_host_static", "attn_fwd_host_static_capacity",
            "attn_query_support", "attn_last_device_status", "attn_status_string"]
 
@@ -63,6 +63,10 @@ def load() -> ctypes.CDLL:
     lib.attn_combine.argtypes = [vp, vp, i, vp, vp, i, i, i, i, i, vp]
     lib.attn_fwd_qkv_dims.restype = i
     lib.attn_fwd_qkv_dims.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, vp]
+    lib.attn_fwd_splitkv.restype = i
+    lib.attn_fwd_splitkv.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, i, vp, ctypes.c_size_t, vp]
+    lib.attn_fwd_splitkv_workspace_bytes.restype = ctypes.c_size_t
+    lib.attn_fwd_splitkv_workspace_bytes.argtypes = [i] * 5
     lib.attn_fwd_fp8.restype = i
     lib.attn_fwd_fp8.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, f, f, f, i, i, vp]
     lib.attn_fwd_simt.restype = i
@@ -231,6 +235,38 @@ def attn_fwd_qkv_dims(q, k, v, scale: float, causal: bool = False, out=None, lse
                                       _stream_ptr(stream))
     if rc != 0:
         raise AttnError(rc, "attn_fwd_qkv_dims")
+    return out, lse
+
+
+def attn_fwd_splitkv_workspace_bytes(B, H, Sq, D, n_splits) -> int:
+    return int(load().attn_fwd_splitkv_workspace_bytes(B, H, Sq, D, n_splits))
+
+
+def attn_fwd_splitkv(q, k, v, scale: float, causal: bool, n_splits: int, workspace=None, out=None, lse=None, stream=None):
+    """attn_fwd_gqa with the keys split into n_splits ranges that run concurrently, then merged (split-KV
+    decoding).  `workspace`: CUDA uint8 tensor of at least attn_fwd_splitkv_workspace_bytes(...) bytes
+    (allocated here when None)."""
+    B, H, Sq, D = q.shape
+    Hkv, Sk = k.shape[1], k.shape[2]
+    if tuple(k.shape) != (B, Hkv, Sk, D) or tuple(v.shape) != tuple(k.shape):
+        raise ValueError("k, v must be [B,Hkv,Sk,D]")
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+        raise ValueError("q, k, v must be contiguous")
+    if not (q.is_cuda and k.is_cuda and v.is_cuda) or not (q.dtype == k.dtype == v.dtype):
+        raise ValueError("q, k, v must be CUDA tensors of one dtype")
+    dt = _dtype_code(q)
+    if workspace is None:
+        workspace = torch.empty(attn_fwd_splitkv_workspace_bytes(B, H, Sq, D, n_splits), dtype=torch.uint8, device=q.device)
+    if out is None:
+        out = torch.empty((B, H, Sq, D), dtype=q.dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(q.device):
+        rc = load().attn_fwd_splitkv(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                     B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)), dt, int(n_splits),
+                                     workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_fwd_splitkv")
     return out, lse
 
 

@@ -65,12 +65,16 @@ EncodeTiledFn get_encode_fn() {
 
 // Rank-3 map over a [BH, S, D] row-major tensor of 16-bit (dtype 0 / 1) or 8-bit (dtype 2) elements;
 // box = [1, box_rows, 128 bytes of columns], 128-byte swizzle, out-of-range rows read as zero.
-bool make_map(CUtensorMap* map, const void* base, int dtype, int64_t BH, int64_t S, int D, int box_rows) {
+// head_stride_rows: distance between consecutive (batch, head) slices in rows (S for a contiguous tensor; larger
+// when the map covers a range of rows of a bigger tensor: a K/V shard addressed in place).
+bool make_map(CUtensorMap* map, const void* base, int dtype, int64_t BH, int64_t S, int D, int box_rows,
+              int64_t head_stride_rows = -1) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
     const cuuint64_t es = dtype == ATTN_DTYPE_FP8_E4M3 ? 1 : 2;
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S), static_cast<cuuint64_t>(BH)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * es, static_cast<cuuint64_t>(S) * D * es};
+    const cuuint64_t hs = static_cast<cuuint64_t>(head_stride_rows < 0 ? S : head_stride_rows);
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * es, hs * D * es};
     cuuint32_t box[3] = {static_cast<cuuint32_t>(128 / es), static_cast<cuuint32_t>(box_rows), 1};
     cuuint32_t estr[3] = {1, 1, 1};
     const CUtensorMapDataType type = dtype == ATTN_DTYPE_FP16   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
@@ -181,7 +185,7 @@ long long* g_prof_buffer = nullptr;  // development builds only
 // Pipelined, warp-specialised kernel (head dims 64 and 128): one CTA per pair of 128-row Q tiles.
 template <int D, int DTYPE>
 int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                   float scale, int causal, int k_offset, cudaStream_t st, float o_scale = 1.f) {
+                   float scale, int causal, int k_offset, cudaStream_t st, float o_scale = 1.f, int64_t kv_stride_rows = -1) {
     constexpr int ES = DTYPE == ATTN_DTYPE_FP8_E4M3 ? 1 : 2;                 // bytes per Q/K/V element
     constexpr int ODT = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_DTYPE_BF16 : DTYPE;   // O storage type
     using C = attn_tc::PipeCfg<D, ES>;
@@ -195,8 +199,9 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     const int64_t n_pairs = (static_cast<int64_t>(Sq) + 2 * C::BM - 1) / (2 * C::BM);
     if (n_pairs * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
     CUtensorMap mq, mk, mv, mo;
-    if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) || !make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) ||
-        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN) || !make_map(&mo, o, ODT, BH, Sq, D, C::BM))
+    if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) ||
+        !make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN, kv_stride_rows) ||
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN, kv_stride_rows) || !make_map(&mo, o, ODT, BH, Sq, D, C::BM))
         return ATTN_ERR_CUDA;
     attn_tc::PipeParams prm;
     prm.o = o;
@@ -248,7 +253,7 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
 // One Q tile per CTA, Q in tensor memory, double-buffered S: head dim 256 and the 192/128 head shape.
 template <int DQK, int DV, int BN, int DTYPE>
 int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                    float scale, int causal, int k_offset, cudaStream_t st) {
+                    float scale, int causal, int k_offset, cudaStream_t st, int64_t kv_stride_rows = -1) {
     using C = attn_tc::QTmemCfg<DQK, DV, BN>;
     auto kern = attn_tc::attn_fwd_tc_qtmem_kernel<DQK, DV, BN, DTYPE>;
     if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), C::SMEM_BYTES)) return ATTN_ERR_CUDA;
@@ -256,8 +261,8 @@ int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float*
     const int64_t n_qtiles = (static_cast<int64_t>(Sq) + C::BM - 1) / C::BM;
     if (n_qtiles * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
     CUtensorMap mk, mv, mo;
-    if (!make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, DQK, C::BN) ||
-        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, DV, C::BN) || !make_map(&mo, o, DTYPE, BH, Sq, DV, C::BM))
+    if (!make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, DQK, C::BN, kv_stride_rows) ||
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, DV, C::BN, kv_stride_rows) || !make_map(&mo, o, DTYPE, BH, Sq, DV, C::BM))
         return ATTN_ERR_CUDA;
     attn_tc::QTmemParams prm;
     prm.q = q;
@@ -314,7 +319,7 @@ enum class Impl { TensorCore, Simt };
 
 template <Impl IMPL>
 int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk, int D,
-             float scale, int causal, int k_offset, int dtype, void* stream) {
+             float scale, int causal, int k_offset, int dtype, void* stream, int64_t kv_stride_rows = -1) {
     int rc = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, dtype, true);
     if (rc != ATTN_OK) return rc;
     if (k_offset < 0 || static_cast<int64_t>(k_offset) + Sk > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
@@ -324,11 +329,20 @@ int dispatch(const void* q, const void* k, const void* v, void* o, float* lse, i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (Sk == 0)
         return fill_empty(o, lse, static_cast<int64_t>(B) * H * Sq * D, static_cast<int64_t>(B) * H * Sq, st);
+    // Grouped K/V heads without a mask and with few query rows per head (decoding, short chunks): the H / Hkv
+    // query heads of one K/V head lie next to each other in Q, O and LSE, so they ARE one head of (H / Hkv) * Sq
+    // rows over the same keys.  Taken that way they share Q tiles (one tile of 128 rows instead of H / Hkv
+    // tiles with Sq valid rows each) and K/V is streamed once for the group.
+    if (IMPL == Impl::TensorCore && !causal && Hkv < H && Sq < 256 &&
+        static_cast<int64_t>(H / Hkv) * Sq <= 2147483647LL - 256) {
+        Sq *= H / Hkv;
+        H = Hkv;
+    }
 #define ATTN_CASE(DD, TT)                                                                              \
     if (D == DD && dtype == TT) {                                                                      \
         if (IMPL == Impl::Simt) return launch_simt<DD, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, k_offset, st); \
-        if (DD == 256) return launch_tc_qtmem<256, 256, 64, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, k_offset, st); \
-        return launch_tc_pipe<(DD == 256 ? 128 : DD), TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, k_offset, st); \
+        if (DD == 256) return launch_tc_qtmem<256, 256, 64, TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, k_offset, st, kv_stride_rows); \
+        return launch_tc_pipe<(DD == 256 ? 128 : DD), TT>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, scale, causal, k_offset, st, 1.f, kv_stride_rows); \
     }
     ATTN_CASE(64, 0)
     ATTN_CASE(64, 1)
@@ -383,6 +397,16 @@ struct HostPipe {
     std::mutex mu;   // one enqueue sequence at a time: the events are shared by every call on the device
 };
 HostPipe g_host_pipe[64];
+
+// ---- attn_fwd_splitkv: the K/V shards of one problem as concurrent launches on internal streams ----
+constexpr int kSplitStreams = 16;
+struct SplitPipe {
+    bool ready = false;
+    cudaStream_t s[kSplitStreams] = {};
+    cudaEvent_t ev_start = nullptr, ev_done[kSplitStreams] = {};
+    std::mutex mu;
+};
+SplitPipe g_split_pipe[64];
 
 // at least 16 MiB to copy in (more than the built-in buffer of attn_fwd_host_static can hold, so that entry point
 // never takes this path and keeps its promise to create nothing) and at least 4 heads to split
@@ -497,6 +521,68 @@ int attn_combine(const void* o_parts, const float* lse_parts, int n_parts, void*
     }
 #undef ATTN_COMBINE
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+size_t attn_fwd_splitkv_workspace_bytes(int B, int H, int Sq, int D, int n_splits) {
+    if (B < 0 || H < 0 || Sq < 0 || D <= 0 || n_splits < 1) return 0;
+    const size_t rows = static_cast<size_t>(B) * H * Sq;
+    return align256(static_cast<size_t>(n_splits) * rows * D * 2) + align256(static_cast<size_t>(n_splits) * rows * 4);
+}
+
+int attn_fwd_splitkv(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
+                     int D, float scale, int causal, int dtype, int n_splits, void* workspace, size_t workspace_bytes,
+                     void* stream) {
+    int rc = validate(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, dtype, true);
+    if (rc != ATTN_OK) return rc;
+    if (n_splits < 1 || n_splits > 64) return ATTN_ERR_BAD_SHAPE;
+    const size_t rows = static_cast<size_t>(B) * H * Sq;
+    if (rows == 0) return ATTN_OK;
+    // shards are whole 128-key tiles; no more shards than tiles
+    const int tiles = (Sk + 127) / 128;
+    if (n_splits > tiles) n_splits = tiles > 0 ? tiles : 1;
+    if (n_splits == 1 || Sk == 0) return attn_fwd_gqa(q, k, v, o, lse, B, H, Hkv, Sq, Sk, D, scale, causal, dtype, stream);
+    // partial results as attn_combine reads them: [n_splits, rows, D] 16-bit, then [n_splits, rows] fp32
+    const size_t part_o = rows * D * 2, part_l = rows * 4;
+    const size_t o_all = align256(static_cast<size_t>(n_splits) * part_o), l_all = align256(static_cast<size_t>(n_splits) * part_l);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < o_all + l_all)
+        return ATTN_ERR_WORKSPACE;
+    rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ATTN_ERR_CUDA;
+    SplitPipe& sp = g_split_pipe[dev];
+    std::lock_guard<std::mutex> lock(sp.mu);
+    if (!sp.ready) {
+        bool ok = cudaEventCreateWithFlags(&sp.ev_start, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < kSplitStreams; ++i)
+            ok = cudaStreamCreateWithFlags(&sp.s[i], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&sp.ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return ATTN_ERR_CUDA;
+        sp.ready = true;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* w_o = static_cast<uint8_t*>(workspace);
+    uint8_t* w_l = w_o + o_all;
+    const int n_streams = n_splits < kSplitStreams ? n_splits : kSplitStreams;
+    if (cudaEventRecord(sp.ev_start, st) != cudaSuccess) return ATTN_ERR_CUDA;
+    for (int i = 0; i < n_streams; ++i)
+        if (cudaStreamWaitEvent(sp.s[i], sp.ev_start, 0) != cudaSuccess) return ATTN_ERR_CUDA;
+    for (int s = 0; s < n_splits; ++s) {
+        const int t0 = static_cast<int>(static_cast<int64_t>(tiles) * s / n_splits);
+        const int t1 = static_cast<int>(static_cast<int64_t>(tiles) * (s + 1) / n_splits);
+        const int k0 = t0 * 128, k1 = (t1 * 128 < Sk) ? t1 * 128 : Sk;
+        // the shard is addressed in place: rows k0 .. k1-1 of every (batch, K/V head), head stride Sk rows
+        const uint8_t* ks = static_cast<const uint8_t*>(k) + static_cast<size_t>(k0) * D * 2;
+        const uint8_t* vs = static_cast<const uint8_t*>(v) + static_cast<size_t>(k0) * D * 2;
+        rc = dispatch<Impl::TensorCore>(q, ks, vs, w_o + s * part_o, reinterpret_cast<float*>(w_l + s * part_l), B, H, Hkv, Sq,
+                                        k1 - k0, D, scale, causal, k0, dtype, sp.s[s % n_streams], Sk);
+        if (rc != ATTN_OK) return rc;
+    }
+    for (int i = 0; i < n_streams; ++i) {
+        if (cudaEventRecord(sp.ev_done[i], sp.s[i]) != cudaSuccess) return ATTN_ERR_CUDA;
+        if (cudaStreamWaitEvent(st, sp.ev_done[i], 0) != cudaSuccess) return ATTN_ERR_CUDA;
+    }
+    return attn_combine(w_o, reinterpret_cast<const float*>(w_l), n_splits, o, lse, B, H, Sq, D, dtype, stream);
 }
 
 int attn_fwd_qkv_dims(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq,

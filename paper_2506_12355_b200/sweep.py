@@ -1,6 +1,6 @@
 """Throughput sweep over the benchmark grid of the paper's Section 4.1.
 
-    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16|fp8] [--gqa Hkv] [--iters N] [--seq S] [--shards N]
+    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16|fp8] [--gqa Hkv] [--iters N] [--seq S] [--shards N] [--decode]
 
 Grid: sequence length 512 .. 16k with the batch chosen so that batch x sequence = 16k tokens,
 hidden size 2048 (32 heads of dim 64 or 16 heads of dim 128), with and without the causal mask; in
@@ -15,6 +15,10 @@ timed with CUDA events over isolated launches with a buffer larger than L2 rewri
 sharding across GPUs): N partial launches over N key ranges of one problem (causal, 32 heads of dim
 128, bf16) and the merge of their results, against the unsharded call; the merge kernel is
 memory-bound and is reported in GB/s of the bytes it must move.
+
+`--decode` times decoding shapes (one query per head, long key/value cache, bf16, head dim 128) through
+`attn_fwd_splitkv` for several numbers of key ranges: with one query row per head the work is reading K
+and V once, so the figure of merit is GB/s of K and V bytes against the memory bandwidth.
 """
 from __future__ import annotations
 
@@ -73,6 +77,32 @@ def shard_table(args, dev, flush):
         raise SystemExit("device timeout status")
 
 
+def decode_table(args, dev, flush):
+    D, dt = 128, inputs.DTYPE_BF16
+    splits = [1, 2, 4, 8, 16, 32]
+    print("| batch x heads (K/V heads) x keys | K+V MB | " + " | ".join("%d ranges: us (GB/s)" % n for n in splits) + " |")
+    print("|---|---|" + "---|" * len(splits))
+    for (B, H, Hkv, Sk) in ((1, 32, 8, 16384), (1, 32, 8, 65536), (1, 32, 32, 65536), (8, 32, 8, 16384)):
+        if args.seq and Sk != args.seq:
+            continue
+        q = inputs.randn16((B, H, 1, D), 1, dt).to(dev)
+        k = inputs.randn16((B, Hkv, Sk, D), 2, dt).to(dev)
+        v = inputs.randn16((B, Hkv, Sk, D), 3, dt).to(dev)
+        o = torch.empty_like(q)
+        lse = torch.empty((B, H, 1), dtype=torch.float32, device=dev)
+        ws = torch.empty(api.attn_fwd_splitkv_workspace_bytes(B, H, 1, D, max(splits)), dtype=torch.uint8, device=dev)
+        kv_bytes = 2.0 * B * Hkv * Sk * D * 2
+        cells = []
+        for n in splits:
+            ms = time_call(lambda: api.attn_fwd_splitkv(q, k, v, D ** -0.5, False, n, workspace=ws, out=o, lse=lse),
+                           flush, args.iters)
+            cells.append("%.0f (%.0f)" % (ms * 1e3, kv_bytes / ms / 1e6))
+        print("| %d x %d (%d) x %d | %.0f | %s |" % (B, H, Hkv, Sk, kv_bytes / 1e6, " | ".join(cells)), flush=True)
+        del q, k, v, o, lse, ws
+    if api.attn_last_device_status() != 0:
+        raise SystemExit("device timeout status")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16", "fp8"])
@@ -80,12 +110,16 @@ def main():
     ap.add_argument("--iters", type=int, default=15)
     ap.add_argument("--seq", type=int, default=0, help="only this sequence length (a power of two, 512..16384)")
     ap.add_argument("--shards", type=int, default=0, help="time N K/V shards + merge against the unsharded call")
+    ap.add_argument("--decode", action="store_true", help="decoding shapes through attn_fwd_splitkv")
     args = ap.parse_args()
     dt = inputs.DTYPE_BF16 if args.dtype == "bf16" else inputs.DTYPE_FP16
     dev = torch.device("cuda:0")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     if args.shards:
         shard_table(args, dev, flush)
+        return
+    if args.decode:
+        decode_table(args, dev, flush)
         return
     seqs = [512, 1024, 2048, 4096, 8192, 16384]
     if args.seq:

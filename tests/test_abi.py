@@ -98,6 +98,23 @@ def test_fp8_entry_validation(lib):
     assert f8() in (7, 8) or True               # valid arguments reach the device check (no device here: 7 or 8)
 
 
+def test_splitkv_entry_validation(lib):
+    lib.attn_fwd_splitkv_workspace_bytes.restype = __import__("ctypes").c_size_t
+    assert lib.attn_fwd_splitkv_workspace_bytes(1, 4, 3, 128, 6) == (6 * 12 * 128 * 2 + 255) // 256 * 256 + (6 * 12 * 4 + 255) // 256 * 256
+    assert lib.attn_fwd_splitkv_workspace_bytes(1, 4, 3, 128, 0) == 0
+    args = [0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 1, 4, 2, 3, 4096, 128, 0.1, 0, 1]
+    assert lib.attn_fwd_splitkv(*args, 0, 0x10000, 1 << 30, None) == 2      # n_splits out of range
+    assert lib.attn_fwd_splitkv(*args, 65, 0x10000, 1 << 30, None) == 2
+    assert lib.attn_fwd_splitkv(*args, 4, None, 0, None) == 10              # no workspace
+    assert lib.attn_fwd_splitkv(*args, 4, 0x10010, 1 << 30, None) == 10     # misaligned
+    bad = list(args)
+    bad[7] = 3                                                              # H % Hkv != 0
+    assert lib.attn_fwd_splitkv(*bad, 4, 0x10000, 1 << 30, None) == 2
+    bad = list(args)
+    bad[8] = 0                                                              # no query rows: nothing to do
+    assert lib.attn_fwd_splitkv(*bad, 4, None, 0, None) == 0
+
+
 def test_host_entry_validation(lib):
     n = lib.attn_fwd_host_workspace_bytes(2, 3, 100, 50, 64)
     qo = (2 * 3 * 100 * 64 * 2 + 255) // 256 * 256

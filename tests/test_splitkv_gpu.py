@@ -71,3 +71,27 @@ def test_splitkv_rejects_bad_arguments():
     with pytest.raises(api.AttnError) as e:
         api.attn_fwd_splitkv(qd, kd, vd, 0.1, False, 4, workspace=torch.empty(256, dtype=torch.uint8, device=dev))
     assert e.value.status == 10
+
+
+def test_splitkv_in_a_cuda_graph():
+    # the concurrent launches on the library's own streams fork from and join the capturing stream, so the whole
+    # call (counter resets, partial launches, merge) is one graph; a decoding loop replays it
+    dev = torch.device("cuda:0")
+    q, k, v = inputs.make_qkv(1, 8, 1, 8192, 128, 1, seed=8600)
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    ws = torch.empty(api.attn_fwd_splitkv_workspace_bytes(1, 8, 1, 128, 8), dtype=torch.uint8, device=dev)
+    ref_o, ref_l = api.attn_fwd_splitkv(qd, kd, vd, 0.09, False, 8, workspace=ws)   # one-time set-up outside capture
+    torch.cuda.synchronize()
+    o = torch.empty_like(ref_o)
+    lse = torch.empty_like(ref_l)
+    g = torch.cuda.CUDAGraph()
+    st = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            api.attn_fwd_splitkv(qd, kd, vd, 0.09, False, 8, workspace=ws, out=o, lse=lse, stream=st)
+    for _ in range(3):
+        o.zero_()
+        g.replay()
+    torch.cuda.synchronize()
+    assert api.attn_last_device_status() == 0
+    assert torch.equal(o.view(torch.int16), ref_o.view(torch.int16)) and torch.equal(lse, ref_l)

@@ -10,7 +10,7 @@
  * exp2, no blocking.  FlashAttention-style kernels are an exact reformulation
  * of this (up to rounding order), so the definition is the oracle.
  *
- * Readings where the paper is silent (each is stated again in the design notes):
+ * Readings where the paper is silent:
  *   - scale is an explicit argument (the paper uses 1/sqrt(d));
  *   - the causal mask is lower-triangular including the diagonal and aligned
  *     to the top-left corner: key j is visible to query i iff j <= i, also

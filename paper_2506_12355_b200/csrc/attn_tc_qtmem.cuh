@@ -39,8 +39,8 @@ struct QTmemCfg {
     static constexpr int K_BYTES = BN * DQK * 2;                // one K tile
     static constexpr int V_BYTES = BN * DV * 2;                 // one V tile
     static constexpr int SLOT_BYTES = K_BYTES > V_BYTES ? K_BYTES : V_BYTES;
-    static constexpr int OST_BYTES = BM * 128;                  // epilogue staging: 128 rows x 64 columns
-    static constexpr int NSLOT = (208 * 1024) / SLOT_BYTES > 6 ? 6 : (208 * 1024) / SLOT_BYTES;
+    static constexpr int OST_BYTES = 2 * BM * 128;              // epilogue staging: two tiles of 128 rows x 64 columns
+    static constexpr int NSLOT = (192 * 1024) / SLOT_BYTES > 6 ? 6 : (192 * 1024) / SLOT_BYTES;
     static constexpr int TILE_BYTES = NSLOT * SLOT_BYTES + OST_BYTES;
     static constexpr int MISC_BYTES = 512;
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
@@ -199,6 +199,13 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
                     e[2] = d.kv_bh;
                     e[3] = d.q0;
                     e[4] = d.n;
+                    // its Q tile (rows q0 .. of one head: one contiguous block) on its way into L2 now, so that the
+                    // softmax threads' loads of it, a few steps from now, do not pay the latency of HBM
+                    if (k > 0 && d.n > 0) {
+                        const int nrows = prm.Sq - d.q0 < BM ? prm.Sq - d.q0 : BM;
+                        bulk_prefetch_l2(static_cast<const uint8_t*>(prm.q) + (static_cast<int64_t>(d.bh) * prm.Sq + d.q0) * DQK * 2,
+                                         static_cast<uint32_t>(nrows) * DQK * 2);
+                    }
                 }
                 e[0] = next;
                 mbar_arrive(bar(B_SCHEDFULL + slot));
@@ -301,22 +308,55 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 
         // Q row of an item -> tensor memory (two 16-bit values per column, in memory order)
         auto load_q = [&](const QTmemItem& it) {
-            const int qrow_idx = it.q0 + r;
-            const uint4* qrow = reinterpret_cast<const uint4*>(
-                static_cast<const uint8_t*>(prm.q) + (static_cast<int64_t>(it.bh) * prm.Sq + qrow_idx) * DQK * 2);
+            // Coalesced: a warp reads its 32 rows 128 columns at a time, every instruction covering whole rows
+            // (consecutive lanes take consecutive 16-byte chunks), parks them in its own 8 KB of the epilogue's
+            // staging tiles, and each thread then picks up its row from there (swizzled by row: no bank
+            // conflicts either way).  One row per thread straight from global memory would touch 32 lines per
+            // instruction.  The staging tiles are free once the previous epilogue's stores have read them.
+            if (r == 0) tma_store_wait_read<0>();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const uint32_t mine = sOst + warp * 8192;
+            const int rows_left = prm.Sq - (it.q0 + warp * 32);   // rows of this warp that exist
+            const uint8_t* qbase = static_cast<const uint8_t*>(prm.q) +
+                                   (static_cast<int64_t>(it.bh) * prm.Sq + it.q0 + warp * 32) * DQK * 2;
 #pragma unroll
-            for (int ch = 0; ch < DQK / 64; ++ch) {   // 32 columns = 64 elements = 8 x 16 bytes per chunk
-                uint32_t w[32];
+            for (int c0 = 0; c0 < DQK / 8; c0 += 16) {   // 16-byte chunks of a row, at most 16 per round
+                constexpr int TOTAL = DQK / 8;
+                const int CH = TOTAL - c0 < 16 ? TOTAL - c0 : 16;   // 16 or 8 (compile-time after unrolling)
+                const int RPI = 32 / CH;                            // rows per load instruction
+                uint4 x[16];
 #pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    uint4 x = make_uint4(0u, 0u, 0u, 0u);
-                    if (qrow_idx < prm.Sq) x = __ldg(qrow + ch * 8 + g);
-                    w[g * 4 + 0] = x.x;
-                    w[g * 4 + 1] = x.y;
-                    w[g * 4 + 2] = x.z;
-                    w[g * 4 + 3] = x.w;
+                for (int i = 0; i < 16; ++i) {
+                    if (i < CH) {
+                        const int row_l = i * RPI + lane / CH, ch = lane % CH;
+                        x[i] = (row_l < rows_left)
+                                   ? __ldg(reinterpret_cast<const uint4*>(qbase + static_cast<int64_t>(row_l) * DQK * 2 + (c0 + ch) * 16))
+                                   : make_uint4(0u, 0u, 0u, 0u);
+                    }
                 }
-                tmem_st_32x32b_x32(tQ + ch * 32, w);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    if (i < CH) {
+                        const int row_l = i * RPI + lane / CH, ch = lane % CH;
+                        const uint32_t dst = mine + row_l * 256 + ((ch ^ (row_l & (CH - 1))) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(x[i].x), "r"(x[i].y), "r"(x[i].z), "r"(x[i].w) : "memory");
+                    }
+                }
+                __syncwarp();
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {   // 8 chunks = 32 tensor-memory columns per store
+                    if (half * 8 < CH) {
+                        uint32_t w[32];
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const uint32_t src = mine + lane * 256 + (((half * 8 + g) ^ (lane & (CH - 1))) << 4);
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(w[g * 4 + 0]), "=r"(w[g * 4 + 1]), "=r"(w[g * 4 + 2]), "=r"(w[g * 4 + 3]) : "r"(src) : "memory");
+                        }
+                        tmem_st_32x32b_x32(tQ + (c0 + half * 8) * 4, w);
+                    }
+                }
+                __syncwarp();
             }
             tmem_st_wait();
             tc_fence_before_sync();
@@ -520,7 +560,8 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
                         tc_fence_before_sync();
                         mbar_arrive(bar(B_OFREE));
                     }
-                    if (r == 0) tma_store_wait_read<0>();          // the previous store has read the staging tile
+                    const uint32_t ost = sOst + (h & 1) * (BM * 128);   // two staging tiles take turns
+                    if (r == 0) tma_store_wait_read<1>();          // the store before the previous one has read this tile
                     asm volatile("bar.sync 1, 128;" ::: "memory");
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
@@ -528,13 +569,13 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
                         const uint32_t w1 = pack2<DTYPE>(__uint_as_float(orr[e * 8 + 2]) * inv, __uint_as_float(orr[e * 8 + 3]) * inv);
                         const uint32_t w2 = pack2<DTYPE>(__uint_as_float(orr[e * 8 + 4]) * inv, __uint_as_float(orr[e * 8 + 5]) * inv);
                         const uint32_t w3 = pack2<DTYPE>(__uint_as_float(orr[e * 8 + 6]) * inv, __uint_as_float(orr[e * 8 + 7]) * inv);
-                        const uint32_t dst = sOst + r * 128 + ((e ^ (r & 7)) << 4);   // 128-byte swizzle
+                        const uint32_t dst = ost + r * 128 + ((e ^ (r & 7)) << 4);   // 128-byte swizzle
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
                     }
                     fence_proxy_async_smem();
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                     if (r == 0) {
-                        tma_store_3d(&tmO, sOst, h * 64, q0, bh);
+                        tma_store_3d(&tmO, ost, h * 64, q0, bh);
                         tma_store_commit();
                     }
                 }

@@ -1,6 +1,6 @@
 """Throughput sweep over the benchmark grid of the paper's Section 4.1.
 
-    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16|fp8] [--gqa Hkv] [--iters N] [--seq S] [--shards N] [--decode]
+    python -m paper_2506_12355_b200.sweep [--dtype bf16|fp16|fp8] [--gqa Hkv] [--iters N] [--seq S] [--shards N] [--decode] [--configs]
 
 Grid: sequence length 512 .. 16k with the batch chosen so that batch x sequence = 16k tokens,
 hidden size 2048 (32 heads of dim 64 or 16 heads of dim 128), with and without the causal mask; in
@@ -15,6 +15,8 @@ timed with CUDA events over isolated launches with a buffer larger than L2 rewri
 sharding across GPUs): N partial launches over N key ranges of one problem (causal, 32 heads of dim
 128, bf16) and the merge of their results, against the unsharded call; the merge kernel is
 memory-bound and is reported in GB/s of the bytes it must move.
+
+`--configs` times the five benchmark configurations C1..C5 the same way (isolated launches, L2 flushed).
 
 `--decode` times decoding shapes (one query per head, long key/value cache, bf16, head dim 128) through
 `attn_fwd_splitkv` for several numbers of key ranges: with one query row per head the work is reading K
@@ -111,6 +113,7 @@ def main():
     ap.add_argument("--seq", type=int, default=0, help="only this sequence length (a power of two, 512..16384)")
     ap.add_argument("--shards", type=int, default=0, help="time N K/V shards + merge against the unsharded call")
     ap.add_argument("--decode", action="store_true", help="decoding shapes through attn_fwd_splitkv")
+    ap.add_argument("--configs", action="store_true", help="the benchmark configurations C1..C5, isolated launches")
     args = ap.parse_args()
     dt = inputs.DTYPE_BF16 if args.dtype == "bf16" else inputs.DTYPE_FP16
     dev = torch.device("cuda:0")
@@ -120,6 +123,20 @@ def main():
         return
     if args.decode:
         decode_table(args, dev, flush)
+        return
+    if args.configs:
+        print("| config | time | TFLOP/s | GB/s at algorithmic bytes |")
+        print("|---|---|---|---|")
+        for name in sorted(inputs.CONFIGS):
+            cfg = inputs.CONFIGS[name]
+            q, k, v = (t.to(dev) for t in inputs.make_config_inputs(cfg))
+            o = torch.empty_like(q)
+            lse = torch.empty((cfg.B, cfg.H, cfg.Sq), dtype=torch.float32, device=dev)
+            ms = time_call(lambda: api.attn_fwd(q, k, v, cfg.scale, cfg.causal, out=o, lse=lse), flush, max(args.iters, 30))
+            print("| %s | %.1f us | %.1f | %.0f |" % (cfg.workload, ms * 1e3, cfg.flops / ms / 1e9, cfg.min_hbm_bytes / ms / 1e6), flush=True)
+            del q, k, v, o, lse
+        if api.attn_last_device_status() != 0:
+            raise SystemExit("device timeout status")
         return
     seqs = [512, 1024, 2048, 4096, 8192, 16384]
     if args.seq:

@@ -112,17 +112,19 @@ int attn_combine(const void* o_parts, const float* lse_parts, int n_parts, void*
                  int Sq, int D, int dtype, void* stream);
 
 /*
- * attn_fwd_splitkv -- attn_fwd_gqa with the keys split into n_splits ranges that run as concurrent
- * launches, followed by the merge of attn_combine: split-KV decoding in the manner of FlashDecoding,
+ * attn_fwd_splitkv -- attn_fwd_gqa with the keys split into n_splits ranges that are computed side by
+ * side, followed by the merge of attn_combine: split-KV decoding in the manner of FlashDecoding,
  * which the paper cites in its related work.  For problems with few query rows (a handful of heads,
  * one or a few queries each) and many keys, one launch has too few work items to fill the GPU;
  * splitting the keys gives every range its own items.  Arguments and conventions as attn_fwd_gqa,
  * plus: n_splits in 1..64 (clamped to the number of 128-key tiles; 1 is plain attn_fwd_gqa);
  * workspace: caller-owned DEVICE buffer of at least attn_fwd_splitkv_workspace_bytes(...) bytes,
  * 256-byte aligned, which receives the ranges' partial results ([n_splits,B,H,Sq,D] in `dtype`, then
- * [n_splits,B,H,Sq] fp32).  K and V are read in place (no copies).  The launches run on up to 16
- * streams of the library's own (created with their events on the first such call on a device),
- * ordered after the work already on `stream`; the merge runs on `stream` after all of them.
+ * [n_splits,B,H,Sq] fp32).  K and V are read in place (no copies).  For head dims 64 and 128 the key
+ * ranges are work items of ONE launch of the persistent kernel on `stream`; for head dim 256 they
+ * are one launch each, on up to 16 streams of the library's own (created with their events on the
+ * first such call on a device), ordered after the work already on `stream`.  The merge runs on
+ * `stream` after them.
  * The partial outputs are rounded to `dtype` before the merge, so O carries one more 16-bit rounding
  * than attn_fwd_gqa.  Errors: as attn_fwd_gqa, plus ATTN_ERR_BAD_SHAPE for n_splits outside 1..64
  * and ATTN_ERR_WORKSPACE.

@@ -185,7 +185,10 @@ long long* g_prof_buffer = nullptr;  // development builds only
 // Pipelined, warp-specialised kernel (head dims 64 and 128): one CTA per pair of 128-row Q tiles.
 template <int D, int DTYPE>
 int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Hkv, int Sq, int Sk,
-                   float scale, int causal, int k_offset, cudaStream_t st, float o_scale = 1.f, int64_t kv_stride_rows = -1) {
+                   float scale, int causal, int k_offset, cudaStream_t st, float o_scale = 1.f, int64_t kv_stride_rows = -1,
+                   int n_splits = 1) {
+    // n_splits > 1: the keys are cut into n_splits ranges of whole tiles; range s of a head is a work item of its own
+    // and writes its partial result as head s * (B * H) + bh of o and lse, which then hold n_splits partial results
     constexpr int ES = DTYPE == ATTN_DTYPE_FP8_E4M3 ? 1 : 2;                 // bytes per Q/K/V element
     constexpr int ODT = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_DTYPE_BF16 : DTYPE;   // O storage type
     using C = attn_tc::PipeCfg<D, ES>;
@@ -193,15 +196,16 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     // head dim 64, where the tensor core leaves more issue slots to the softmax warps
     constexpr int PN = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_FP8_POLY_NUM : (D == 64 ? ATTN_POLY64_NUM : ATTN_POLY_NUM);
     constexpr int PD = DTYPE == ATTN_DTYPE_FP8_E4M3 ? ATTN_FP8_POLY_DEN : (D == 64 ? ATTN_POLY64_DEN : ATTN_POLY_DEN);
-    auto kern = attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE, PN, PD>;
+    auto kern = n_splits > 1 ? attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE, PN, PD, true> : attn_tc::attn_fwd_tc_pipe_kernel<D, DTYPE, PN, PD, false>;
     if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), C::SMEM_BYTES)) return ATTN_ERR_CUDA;
     const int64_t BH = static_cast<int64_t>(B) * H;
     const int64_t n_pairs = (static_cast<int64_t>(Sq) + 2 * C::BM - 1) / (2 * C::BM);
-    if (n_pairs * BH > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
+    if (n_pairs * BH * n_splits > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
     CUtensorMap mq, mk, mv, mo;
     if (!make_map(&mq, q, DTYPE, BH, Sq, D, C::BM) ||
         !make_map(&mk, k, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN, kv_stride_rows) ||
-        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN, kv_stride_rows) || !make_map(&mo, o, ODT, BH, Sq, D, C::BM))
+        !make_map(&mv, v, DTYPE, static_cast<int64_t>(B) * Hkv, Sk, D, C::BN, kv_stride_rows) ||
+        !make_map(&mo, o, ODT, BH * n_splits, Sq, D, C::BM))
         return ATTN_ERR_CUDA;
     attn_tc::PipeParams prm;
     prm.o = o;
@@ -232,7 +236,12 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
         const int64_t n_groups = (BH + hpg - 1) / hpg;
         prm.last_group = static_cast<int>(n_groups >= ATTN_MERGE_LAST ? n_groups - ATTN_MERGE_LAST : 0);
     }
-    prm.n_items = static_cast<int>(n_pairs * BH);
+    prm.n_items = static_cast<int>(n_pairs * BH * n_splits);
+    prm.n_splits = n_splits;
+    {
+        const int tiles = (Sk + C::BN - 1) / C::BN;
+        prm.split_tiles = n_splits > 1 ? (tiles + n_splits - 1) / n_splits : 2147483647 / 2;
+    }
 #ifdef ATTN_TC_PROFILE
     prm.prof = g_prof_buffer;
 #endif
@@ -548,6 +557,31 @@ int attn_fwd_splitkv(const void* q, const void* k, const void* v, void* o, float
         return ATTN_ERR_WORKSPACE;
     rc = check_arch();
     if (rc != ATTN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* w_o = static_cast<uint8_t*>(workspace);
+    uint8_t* w_l = w_o + o_all;
+    if (D == 64 || D == 128) {
+        // one launch: the key ranges are work items of the persistent kernel (no internal streams needed)
+        const int split_tiles = (tiles + n_splits - 1) / n_splits;
+        n_splits = (tiles + split_tiles - 1) / split_tiles;   // ranges that are not empty
+        int Hq = H, Sqq = Sq;
+        if (!causal && Hkv < H && Sq < 256) {                 // grouped query heads as rows of one head (see dispatch)
+            Sqq = Sq * (H / Hkv);
+            Hq = Hkv;
+        }
+        float* pl = reinterpret_cast<float*>(w_l);
+#define ATTN_SPLIT_CASE(DD, TT)                                                                                          \
+    if (D == DD && dtype == TT)                                                                                          \
+        rc = launch_tc_pipe<DD, TT>(q, k, v, w_o, pl, B, Hq, Hkv, Sqq, Sk, scale, causal, 0, st, 1.f, -1, n_splits);
+        ATTN_SPLIT_CASE(64, 0)
+        ATTN_SPLIT_CASE(64, 1)
+        ATTN_SPLIT_CASE(128, 0)
+        ATTN_SPLIT_CASE(128, 1)
+#undef ATTN_SPLIT_CASE
+        if (rc != ATTN_OK) return rc;
+        return attn_combine(w_o, pl, n_splits, o, lse, B, H, Sq, D, dtype, stream);
+    }
+    // head dim 256: one launch per key range, concurrent on the library's own streams
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ATTN_ERR_CUDA;
     SplitPipe& sp = g_split_pipe[dev];
@@ -560,9 +594,6 @@ int attn_fwd_splitkv(const void* q, const void* k, const void* v, void* o, float
         if (!ok) return ATTN_ERR_CUDA;
         sp.ready = true;
     }
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    uint8_t* w_o = static_cast<uint8_t*>(workspace);
-    uint8_t* w_l = w_o + o_all;
     const int n_streams = n_splits < kSplitStreams ? n_splits : kSplitStreams;
     if (cudaEventRecord(sp.ev_start, st) != cudaSuccess) return ATTN_ERR_CUDA;
     for (int i = 0; i < n_streams; ++i)

@@ -67,7 +67,9 @@ struct PipeParams {
     int last_group;         // index of the final group, which takes all remaining heads
     int H, Hkv;             // query heads and key/value heads per batch element (H % Hkv == 0)
     int k_offset;           // global index of key 0 of this K/V shard (0 for whole problems); enters the causal mask
-    int n_items;            // n_pairs * BH
+    int n_items;            // n_pairs * BH * n_splits
+    int n_splits;           // key ranges per (head, Q tile pair): 1, or more for split-KV decoding, where range s of
+    int split_tiles;        // split_tiles K/V tiles writes its partial result as head s * BH + bh of o and lse
     unsigned int* counter;  // work counter, zero at launch: item = gridDim.x + atomicAdd(counter, 1); NULL when n_items <= grid
 #ifdef ATTN_TC_PROFILE
     long long* prof;        // development builds: [grid][16] cycle sums of softmax group 1, row 0
@@ -82,12 +84,17 @@ __device__ __forceinline__ void reg_dec_service() { asm volatile("setmaxnreg.dec
 // One work item, decoded identically by every role.
 struct PipeItem {
     int bh, kv_bh, q0;
+    int k_tile0;   // first K/V tile of this item's key range (0 unless the keys are split)
+    int o_bh;      // head index of the item's rows in o and lse (bh unless the keys are split)
     int n_kv[2];   // K/V tiles each Q tile needs (0: tile beyond Sq, or no visible key)
     int n_max;
 };
 
-__device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int lin, int BM, int BN) {
+__device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int lin_all, int BM, int BN) {
     PipeItem it;
+    // the key ranges of one (head, Q tile pair) are neighbours in the item order
+    const int split = lin_all % prm.n_splits;
+    const int lin = lin_all / prm.n_splits;
     const int full_group = prm.heads_per_group * prm.n_pairs;
     int g = lin / full_group;
     if (g > prm.last_group) g = prm.last_group;
@@ -108,12 +115,20 @@ __device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int 
             const int last_key = last_visible_key(qs + BM - 1, prm.Sk, prm.causal, prm.k_offset);
             it.n_kv[t] = last_key < 0 ? 0 : last_key / BN + 1;   // 0: no row of the tile sees a key of this shard
         }
+        // the part of those tiles that lies in this item's key range
+        int in_range = it.n_kv[t] - split * prm.split_tiles;
+        if (in_range > prm.split_tiles) in_range = prm.split_tiles;
+        it.n_kv[t] = in_range < 0 ? 0 : in_range;
     }
+    it.k_tile0 = split * prm.split_tiles;
+    it.o_bh = split * prm.BH + it.bh;
     it.n_max = it.n_kv[0] > it.n_kv[1] ? it.n_kv[0] : it.n_kv[1];
     return it;
 }
 
-template <int D, int DTYPE, int POLY_NUM, int POLY_DEN>
+// SPLITS: the instance for problems whose keys are cut into ranges (split-KV decoding); the plain instance does not
+// carry the range's tile offset and output head through its loops.
+template <int D, int DTYPE, int POLY_NUM, int POLY_DEN, bool SPLITS = false>
 __global__ void __launch_bounds__(384, 1)
 attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -214,6 +229,8 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         it.q0 = e[3];
         it.n_kv[0] = e[4];
         it.n_kv[1] = e[5];
+        it.k_tile0 = SPLITS ? e[6] : 0;
+        it.o_bh = SPLITS ? e[7] : it.bh;
         it.n_max = it.n_kv[0] > it.n_kv[1] ? it.n_kv[0] : it.n_kv[1];
         if (hand_back) mbar_arrive(bar(B_SCHEDEMPTY + slot));
         return item;
@@ -247,6 +264,8 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         e[3] = d.q0;
                         e[4] = d.n_kv[0];
                         e[5] = d.n_kv[1];
+                        e[6] = d.k_tile0;
+                        e[7] = d.o_bh;
                     }
                     e[0] = next;
                     mbar_arrive(bar(B_SCHEDFULL + slot));
@@ -279,7 +298,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         mbar_arrive_expect_tx(bar(B_KVFULL + s), C::KV_BYTES);
 #pragma unroll
                         for (int bx = 0; bx < NBOX; ++bx)
-                            tma_load_3d(sKV(s) + bx * BN * 128, map, bar(B_KVFULL + s), bx * C::BOX_COLS, j * BN, it.kv_bh);
+                            tma_load_3d(sKV(s) + bx * BN * 128, map, bar(B_KVFULL + s), bx * C::BOX_COLS, (it.k_tile0 + j) * BN, it.kv_bh);
                     }
                     return true;
                 };
@@ -431,7 +450,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             if (n == 0) {
                 // beyond Sq, or (K/V shards under the causal mask) rows that see no key: O = 0, LSE = -inf
                 if (row < prm.Sq) {
-                    const int64_t grow0 = static_cast<int64_t>(it.bh) * prm.Sq + row;
+                    const int64_t grow0 = static_cast<int64_t>(it.o_bh) * prm.Sq + row;
                     uint4* orow0 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow0 * D * 2);
 #pragma unroll
                     for (int g = 0; g < D / 8; ++g) orow0[g] = make_uint4(0u, 0u, 0u, 0u);
@@ -448,7 +467,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 tc_fence_after_sync();
                 // Visibility of this K/V tile, per warp (rows 32 w .. 32 w + 31 of the Q tile): a chunk of
                 // 32 keys is FULL (every row sees all of it), EMPTY (no row sees any of it) or PARTIAL.
-                const int kv0 = j * BN;
+                const int kv0 = (it.k_tile0 + j) * BN;
                 const int lim = last_visible_key(row, prm.Sk, prm.causal, prm.k_offset);   // of this row
                 const int lim_lo = last_visible_key(row_w0, prm.Sk, prm.causal, prm.k_offset);
                 const int lim_hi = last_visible_key(row_w0 + 31, prm.Sk, prm.causal, prm.k_offset);
@@ -683,7 +702,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             // the 2^-126 floor of the polynomial exponential: they give O = 0, LSE = -inf.
             const bool seen = l > 1e-30f;
             const float inv = seen ? prm.o_scale / l : 0.f;
-            const int64_t grow = static_cast<int64_t>(it.bh) * prm.Sq + row;
+            const int64_t grow = static_cast<int64_t>(it.o_bh) * prm.Sq + row;
             // O leaves through a swizzled staging tile in shared memory and a TMA store (full-line writes;
             // rows beyond Sq are clipped by the tensor map), 64 columns at a time.
             const uint32_t ost = sOst(t);
@@ -711,7 +730,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 fence_proxy_async_smem();
                 asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
                 if (r == 0) {
-                    tma_store_3d(&tmO, ost, h * 64, q0 + t * BM, it.bh);
+                    tma_store_3d(&tmO, ost, h * 64, q0 + t * BM, it.o_bh);
                     tma_store_commit();
                 }
             }

@@ -112,6 +112,22 @@ int attn_combine(const void* o_parts, const float* lse_parts, int n_parts, void*
                  int Sq, int D, int dtype, void* stream);
 
 /*
+ * attn_combine_gather -- attn_combine with every shard's partial result behind its own pointer, for a range
+ * of rows: the merge step of a K/V-sharded run across GPUs as ONE kernel that reads the other ranks'
+ * partial results in place.  o_parts, lse_parts: HOST arrays of n_parts (1..32) DEVICE pointers; part r is
+ * [B,H,Sq,D] in `dtype` (16-byte aligned) and [B,H,Sq] fp32.  The pointers may refer to peer GPUs' memory
+ * (peer access enabled, or a symmetric-memory / IPC mapping): the kernel reads them with plain loads over
+ * NVLink (no TMA, no multicast), so nothing has to be all-gathered first.  row_begin, row_count: the rows of
+ * the flattened (batch, head, query) axis this call merges (a rank usually takes its own slice); o, lse:
+ * device, full-size [B,H,Sq,D] / [B,H,Sq], of which only those rows are written.  The caller orders the call
+ * after the producers of every part (a barrier across the ranks on `stream`) and keeps the parts alive until it
+ * has finished.  The pointer arrays are read before the call returns.  Errors as attn_combine, plus
+ * ATTN_ERR_BAD_SHAPE for n_parts or a row range out of bounds.
+ */
+int attn_combine_gather(const void* const* o_parts, const float* const* lse_parts, int n_parts, void* o, float* lse,
+                        int B, int H, int Sq, int D, int dtype, long long row_begin, long long row_count, void* stream);
+
+/*
  * attn_fwd_splitkv -- attn_fwd_gqa with the keys split into n_splits ranges that are computed side by
  * side, followed by the merge of attn_combine: split-KV decoding in the manner of FlashDecoding,
  * which the paper cites in its related work.  For problems with few query rows (a handful of heads,

@@ -24,7 +24,7 @@ STATUS_NAMES = {
 }
 
 # every symbol include/attn_fwd.h declares
-EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_partial", "attn_combine", "attn_fwd_qkv_dims", "attn_fwd_splitkv", "attn_fwd_splitkv_workspace_bytes", "attn_fwd_fp8", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
+EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_partial", "attn_combine", "attn_combine_gather", "attn_fwd_qkv_dims", "attn_fwd_splitkv", "attn_fwd_splitkv_workspace_bytes", "attn_fwd_fp8", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
            "attn_fwd_host_static", "attn_fwd_host_static_capacity",
            "attn_query_support", "attn_last_device_status", "attn_status_string"]
 
@@ -61,6 +61,8 @@ def load() -> ctypes.CDLL:
     lib.attn_fwd_partial.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, i, vp]
     lib.attn_combine.restype = i
     lib.attn_combine.argtypes = [vp, vp, i, vp, vp, i, i, i, i, i, vp]
+    lib.attn_combine_gather.restype = i
+    lib.attn_combine_gather.argtypes = [vp, vp, i, vp, vp, i, i, i, i, i, ctypes.c_longlong, ctypes.c_longlong, vp]
     lib.attn_fwd_qkv_dims.restype = i
     lib.attn_fwd_qkv_dims.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, vp]
     lib.attn_fwd_splitkv.restype = i
@@ -210,6 +212,29 @@ def attn_combine(o_parts, lse_parts, out=None, lse=None, stream=None):
                                  B, H, Sq, D, dt, _stream_ptr(stream))
     if rc != 0:
         raise AttnError(rc, "attn_combine")
+    return out, lse
+
+
+def attn_combine_gather(o_part_ptrs, lse_part_ptrs, shape, dtype, out, lse, row_begin=0, row_count=None, stream=None):
+    """Merge of partial results that lie behind separate device pointers (possibly peer GPUs' memory), for the
+    rows [row_begin, row_begin + row_count) of the flattened (batch, head, query) axis.  o_part_ptrs, lse_part_ptrs:
+    lists of integer device addresses; shape: (B, H, Sq, D); dtype: torch.float16 / torch.bfloat16; out, lse: full-size
+    CUDA tensors of which only those rows are written."""
+    B, H, Sq, D = shape
+    n = len(o_part_ptrs)
+    if n != len(lse_part_ptrs):
+        raise ValueError("as many O pointers as LSE pointers")
+    rows = B * H * Sq
+    if row_count is None:
+        row_count = rows - row_begin
+    o_arr = (ctypes.c_void_p * max(n, 1))(*[int(p) for p in o_part_ptrs])
+    l_arr = (ctypes.c_void_p * max(n, 1))(*[int(p) for p in lse_part_ptrs])
+    dt = DTYPE_FP16 if dtype == torch.float16 else DTYPE_BF16
+    with torch.cuda.device(out.device):
+        rc = load().attn_combine_gather(o_arr, l_arr, n, out.data_ptr(), lse.data_ptr(), B, H, Sq, D, dt,
+                                        int(row_begin), int(row_count), _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_combine_gather")
     return out, lse
 
 

@@ -532,6 +532,44 @@ int attn_combine(const void* o_parts, const float* lse_parts, int n_parts, void*
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
+int attn_combine_gather(const void* const* o_parts, const float* const* lse_parts, int n_parts, void* o, float* lse,
+                        int B, int H, int Sq, int D, int dtype, long long row_begin, long long row_count, void* stream) {
+    if (B < 0 || H < 0 || Sq < 0 || D <= 0 || n_parts < 1 || n_parts > attn_merge::kMaxGatherParts) return ATTN_ERR_BAD_SHAPE;
+    if (D % 8 != 0) return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
+    if (dtype != ATTN_DTYPE_FP16 && dtype != ATTN_DTYPE_BF16) return ATTN_ERR_UNSUPPORTED_DTYPE;
+    const int64_t rows = static_cast<int64_t>(B) * H * Sq;
+    if (row_begin < 0 || row_count < 0 || row_begin + row_count > rows) return ATTN_ERR_BAD_SHAPE;
+    if (row_count == 0) return ATTN_OK;
+    if (!o_parts || !lse_parts || !o || !lse) return ATTN_ERR_NULL_POINTER;
+    attn_merge::GatherTable tab;
+    for (int r = 0; r < attn_merge::kMaxGatherParts; ++r) {
+        const int src = r < n_parts ? r : n_parts - 1;
+        if (!o_parts[src] || !lse_parts[src]) return ATTN_ERR_NULL_POINTER;
+        if (reinterpret_cast<uintptr_t>(o_parts[src]) & 15u) return ATTN_ERR_MISALIGNED;
+        if (reinterpret_cast<uintptr_t>(lse_parts[src]) & 3u) return ATTN_ERR_MISALIGNED;
+        tab.o[r] = static_cast<const uint4*>(o_parts[src]);
+        tab.lse[r] = lse_parts[src];
+    }
+    if ((reinterpret_cast<uintptr_t>(o) & 15u) || (reinterpret_cast<uintptr_t>(lse) & 3u)) return ATTN_ERR_MISALIGNED;
+    int rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+    const int segs = D / 8;
+    const int64_t total = row_count * segs;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 64) blocks = 148 * 64;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+#define ATTN_GATHER(TT, BB)                                                                                     \
+    attn_merge::attn_combine_gather_kernel<TT, BB><<<static_cast<unsigned>(blocks), 256, 0, st>>>(                \
+        tab, n_parts, static_cast<uint4*>(o), lse, static_cast<int64_t>(row_begin), static_cast<int64_t>(row_count), segs)
+    if (dtype == ATTN_DTYPE_FP16) {
+        if (n_parts >= 3) ATTN_GATHER(0, 4); else if (n_parts == 2) ATTN_GATHER(0, 2); else ATTN_GATHER(0, 1);
+    } else {
+        if (n_parts >= 3) ATTN_GATHER(1, 4); else if (n_parts == 2) ATTN_GATHER(1, 2); else ATTN_GATHER(1, 1);
+    }
+#undef ATTN_GATHER
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
 size_t attn_fwd_splitkv_workspace_bytes(int B, int H, int Sq, int D, int n_splits) {
     if (B < 0 || H < 0 || Sq < 0 || D <= 0 || n_splits < 1) return 0;
     const size_t rows = static_cast<size_t>(B) * H * Sq;

@@ -1,9 +1,11 @@
-"""Multi-GPU plumbing: one process per GPU, no data-path collective.
+"""Multi-GPU plumbing: one process per GPU.
 
 Every (batch, head) pair is an independent attention problem, so the operator shards with
 no exchange step: a fixed problem is split by heads (`shard_heads`), and the benchmark's
-weak-scaling mode gives every rank its own batch of the same configuration.  The only
-communication is the timing protocol (a barrier and a max/sum reduction of scalars).
+weak-scaling mode gives every rank its own batch of the same configuration; the only
+communication there is the timing protocol (a barrier and a max/sum reduction of scalars).
+When heads run out, the keys are sharded instead (`kv_sharded_attention`), which has one
+exchange step: the partial results, gathered by NCCL or read in place by the merge kernel.
 """
 from __future__ import annotations
 
@@ -44,17 +46,51 @@ def shard_keys(n_keys: int, world: int, rank: int) -> tuple:
     return shard_heads(n_keys, world, rank)
 
 
-def kv_sharded_attention(q, k_shard, v_shard, scale: float, causal: bool, k_offset: int, stream=None):
+_peer_buffers = {}   # (shape, dtype, device) -> (o_buf, lse_buf, o_handle, lse_handle): rendezvous is done once per shape
+
+
+def _peer_partials(o_shape, lse_shape, dtype, device):
+    """Partial-result buffers in symmetric memory, with every rank's pointers to them (cached per shape)."""
+    import torch.distributed._symmetric_memory as symm_mem
+    key = (tuple(o_shape), dtype, str(device))
+    if key not in _peer_buffers:
+        o_buf = symm_mem.empty(tuple(o_shape), dtype=dtype, device=device)
+        l_buf = symm_mem.empty(tuple(lse_shape), dtype=torch.float32, device=device)
+        group = dist.group.WORLD
+        _peer_buffers[key] = (o_buf, l_buf, symm_mem.rendezvous(o_buf, group), symm_mem.rendezvous(l_buf, group))
+    return _peer_buffers[key]
+
+
+def kv_sharded_attention(q, k_shard, v_shard, scale: float, causal: bool, k_offset: int, stream=None,
+                         exchange: str = "nccl"):
     """Attention when every rank holds the full Q but only its own slice of the keys/values.
 
-    Each rank computes the partial result of its shard (attn_fwd_partial), the partial (O_r, LSE_r)
-    pairs are all-gathered into this GPU's own memory (NCCL; the one exchange step of this path), and
-    attn_combine merges them.  Peer memory is never read by a kernel.  Without a process group the
-    single shard is merged alone, which reproduces attn_fwd_gqa.
+    Each rank computes the partial result of its shard (attn_fwd_partial); the partial (O_r, LSE_r) pairs are
+    then merged.  exchange="nccl": they are all-gathered into this GPU's own memory (NCCL; the one exchange step
+    of this path) and attn_combine merges them; no kernel reads peer memory.  exchange="peer": the partial
+    results are written into symmetric memory and ONE kernel (attn_combine_gather) reads every rank's partial
+    result in place over NVLink with plain loads and merges: exchange and merge fused, nothing gathered first
+    (needs torch's symmetric memory and peer access between the GPUs; a barrier across the ranks on the stream
+    orders it after the partial kernels, a second one keeps the partial results alive until every rank has read
+    them).  Without a process group the single shard is merged alone, which reproduces attn_fwd_gqa.
     """
     from . import api
+    multi = dist.is_initialized() and dist.get_world_size() > 1
+    if multi and exchange == "peer":
+        B, H, Sq, D = q.shape
+        o_buf, l_buf, o_hdl, l_hdl = _peer_partials((B, H, Sq, D), (B, H, Sq), q.dtype, q.device)
+        api.attn_fwd_partial(q, k_shard, v_shard, scale, causal, k_offset, out=o_buf, lse=l_buf, stream=stream)
+        o_hdl.barrier()          # every rank's partial result is complete
+        out = torch.empty_like(o_buf)
+        lse = torch.empty_like(l_buf)
+        api.attn_combine_gather(list(o_hdl.buffer_ptrs), list(l_hdl.buffer_ptrs), (B, H, Sq, D), q.dtype, out, lse,
+                                stream=stream)
+        o_hdl.barrier()          # nobody overwrites its partial result while a peer still reads it
+        return out, lse
+    if exchange not in ("nccl", "peer"):
+        raise ValueError("exchange must be 'nccl' or 'peer'")
     o_r, lse_r = api.attn_fwd_partial(q, k_shard, v_shard, scale, causal, k_offset, stream=stream)
-    if dist.is_initialized() and dist.get_world_size() > 1:
+    if multi:
         world = dist.get_world_size()
         o_parts = torch.empty((world,) + tuple(o_r.shape), dtype=o_r.dtype, device=o_r.device)
         l_parts = torch.empty((world,) + tuple(lse_r.shape), dtype=lse_r.dtype, device=lse_r.device)

@@ -115,6 +115,22 @@ def test_splitkv_entry_validation(lib):
     assert lib.attn_fwd_splitkv(*bad, 4, None, 0, None) == 0
 
 
+def test_combine_gather_validation(lib):
+    import ctypes
+    def cg(o_ptrs, l_ptrs, n, o=0x4000, lse=0x5000, B=1, H=2, Sq=8, D=64, dtype=0, rb=0, rc=16):
+        oa = (ctypes.c_void_p * max(len(o_ptrs), 1))(*o_ptrs)
+        la = (ctypes.c_void_p * max(len(l_ptrs), 1))(*l_ptrs)
+        return lib.attn_combine_gather(oa, la, n, o, lse, B, H, Sq, D, dtype, rb, rc, None)
+    good_o, good_l = [0x1000, 0x2000], [0x3000, 0x3100]
+    assert cg(good_o, good_l, 0) == 2 and cg(good_o, good_l, 33) == 2
+    assert cg(good_o, good_l, 2, rb=10, rc=7) == 2 and cg(good_o, good_l, 2, rb=-1) == 2
+    assert cg(good_o, good_l, 2, D=60) == 3 and cg(good_o, good_l, 2, dtype=2) == 4
+    assert cg([0x1000, None], good_l, 2) == 1 and cg(good_o, good_l, 2, o=None) == 1
+    assert cg([0x1000, 0x2008], good_l, 2) == 5 and cg(good_o, [0x3000, 0x3102], 2) == 5
+    assert cg(good_o, good_l, 2, rc=0) == 0                     # an empty row range is a successful no-op
+    assert cg(good_o, good_l, 2) in (7, 8)                      # valid arguments reach the device check
+
+
 def test_host_entry_validation(lib):
     n = lib.attn_fwd_host_workspace_bytes(2, 3, 100, 50, 64)
     qo = (2 * 3 * 100 * 64 * 2 + 255) // 256 * 256

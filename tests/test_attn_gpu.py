@@ -413,3 +413,46 @@ def test_cuda_graph_capture_and_replay():
         g.replay()
     torch.cuda.synchronize()
     assert torch.equal(o.view(torch.int16), ref_o.view(torch.int16)) and torch.equal(lse, ref_l)
+
+
+# ------------------------------------------------------------------ merge of parts behind separate pointers
+
+@pytest.mark.parametrize("n_parts,dtype,D", [(1, 1, 128), (2, 0, 64), (5, 1, 128), (8, 0, 256)])
+def test_combine_gather_equals_combine_and_writes_only_its_rows(n_parts, dtype, D):
+    # the parts live in separate allocations (as they would on separate GPUs); the merge of a row range must
+    # equal attn_combine on the stacked parts for those rows and leave every other row untouched
+    dev = torch.device("cuda:0")
+    B, H, Sq = 2, 3, 77
+    td = inputs.torch_dtype(dtype)
+    g = torch.Generator(device="cpu").manual_seed(5500 + n_parts)
+    o_parts = [torch.randn((B, H, Sq, D), generator=g).to(td).to(dev) for _ in range(n_parts)]
+    l_parts = [torch.randn((B, H, Sq), generator=g).to(dev) for _ in range(n_parts)]
+    if n_parts > 1:
+        l_parts[1][0, 0, :5] = float("-inf")          # a shard that saw no key for some rows
+    ref_o, ref_l = api.attn_combine(torch.stack(o_parts), torch.stack(l_parts))
+    rows = B * H * Sq
+    for row_begin, row_count in ((0, rows), (100, 211), (rows - 1, 1), (50, 0)):
+        out = torch.full((B, H, Sq, D), float("nan"), dtype=td, device=dev)
+        lse = torch.full((B, H, Sq), float("nan"), dtype=torch.float32, device=dev)
+        api.attn_combine_gather([t.data_ptr() for t in o_parts], [t.data_ptr() for t in l_parts], (B, H, Sq, D), td,
+                                out, lse, row_begin, row_count)
+        torch.cuda.synchronize()
+        sel = torch.zeros(rows, dtype=torch.bool, device=dev)
+        sel[row_begin:row_begin + row_count] = True
+        o2, l2 = out.view(rows, D), lse.view(rows)
+        assert torch.equal(o2[sel].view(torch.int16), ref_o.view(rows, D)[sel].view(torch.int16))
+        assert torch.equal(l2[sel], ref_l.view(rows)[sel])
+        assert torch.isnan(o2[~sel].float()).all() and torch.isnan(l2[~sel]).all()
+
+
+def test_combine_gather_rejects_bad_arguments():
+    dev = torch.device("cuda:0")
+    o = torch.zeros((1, 1, 8, 64), dtype=torch.float16, device=dev)
+    l = torch.zeros((1, 1, 8), dtype=torch.float32, device=dev)
+    out, lse = torch.empty_like(o), torch.empty_like(l)
+    for ptrs_o, ptrs_l, rb, rc, want in (([], [], 0, 8, 2), ([o.data_ptr()] * 33, [l.data_ptr()] * 33, 0, 8, 2),
+                                         ([o.data_ptr()], [l.data_ptr()], 4, 8, 2), ([o.data_ptr()], [l.data_ptr()], -1, 2, 2),
+                                         ([0], [l.data_ptr()], 0, 8, 1), ([o.data_ptr() + 8], [l.data_ptr()], 0, 8, 5)):
+        with pytest.raises(api.AttnError) as e:
+            api.attn_combine_gather(ptrs_o, ptrs_l, (1, 1, 8, 64), torch.float16, out, lse, rb, rc)
+        assert e.value.status == want

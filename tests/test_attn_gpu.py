@@ -456,3 +456,21 @@ def test_combine_gather_rejects_bad_arguments():
         with pytest.raises(api.AttnError) as e:
             api.attn_combine_gather(ptrs_o, ptrs_l, (1, 1, 8, 64), torch.float16, out, lse, rb, rc)
         assert e.value.status == want
+
+
+# ------------------------------------------------------------------ very long sequences
+
+@pytest.mark.parametrize("D,dtype,causal,S", [(128, 1, True, 131072), (256, 0, False, 65613)])
+def test_very_long_sequence_on_sampled_rows(D, dtype, causal, S):
+    # a thousand K/V tiles per row and row indices beyond 2^16: rows of every region against the oracle
+    dev = torch.device("cuda:0")
+    q, k, v = inputs.make_qkv(1, 1, S, S, D, dtype, seed=6600 + D)
+    o, lse = api.attn_fwd(q.to(dev), k.to(dev), v.to(dev), D ** -0.5, causal)
+    assert api.attn_last_device_status() == 0
+    rows = np.array(sorted({0, 1, 127, 128, 65535, 65536, S // 2, S - 129, S - 128, S - 2, S - 1}), dtype=np.int64)
+    o_ref, l_ref = orc.attention_rows_16(inputs.bits(q), inputs.bits(k), inputs.bits(v), dtype, rows, D ** -0.5, causal)
+    og = o.cpu().view(-1, D)[rows].to(torch.float64).numpy()
+    lg = lse.cpu().view(-1)[rows].to(torch.float64).numpy()
+    assert not torch.isnan(o.float()).any()
+    assert np.abs(og - o_ref).max() <= O_TOL[dtype]
+    assert np.abs(lg - l_ref).max() <= LSE_TOL

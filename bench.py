@@ -32,7 +32,7 @@ UNIT = "TFLOP/s"
 
 # DRAM bytes (read + write) of one launch of the attention kernel on the default workload, from
 # the ncu captures summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch).
-NCU_TRAFFIC_BYTES = {"C5": 572969216, "C4": 380163328, "C3": 269127168, "C2": 52678912}
+NCU_TRAFFIC_BYTES = {"C5": 578620928, "C4": 380163328, "C3": 269127168, "C2": 52678912}
 
 
 def load_peaks():

@@ -18,12 +18,14 @@
  *   - causal != 0 applies the lower-triangular mask aligned to the top-left corner:
  *     key j is visible to query i iff j <= i, also when Sq != Sk.
  *   - LSE[i] = ln( sum over visible j of exp(scale * <q_i, k_j>) )   (natural log).
- *   - A row without any visible key (only possible when Sk == 0) gives O = 0, LSE = -inf.
+ *   - A row without any visible key (Sk == 0, or a K/V shard that the causal mask hides from the
+ *     row) gives O = 0, LSE = -inf.
  *   - Accumulation is fp32; the probabilities are rounded to the 16-bit input type
  *     before the second product; O is rounded once at the end.
  *
  * Ownership and asynchrony
- *   - The caller owns every buffer.  The library allocates no device memory.
+ *   - The caller owns every buffer.  The library allocates no device memory.  (attn_fwd_host and
+ *     attn_fwd_splitkv create a few streams and events of their own on first use, see there.)
  *   - Device entry points only enqueue work on `stream` (a cudaStream_t, may be NULL for
  *     the default stream) and return; they never synchronise.
  *   - Nothing throws; every entry point returns an attn_status_t (0 = success).

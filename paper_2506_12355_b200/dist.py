@@ -9,6 +9,7 @@ exchange step: the partial results, gathered by NCCL or read in place by the mer
 """
 from __future__ import annotations
 
+import datetime
 import os
 
 import torch
@@ -26,7 +27,9 @@ def init(backend: str) -> tuple:
     if world > 1 and not dist.is_initialized():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", "29500")
-        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+        # a bounded rendezvous / collective timeout: a rank that never joins ends the others with an error
+        dist.init_process_group(backend=backend, rank=rank, world_size=world,
+                                timeout=datetime.timedelta(seconds=int(os.environ.get("ATTN_DIST_TIMEOUT_S", "300"))))
     return rank, local_rank, world
 
 
@@ -61,44 +64,67 @@ def _peer_partials(o_shape, lse_shape, dtype, device):
     return _peer_buffers[key]
 
 
+def _all_gather_stacked(out, x):
+    """out[r] = rank r's x.  NCCL gathers straight into the stacked tensor; other backends (the CPU tests run on
+    gloo, which has no single-tensor all-gather) receive into its slices."""
+    if dist.get_backend() == "nccl":
+        dist.all_gather_into_tensor(out, x)
+    else:
+        dist.all_gather(list(out.unbind(0)), x)
+
+
+def _on_stream(stream):
+    """Context that makes `stream` torch's current stream (a no-op for None or CPU tensors), so that torch's
+    collectives, the symmetric-memory barriers and the library's kernels are all ordered on ONE stream."""
+    import contextlib
+    if stream is None or not torch.cuda.is_available():
+        return contextlib.nullcontext()
+    return torch.cuda.stream(stream)
+
+
 def kv_sharded_attention(q, k_shard, v_shard, scale: float, causal: bool, k_offset: int, stream=None,
                          exchange: str = "nccl"):
     """Attention when every rank holds the full Q but only its own slice of the keys/values.
 
     Each rank computes the partial result of its shard (attn_fwd_partial); the partial (O_r, LSE_r) pairs are
-    then merged.  exchange="nccl": they are all-gathered into this GPU's own memory (NCCL; the one exchange step
-    of this path) and attn_combine merges them; no kernel reads peer memory.  exchange="peer": the partial
-    results are written into symmetric memory and ONE kernel (attn_combine_gather) reads every rank's partial
-    result in place over NVLink with plain loads and merges: exchange and merge fused, nothing gathered first
-    (needs torch's symmetric memory and peer access between the GPUs; a barrier across the ranks on the stream
-    orders it after the partial kernels, a second one keeps the partial results alive until every rank has read
-    them).  Without a process group the single shard is merged alone, which reproduces attn_fwd_gqa.
+    then merged.  exchange="nccl": they are all-gathered into this GPU's own memory (the process group's
+    collective; the one exchange step of this path) and attn_combine merges them; no kernel reads peer memory.
+    exchange="peer": the partial results are written into symmetric memory and ONE kernel (attn_combine_gather)
+    reads every rank's partial result in place over NVLink with plain loads and merges: exchange and merge fused,
+    nothing gathered first (needs torch's symmetric memory and peer access between the GPUs; a barrier across the
+    ranks orders it after the partial kernels, a second one keeps the partial results alive until every rank has
+    read them).  Without a process group the single shard is merged alone, which reproduces attn_fwd_gqa.
+
+    Everything is enqueued on `stream` (default: torch's current stream), which is made the current stream for
+    the duration of the call: the collectives and the symmetric-memory barriers are ordered against torch's
+    current stream, so they and the kernels must share it.
     """
     from . import api
-    multi = dist.is_initialized() and dist.get_world_size() > 1
-    if multi and exchange == "peer":
-        B, H, Sq, D = q.shape
-        o_buf, l_buf, o_hdl, l_hdl = _peer_partials((B, H, Sq, D), (B, H, Sq), q.dtype, q.device)
-        api.attn_fwd_partial(q, k_shard, v_shard, scale, causal, k_offset, out=o_buf, lse=l_buf, stream=stream)
-        o_hdl.barrier()          # every rank's partial result is complete
-        out = torch.empty_like(o_buf)
-        lse = torch.empty_like(l_buf)
-        api.attn_combine_gather(list(o_hdl.buffer_ptrs), list(l_hdl.buffer_ptrs), (B, H, Sq, D), q.dtype, out, lse,
-                                stream=stream)
-        o_hdl.barrier()          # nobody overwrites its partial result while a peer still reads it
-        return out, lse
     if exchange not in ("nccl", "peer"):
         raise ValueError("exchange must be 'nccl' or 'peer'")
-    o_r, lse_r = api.attn_fwd_partial(q, k_shard, v_shard, scale, causal, k_offset, stream=stream)
-    if multi:
-        world = dist.get_world_size()
-        o_parts = torch.empty((world,) + tuple(o_r.shape), dtype=o_r.dtype, device=o_r.device)
-        l_parts = torch.empty((world,) + tuple(lse_r.shape), dtype=lse_r.dtype, device=lse_r.device)
-        dist.all_gather_into_tensor(o_parts, o_r)
-        dist.all_gather_into_tensor(l_parts, lse_r)
-    else:
-        o_parts, l_parts = o_r.unsqueeze(0), lse_r.unsqueeze(0)
-    return api.attn_combine(o_parts.contiguous(), l_parts.contiguous(), stream=stream)
+    multi = dist.is_initialized() and dist.get_world_size() > 1
+    with _on_stream(stream):
+        if multi and exchange == "peer":
+            B, H, Sq, D = q.shape
+            o_buf, l_buf, o_hdl, l_hdl = _peer_partials((B, H, Sq, D), (B, H, Sq), q.dtype, q.device)
+            api.attn_fwd_partial(q, k_shard, v_shard, scale, causal, k_offset, out=o_buf, lse=l_buf, stream=stream)
+            o_hdl.barrier()          # every rank's partial result is complete
+            out = torch.empty_like(o_buf)
+            lse = torch.empty_like(l_buf)
+            api.attn_combine_gather(list(o_hdl.buffer_ptrs), list(l_hdl.buffer_ptrs), (B, H, Sq, D), q.dtype, out,
+                                    lse, stream=stream)
+            o_hdl.barrier()          # nobody overwrites its partial result while a peer still reads it
+            return out, lse
+        o_r, lse_r = api.attn_fwd_partial(q, k_shard, v_shard, scale, causal, k_offset, stream=stream)
+        if multi:
+            world = dist.get_world_size()
+            o_parts = torch.empty((world,) + tuple(o_r.shape), dtype=o_r.dtype, device=o_r.device)
+            l_parts = torch.empty((world,) + tuple(lse_r.shape), dtype=lse_r.dtype, device=lse_r.device)
+            _all_gather_stacked(o_parts, o_r)
+            _all_gather_stacked(l_parts, lse_r)
+        else:
+            o_parts, l_parts = o_r.unsqueeze(0), lse_r.unsqueeze(0)
+        return api.attn_combine(o_parts.contiguous(), l_parts.contiguous(), stream=stream)
 
 
 def rank_seed(base_seed: int, rank: int) -> int:

@@ -12,6 +12,13 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 HEADER = os.path.join(ROOT, "include", "attn_fwd.h")
 
 
+def no_device():
+    """True on a box without a CUDA device.  Calls whose arguments pass validation carry FAKE pointers here, so
+    they may only be made where the library stops at its device check; with a GPU present they would launch."""
+    import torch
+    return not torch.cuda.is_available()
+
+
 @pytest.fixture(scope="module")
 def lib():
     build.build()
@@ -75,7 +82,8 @@ def test_argument_validation_happens_before_any_launch(lib, fn):
     assert call(lib, fn, Sq=0) == 0
     assert call(lib, fn, Sq=0, q=None, o=None, lse=None) == 0
     # k, v may be NULL only when there are no keys (that case reaches the device check)
-    assert call(lib, fn, Sk=0, k=None, v=None) != 1
+    if no_device():
+        assert call(lib, fn, Sk=0, k=None, v=None) in (7, 8)
 
 
 def test_fp8_entry_validation(lib):
@@ -95,7 +103,8 @@ def test_fp8_entry_validation(lib):
     assert f8(scale=3e38, fq=10.0) == 6         # the effective scale must stay finite
     assert f8(impl=2) == 4
     assert f8(Sq=0) == 0
-    assert f8() in (7, 8) or True               # valid arguments reach the device check (no device here: 7 or 8)
+    if no_device():
+        assert f8() in (7, 8)                   # valid arguments reach the device check
 
 
 def test_splitkv_entry_validation(lib):
@@ -128,7 +137,8 @@ def test_combine_gather_validation(lib):
     assert cg([0x1000, None], good_l, 2) == 1 and cg(good_o, good_l, 2, o=None) == 1
     assert cg([0x1000, 0x2008], good_l, 2) == 5 and cg(good_o, [0x3000, 0x3102], 2) == 5
     assert cg(good_o, good_l, 2, rc=0) == 0                     # an empty row range is a successful no-op
-    assert cg(good_o, good_l, 2) in (7, 8)                      # valid arguments reach the device check
+    if no_device():
+        assert cg(good_o, good_l, 2) in (7, 8)                  # valid arguments reach the device check
 
 
 def test_host_entry_validation(lib):
@@ -148,8 +158,7 @@ def test_host_entry_validation(lib):
 
 
 def test_no_fallback_without_a_device(lib):
-    import torch
-    if torch.cuda.is_available():
+    if not no_device():
         pytest.skip("a device is present")
     # valid arguments but no B200: the library must report an error, not compute on the CPU
     assert call(lib) in (7, 8)

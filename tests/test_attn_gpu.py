@@ -28,6 +28,12 @@ def guards_intact(buf):
     return bool(torch.isnan(buf[:GUARD]).all()) and bool(torch.isnan(buf[-GUARD:]).all())
 
 
+def f32_scale(D):
+    """1/sqrt(D) as the fp32 value that crosses the C ABI, widened to a Python float: the oracle
+    is given exactly the number the kernels see."""
+    return float(np.float32(1.0) / np.sqrt(np.float32(D)))
+
+
 def run_gpu(fn, q, k, v, scale, causal):
     dev = torch.device("cuda:0")
     qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
@@ -86,7 +92,7 @@ def test_small_shapes(shape, D, dtype, causal, impl):
     if impl == "simt" and (D == 256 or Sq * Sk > 70000) and dtype == inputs.DTYPE_BF16:
         pytest.skip("cross-check kernel: subset only")
     q, k, v = inputs.make_qkv(B, H, Sq, Sk, D, dtype, seed=1000 + Sq * 7 + Sk + D)
-    check_against_oracle(IMPLS[impl], q, k, v, dtype, 1.0 / math.sqrt(D), causal)
+    check_against_oracle(IMPLS[impl], q, k, v, dtype, f32_scale(D), causal)
 
 
 def test_config_c1_full():
@@ -100,7 +106,7 @@ def test_config_c1_full():
 def test_several_tiles_and_ragged_tail(D, dtype, causal):
     # several 128-row Q tiles and K/V tiles plus a ragged tail, several heads
     q, k, v = inputs.make_qkv(2, 3, 128 * 3 + 37, 128 * 4 + 91, D, dtype, seed=4242 + D)
-    check_against_oracle(api.attn_fwd, q, k, v, dtype, 1.0 / math.sqrt(D), causal)
+    check_against_oracle(api.attn_fwd, q, k, v, dtype, f32_scale(D), causal)
 
 
 # ------------------------------------------------------------------ hand-derived cases on the GPU
@@ -220,22 +226,35 @@ def test_host_entry_pipelined_over_groups_of_heads(D, dtype, causal, B, H, S):
         assert torch.equal(o.view(torch.int16), o_dev.view(torch.int16)) and torch.equal(lse, lse_dev)
 
 
-# ------------------------------------------------------------------ full-size configurations, sampled rows
+# ------------------------------------------------------------------ full-size configurations, every row
 
 @pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5"])
-def test_full_size_configs_on_sampled_rows(name):
+def test_full_size_configs_against_oracle_on_every_row(name):
+    # the whole output tensor of each benchmark configuration against the fp64 oracle, one (batch, head)
+    # at a time so that the fp64 reference of a head (at most 16 MiB) is all that is held at once
     cfg = inputs.CONFIGS[name]
     q, k, v = inputs.make_config_inputs(cfg)
     o, lse = run_gpu(api.attn_fwd, q, k, v, cfg.scale, cfg.causal)
-    rows = inputs.sample_rows(cfg.B * cfg.H * cfg.Sq, cfg.Sq, 192, seed=cfg.index)
-    o_ref, lse_ref = orc.attention_rows_16(inputs.bits(q), inputs.bits(k), inputs.bits(v), cfg.dtype, rows,
-                                           cfg.scale, cfg.causal)
-    got_o = o.view(-1, cfg.D)[torch.from_numpy(rows)].double().numpy()
-    got_l = lse.view(-1)[torch.from_numpy(rows)].double().numpy()
-    err = np.abs(got_o - o_ref)
-    assert err.max() <= O_TOL[cfg.dtype], "max |dO| = %g at sampled row %d" % (err.max(), rows[err.max(axis=1).argmax()])
-    assert np.abs(got_l - lse_ref).max() <= LSE_TOL
-    # properties that hold at any size, over ALL rows: finite outputs, |O| bounded by max |V| per head
+    qb, kb, vb = inputs.bits(q), inputs.bits(k), inputs.bits(v)
+    o2, l2 = o.view(-1, cfg.D), lse.view(-1)
+    worst_o, worst_l, where, sq_err, sq_ref = 0.0, 0.0, None, 0.0, 0.0
+    for bh in range(cfg.B * cfg.H):
+        rows = np.arange(bh * cfg.Sq, (bh + 1) * cfg.Sq, dtype=np.int64)
+        o_ref, lse_ref = orc.attention_rows_16(qb, kb, vb, cfg.dtype, rows, cfg.scale, cfg.causal)
+        err = np.abs(o2[rows[0]:rows[-1] + 1].double().numpy() - o_ref)
+        if err.max() > worst_o:
+            worst_o = float(err.max())
+            where = (bh, int(err.max(axis=1).argmax()))
+        worst_l = max(worst_l, float(np.abs(l2[rows[0]:rows[-1] + 1].double().numpy() - lse_ref).max()))
+        sq_err += float((err ** 2).sum())
+        sq_ref += float((o_ref ** 2).sum())
+    print("%s: all %d rows  max|dO| = %.3g at (head, row) %s  max|dLSE| = %.3g  rms dO / rms O = %.3g" % (
+        name, cfg.B * cfg.H * cfg.Sq, worst_o, where, worst_l, math.sqrt(sq_err / sq_ref)))
+    assert worst_o <= O_TOL[cfg.dtype], "max |dO| = %g at (head, row) %s" % (worst_o, where)
+    assert worst_l <= LSE_TOL, "max |dLSE| = %g" % worst_l
+    # the absolute bar is loose for long diffuse rows (|O| ~ 0.03): the error must also be small against O itself
+    assert math.sqrt(sq_err / sq_ref) <= (2.0 ** -9 if cfg.dtype == inputs.DTYPE_FP16 else 2.0 ** -6)
+    # properties that hold at any size: finite outputs, |O| bounded by max |V| per head
     assert bool(torch.isfinite(o.float()).all()) and bool(torch.isfinite(lse).all())
     vmax = v.float().abs().amax(dim=(2, 3), keepdim=True)
     assert bool((o.float().abs() <= vmax * (1 + 1e-2)).all())
@@ -267,7 +286,7 @@ def test_gqa_against_oracle(D, dtype, causal, H, Hkv):
     dev = torch.device("cuda:0")
     obuf, o = guarded((B, H, Sq, D), q.dtype, dev)
     lbuf, lse = guarded((B, H, Sq), torch.float32, dev)
-    scale = 1.0 / math.sqrt(D)
+    scale = f32_scale(D)
     api.attn_fwd_gqa(q.to(dev), k.to(dev), v.to(dev), scale, causal, out=o, lse=lse)
     assert api.attn_last_device_status() == 0 and guards_intact(obuf) and guards_intact(lbuf)
     o_ref, lse_ref = orc.attention_gqa(*(orc.widen(inputs.bits(t), dtype) for t in (q, k, v)), scale, causal)
@@ -295,7 +314,7 @@ def test_qk192_v128_against_oracle(dtype, causal, H, Hkv, Sq, Sk):
     dev = torch.device("cuda:0")
     obuf, o = guarded((B, H, Sq, 128), q.dtype, dev)
     lbuf, lse = guarded((B, H, Sq), torch.float32, dev)
-    scale = 1.0 / math.sqrt(192)
+    scale = f32_scale(192)
     api.attn_fwd_qkv_dims(q.to(dev), k.to(dev), v.to(dev), scale, causal, out=o, lse=lse)
     assert api.attn_last_device_status() == 0 and guards_intact(obuf) and guards_intact(lbuf)
     o_ref, lse_ref = orc.attention_gqa_dv(*(orc.widen(inputs.bits(t), dtype) for t in (q, k, v)), scale, causal)
@@ -321,7 +340,7 @@ def test_kv_shards_and_combine_against_oracle(D, dtype, causal, Hkv):
     v = inputs.randn16((B, Hkv, Sk, D), 702, dtype)
     dev = torch.device("cuda:0")
     qd = q.to(dev)
-    scale = 1.0 / math.sqrt(D)
+    scale = f32_scale(D)
     cuts = [0, 130, 384, Sk]        # uneven shards, one boundary off the tile grid
     n = len(cuts) - 1
     o_parts = torch.full((n, B, H, Sq, D), float("nan"), dtype=q.dtype, device=dev)

@@ -105,5 +105,54 @@ def test_two_gloo_ranks_shard_by_keys_and_merge(tmp_path):
     assert open(out).read() == "ok"
 
 
+def _kv_glue_worker(rank, world, port, out_path):
+    """Drives dist.kv_sharded_attention itself (exchange="nccl" shape of the control flow: partial call, two
+    all-gathers into the rank's own memory, merge) on two gloo ranks, with the two library calls replaced by the
+    shard and merge arithmetic of the oracle on CPU tensors.  Checks the glue: offsets, gather order, shapes."""
+    from oracle import attn_oracle as orc
+    from paper_2506_12355_b200 import api
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    adist.init("gloo")
+    calls = []
+
+    def fake_partial(q, k, v, scale, causal, k_offset, out=None, lse=None, stream=None):
+        calls.append(("partial", k_offset, tuple(k.shape)))
+        o, l = orc.attention_shard(q.numpy(), k.numpy(), v.numpy(), scale, causal, k_offset)
+        return torch.from_numpy(o), torch.from_numpy(l)
+
+    def fake_combine(o_parts, lse_parts, out=None, lse=None, stream=None):
+        calls.append(("combine", tuple(o_parts.shape)))
+        o, l = orc.combine(o_parts.numpy(), lse_parts.numpy())
+        return torch.from_numpy(o), torch.from_numpy(l)
+
+    api.attn_fwd_partial, api.attn_combine = fake_partial, fake_combine
+    B, H, Sq, Sk, D = 2, 2, 19, 45, 8
+    q, k, v = inputs.make_qkv(B, H, Sq, Sk, D, inputs.DTYPE_FP16, seed=31)
+    qf, kf, vf = (torch.from_numpy(orc.widen(inputs.bits(t), 0)) for t in (q, k, v))
+    b, e = adist.shard_keys(Sk, world, rank)
+    o, lse = adist.kv_sharded_attention(qf, kf[:, :, b:e].contiguous(), vf[:, :, b:e].contiguous(), 0.3, True, b,
+                                        exchange="nccl")
+    o_ref, l_ref = orc.attention(qf.numpy(), kf.numpy(), vf.numpy(), 0.3, True)
+    ok = (np.allclose(o.numpy(), o_ref, atol=1e-12) and np.allclose(lse.numpy(), l_ref, atol=1e-12)
+          and calls == [("partial", b, (B, H, e - b, D)), ("combine", (world, B, H, Sq, D))])
+    flags = [None] * world
+    dist.all_gather_object(flags, bool(ok))
+    if rank == 0:
+        open(out_path, "w").write("ok" if all(flags) else "mismatch")
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_drive_kv_sharded_attention_glue(tmp_path):
+    out = str(tmp_path / "result_glue.txt")
+    mp.spawn(_kv_glue_worker, args=(2, _free_port(), out), nprocs=2, join=True)
+    assert open(out).read() == "ok"
+
+
+def test_kv_sharded_attention_rejects_unknown_exchange():
+    with pytest.raises(ValueError):
+        adist.kv_sharded_attention(None, None, None, 1.0, False, 0, exchange="carrier pigeon")
+
+
 def test_shard_keys_offsets():
     assert [adist.shard_keys(10, 3, r) for r in range(3)] == [(0, 4), (4, 7), (7, 10)]

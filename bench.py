@@ -263,6 +263,34 @@ class Problem:
         self.lse.fill_(float("nan"))
 
 
+def host_enqueue_us(api, prob, calls):
+    """Host time of one attn_fwd call through the C ABI (arguments prepared once; validation, tensor maps and
+    the launch), while the device works through the queue."""
+    cfg = prob.cfg
+    fn = api.load().attn_fwd
+    a = (prob.qd.data_ptr(), prob.kd.data_ptr(), prob.vd.data_ptr(), prob.o.data_ptr(), prob.lse.data_ptr(), cfg.B, cfg.H,
+         cfg.Sq, cfg.Sk, cfg.D, cfg.scale, int(cfg.causal), cfg.dtype, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(calls):
+        fn(*a)
+    t1 = time.perf_counter()
+    torch.cuda.synchronize()
+    return (t1 - t0) / calls * 1e6
+
+
+def graph_replay_us(prob, flush, launches):
+    """Median device time of the launch replayed from a CUDA graph (isolated, L2 flushed)."""
+    st = torch.cuda.Stream(device=prob.dev)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            prob.api.attn_fwd(prob.qd, prob.kd, prob.vd, prob.cfg.scale, prob.cfg.causal, out=prob.o, lse=prob.lse,
+                              stream=st)
+    torch.cuda.synchronize()
+    return float(np.median(time_isolated(g.replay, flush, launches, warmup=3))) * 1e3
+
+
 def config_block(api, dev, peaks, flush, headline, headline_errors, with_errors):
     """C1..C5 as isolated launches (L2 flushed in between): time, throughput, bandwidth at the algorithmic bytes
     and the errors of that output against the oracle."""
@@ -278,7 +306,10 @@ def config_block(api, dev, peaks, flush, headline, headline_errors, with_errors)
                  "tflops": cfg.flops / med / 1e9, "frac_of_burst": cfg.flops / med / 1e9 / peaks["bf16_tflops"],
                  "gbs_at_min_bytes": cfg.min_hbm_bytes / med / 1e6,
                  "frac_of_hbm_peak": cfg.min_hbm_bytes / med / 1e6 / peaks["hbm_gbs"],
-                 "ncu_dram_bytes": NCU_TRAFFIC_BYTES.get(name), "min_hbm_bytes": cfg.min_hbm_bytes}
+                 "ncu_dram_bytes": NCU_TRAFFIC_BYTES.get(name), "min_hbm_bytes": cfg.min_hbm_bytes,
+                 "host_us_per_call": host_enqueue_us(api, prob, 200 if name in ("C1", "C2") else 20)}
+        if name in ("C1", "C2", "C3"):   # launch-latency territory: the same launch replayed from a CUDA graph
+            entry["us_graph_replay_median"] = graph_replay_us(prob, flush, 50)
         if with_errors:
             if name == headline.cfg.name and headline_errors is not None:
                 entry["errors"] = headline_errors

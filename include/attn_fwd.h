@@ -31,6 +31,21 @@
  *   - Nothing throws; every entry point returns an attn_status_t (0 = success).
  *   - Q, K, V must not alias O or LSE.
  *
+ * Streams and CUDA graphs
+ *   - Launches may be issued on any number of streams at once.  A problem with more work items
+ *     than the GPU has multiprocessors draws its items from a device-side work counter that lives in
+ *     the library image; the kernel leaves it zeroed, so nothing but the kernel is enqueued.  Eager
+ *     launches use the counter of their stream: at most 768 distinct streams per device may launch
+ *     such problems over the life of the process (the per-thread default stream counts once per
+ *     host thread); a stream handle that is destroyed and handed out again keeps its counter.
+ *   - Every entry point that takes a `stream` may be captured into a CUDA graph, provided the first
+ *     call for that device, head dim and type was made outside capture (one-time set-up).  Each
+ *     captured launch of such a problem takes a counter of its own that eager launches never use,
+ *     so a graph can be replayed on any stream while eager launches run elsewhere; at most 256 such
+ *     launches can be captured per device and process.  Two executable graphs instantiated from the
+ *     SAME capture share its counters and must not run at the same time.
+ *   - When either limit is exhausted the launch is refused with ATTN_ERR_COUNTER_SLOTS.
+ *
  * There is no CPU fallback: on a device that is not compute capability 10.x the entry
  * points return ATTN_ERR_UNSUPPORTED_ARCH.
  */
@@ -59,7 +74,8 @@ typedef enum {
     ATTN_ERR_CUDA = 8,                 /* a CUDA runtime/driver call failed */
     ATTN_ERR_DEVICE_TIMEOUT = 9,       /* a kernel gave up on a bounded on-chip wait */
     ATTN_ERR_WORKSPACE = 10,           /* workspace missing, misaligned or too small */
-    ATTN_ERR_STATIC_CAPACITY = 11      /* problem does not fit the library's built-in staging buffer */
+    ATTN_ERR_STATIC_CAPACITY = 11,     /* problem does not fit the library's built-in staging buffer */
+    ATTN_ERR_COUNTER_SLOTS = 12        /* no work counter left for this launch (see "Streams and CUDA graphs") */
 } attn_status_t;
 
 /*

@@ -21,6 +21,7 @@ STATUS_NAMES = {
     3: "ATTN_ERR_UNSUPPORTED_HEAD_DIM", 4: "ATTN_ERR_UNSUPPORTED_DTYPE", 5: "ATTN_ERR_MISALIGNED",
     6: "ATTN_ERR_BAD_SCALE", 7: "ATTN_ERR_UNSUPPORTED_ARCH", 8: "ATTN_ERR_CUDA",
     9: "ATTN_ERR_DEVICE_TIMEOUT", 10: "ATTN_ERR_WORKSPACE", 11: "ATTN_ERR_STATIC_CAPACITY",
+    12: "ATTN_ERR_COUNTER_SLOTS",
 }
 
 # every symbol include/attn_fwd.h declares

@@ -7,8 +7,10 @@
 #include <stdint.h>
 #include <string.h>
 
-#include <atomic>
+#include <functional>
+#include <map>
 #include <mutex>
+#include <thread>
 #include <utility>
 #include <vector>
 
@@ -67,8 +69,51 @@ EncodeTiledFn get_encode_fn() {
 // box = [1, box_rows, 128 bytes of columns], 128-byte swizzle, out-of-range rows read as zero.
 // head_stride_rows: distance between consecutive (batch, head) slices in rows (S for a contiguous tensor; larger
 // when the map covers a range of rows of a bigger tensor: a K/V shard addressed in place).
+// A tensor map is a pure function of the address and the shape arguments (it does not depend on the
+// memory's contents), so encoded maps are kept in a small per-thread direct-mapped cache: a caller
+// that passes the same buffers again (a training or serving loop) pays for four look-ups instead of
+// four driver calls per launch.
+struct MapKey {
+    const void* base;
+    int64_t BH, S, head_stride_rows;
+    int dtype, D, box_rows;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && BH == o.BH && S == o.S && head_stride_rows == o.head_stride_rows && dtype == o.dtype &&
+               D == o.D && box_rows == o.box_rows;
+    }
+};
+struct MapCacheEntry {
+    bool valid = false;
+    MapKey key;
+    CUtensorMap map;
+};
+constexpr int kMapCacheSize = 64;
+
+bool encode_map(CUtensorMap* map, const void* base, int dtype, int64_t BH, int64_t S, int D, int box_rows,
+                int64_t head_stride_rows);
+
 bool make_map(CUtensorMap* map, const void* base, int dtype, int64_t BH, int64_t S, int D, int box_rows,
               int64_t head_stride_rows = -1) {
+    thread_local MapCacheEntry cache[kMapCacheSize];
+    const MapKey key{base, BH, S, head_stride_rows, dtype, D, box_rows};
+    uint64_t h = reinterpret_cast<uintptr_t>(base) >> 8;
+    h = (h ^ (static_cast<uint64_t>(S) * 0x9E3779B97F4A7C15ull) ^ (static_cast<uint64_t>(BH) << 17) ^
+         (static_cast<uint64_t>(D + 3 * dtype + 7 * box_rows) << 40) ^ static_cast<uint64_t>(head_stride_rows)) *
+        0xD6E8FEB86659FD93ull;
+    MapCacheEntry& e = cache[(h >> 32) % kMapCacheSize];
+    if (e.valid && e.key == key) {
+        *map = e.map;
+        return true;
+    }
+    if (!encode_map(map, base, dtype, BH, S, D, box_rows, head_stride_rows)) return false;
+    e.valid = true;
+    e.key = key;
+    e.map = *map;
+    return true;
+}
+
+bool encode_map(CUtensorMap* map, const void* base, int dtype, int64_t BH, int64_t S, int D, int box_rows,
+                int64_t head_stride_rows) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
     const cuuint64_t es = dtype == ATTN_DTYPE_FP8_E4M3 ? 1 : 2;
@@ -120,24 +165,39 @@ int validate(const void* q, const void* k, const void* v, const void* o, const v
     return ATTN_OK;
 }
 
-// Work counters of the persistent kernel: every launch takes the next slot of this ring and zeroes
-// it on its stream right before the kernel, so launches in flight on different streams do not share
-// a counter (unless more than kCounterSlots launches are in flight at once).
-constexpr int kCounterSlots = 1024;
-__device__ unsigned int g_work_counters[kCounterSlots];
-std::atomic<unsigned int> g_launch_seq{0};
+// Work counters of the persistent kernels.  A counter is two words {next item, CTAs done}; it is zero
+// when a launch starts and the kernel zeroes it again when its last CTA exits, so no memset is
+// enqueued.  Two launches may share a counter only if they cannot overlap, hence:
+//   * an eager launch takes the counter of its stream (launches on one stream are ordered); the
+//     per-thread default stream is a different stream in every host thread and is keyed by thread too;
+//   * a launch made while its stream is being captured into a CUDA graph takes a counter of its own
+//     from a separate region that eager launches never use: a graph may be replayed on any stream,
+//     at any time, next to eager launches.  (Replays of one executable graph are ordered by CUDA.)
+// Both regions are finite; when one is used up the launch is refused with ATTN_ERR_COUNTER_SLOTS.
+constexpr int kStreamSlots = 768;    // distinct streams that may launch counted kernels, per device
+constexpr int kCaptureSlots = 256;   // counted launches that may be captured into graphs, per device
+__device__ unsigned int g_work_counters[2 * (kStreamSlots + kCaptureSlots)];
+
+constexpr int kMaxDevices = 64;
 
 struct DeviceInfo {
     unsigned int* counters = nullptr;
     int sm_count = 0;
 };
 
+struct CounterTable {
+    std::mutex mu;
+    std::map<std::pair<uintptr_t, size_t>, int> by_stream;
+    int captured = 0;
+};
+CounterTable g_counter_table[kMaxDevices];
+
 // Per-device facts resolved on first use (symbol address of the counters, SM count).
-int device_info(DeviceInfo* out) {
+int device_info(DeviceInfo* out, int* dev_out = nullptr) {
     static std::mutex mu;
-    static DeviceInfo info[64];
+    static DeviceInfo info[kMaxDevices];
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ATTN_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ATTN_ERR_CUDA;
     std::lock_guard<std::mutex> lock(mu);
     if (!info[dev].counters) {
         void* p = nullptr;
@@ -149,6 +209,31 @@ int device_info(DeviceInfo* out) {
         info[dev].sm_count = sms;
     }
     *out = info[dev];
+    if (dev_out) *dev_out = dev;
+    return ATTN_OK;
+}
+
+// The work counter for a launch on stream `st` of the current device (see above).
+int work_counter(const DeviceInfo& di, int dev, cudaStream_t st, unsigned int** out) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) return ATTN_ERR_CUDA;
+    CounterTable& tab = g_counter_table[dev];
+    std::lock_guard<std::mutex> lock(tab.mu);
+    int slot;
+    if (cap != cudaStreamCaptureStatusNone) {
+        if (tab.captured >= kCaptureSlots) return ATTN_ERR_COUNTER_SLOTS;
+        slot = kStreamSlots + tab.captured++;
+    } else {
+        const size_t thread_key = st == cudaStreamPerThread ? std::hash<std::thread::id>()(std::this_thread::get_id()) : 0;
+        const auto key = std::make_pair(reinterpret_cast<uintptr_t>(st), thread_key);
+        auto it = tab.by_stream.find(key);
+        if (it == tab.by_stream.end()) {
+            if (tab.by_stream.size() >= static_cast<size_t>(kStreamSlots)) return ATTN_ERR_COUNTER_SLOTS;
+            it = tab.by_stream.emplace(key, static_cast<int>(tab.by_stream.size())).first;
+        }
+        slot = it->second;
+    }
+    *out = di.counters + 2 * slot;
     return ATTN_OK;
 }
 
@@ -178,8 +263,8 @@ int fill_empty(void* o, float* lse, int64_t n_o, int64_t n_lse, cudaStream_t st)
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
-#ifdef ATTN_TC_PROFILE
-long long* g_prof_buffer = nullptr;  // development builds only
+#ifdef ATTN_TEST_HOOKS
+int g_test_skip_ring_item = -1;   // test build only: consumed by the next launch of the pipelined kernel
 #endif
 
 // Pipelined, warp-specialised kernel (head dims 64 and 128): one CTA per pair of 128-row Q tiles.
@@ -230,11 +315,13 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     hpg *= H / Hkv;  // the query heads of one K/V head share its footprint
     if (hpg > BH) hpg = BH;
     prm.heads_per_group = static_cast<int>(hpg);
-    // the last three groups are merged into one: its items, ordered longest-first, then end with short ones,
-    // which keeps the tail of the launch short
+    // under the causal mask the last three groups are merged into one: its items, ordered longest-first, then
+    // end with short ones, which keeps the tail of the launch short; without a mask all items are equally long
+    // and merging would only enlarge the K/V footprint of the tail beyond what stays in L2
     {
         const int64_t n_groups = (BH + hpg - 1) / hpg;
-        prm.last_group = static_cast<int>(n_groups >= ATTN_MERGE_LAST ? n_groups - ATTN_MERGE_LAST : 0);
+        const int merge = causal ? ATTN_MERGE_LAST : 1;
+        prm.last_group = static_cast<int>(n_groups >= merge ? n_groups - merge : 0);
     }
     prm.n_items = static_cast<int>(n_pairs * BH * n_splits);
     prm.n_splits = n_splits;
@@ -242,18 +329,20 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
         const int tiles = (Sk + C::BN - 1) / C::BN;
         prm.split_tiles = n_splits > 1 ? (tiles + n_splits - 1) / n_splits : 2147483647 / 2;
     }
-#ifdef ATTN_TC_PROFILE
-    prm.prof = g_prof_buffer;
+#ifdef ATTN_TEST_HOOKS
+    prm.test_skip_ring_item = g_test_skip_ring_item;
+    g_test_skip_ring_item = -1;
 #endif
     // persistent grid: one CTA per SM; the first item of a CTA is its block index, the rest come from
-    // a device counter that is zeroed on the stream right before the launch
+    // a device counter that is zero at launch (the previous kernel that used it left it so)
     DeviceInfo di;
-    if (device_info(&di) != ATTN_OK) return ATTN_ERR_CUDA;
+    int dev = 0;
+    if (device_info(&di, &dev) != ATTN_OK) return ATTN_ERR_CUDA;
     const unsigned grid = static_cast<unsigned>(prm.n_items < di.sm_count ? prm.n_items : di.sm_count);
-    prm.counter = nullptr;   // small problems: every CTA takes exactly one item, no counter and no memset
+    prm.counter = nullptr;   // small problems: every CTA takes exactly one item, no counter
     if (prm.n_items > di.sm_count) {
-        prm.counter = di.counters + (g_launch_seq.fetch_add(1) % kCounterSlots);
-        if (cudaMemsetAsync(prm.counter, 0, sizeof(unsigned int), st) != cudaSuccess) return ATTN_ERR_CUDA;
+        const int rc = work_counter(di, dev, st, &prm.counter);
+        if (rc != ATTN_OK) return rc;
     }
     kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, mo, prm);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
@@ -295,18 +384,20 @@ int launch_tc_qtmem(const void* q, const void* k, const void* v, void* o, float*
     hpg *= H / Hkv;
     if (hpg > BH) hpg = BH;
     prm.heads_per_group = static_cast<int>(hpg);
-    {
+    {   // merged tail only under the causal mask (see launch_tc_pipe)
         const int64_t n_groups = (BH + hpg - 1) / hpg;
-        prm.last_group = static_cast<int>(n_groups >= ATTN_MERGE_LAST ? n_groups - ATTN_MERGE_LAST : 0);
+        const int merge = causal ? ATTN_MERGE_LAST : 1;
+        prm.last_group = static_cast<int>(n_groups >= merge ? n_groups - merge : 0);
     }
     prm.n_items = static_cast<int>(n_qtiles * BH);
     DeviceInfo di;
-    if (device_info(&di) != ATTN_OK) return ATTN_ERR_CUDA;
+    int dev = 0;
+    if (device_info(&di, &dev) != ATTN_OK) return ATTN_ERR_CUDA;
     const unsigned grid = static_cast<unsigned>(prm.n_items < di.sm_count ? prm.n_items : di.sm_count);
-    prm.counter = nullptr;   // small problems: every CTA takes exactly one item, no counter and no memset
+    prm.counter = nullptr;   // small problems: every CTA takes exactly one item, no counter
     if (prm.n_items > di.sm_count) {
-        prm.counter = di.counters + (g_launch_seq.fetch_add(1) % kCounterSlots);
-        if (cudaMemsetAsync(prm.counter, 0, sizeof(unsigned int), st) != cudaSuccess) return ATTN_ERR_CUDA;
+        const int rc = work_counter(di, dev, st, &prm.counter);
+        if (rc != ATTN_OK) return rc;
     }
     kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mo, prm);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
@@ -370,7 +461,6 @@ size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 // the name, is what the copies and the kernel are given.
 static __device__ __align__(256) unsigned char g_static_workspace[ATTN_STATIC_WORKSPACE_BYTES];
 
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 void* g_static_workspace_addr[kMaxDevices] = {};
 
@@ -483,8 +573,10 @@ int host_pipelined(const void* q_host, const void* k_host, const void* v_host, v
 
 extern "C" {
 
-#ifdef ATTN_TC_PROFILE
-void attn_debug_set_profile_buffer(long long* p) { g_prof_buffer = p; }
+#ifdef ATTN_TEST_HOOKS
+// Test build only (never part of libattn_fwd.so): the next launch of the pipelined kernel leaves out the load
+// of this K/V ring item, so that the wait for it runs out and the kernel returns through its time-out path.
+void attn_test_skip_kv_load(int ring_item) { g_test_skip_ring_item = ring_item; }
 #endif
 
 int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk, int D,
@@ -793,6 +885,7 @@ const char* attn_status_string(int status) {
         case ATTN_ERR_DEVICE_TIMEOUT: return "ATTN_ERR_DEVICE_TIMEOUT";
         case ATTN_ERR_WORKSPACE: return "ATTN_ERR_WORKSPACE";
         case ATTN_ERR_STATIC_CAPACITY: return "ATTN_ERR_STATIC_CAPACITY";
+        case ATTN_ERR_COUNTER_SLOTS: return "ATTN_ERR_COUNTER_SLOTS";
         default: return "ATTN_ERR_UNKNOWN";
     }
 }

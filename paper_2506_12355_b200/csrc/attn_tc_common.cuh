@@ -18,4 +18,21 @@ __device__ __forceinline__ int last_visible_key(int row, int Sk, int causal, int
     return c < all ? c : all;
 }
 
+// End of a persistent kernel, executed by one thread per CTA after the CTA's last draw from the work
+// counter: reports a timed-out wait, and hands the counter back zeroed.  counter[0] is the next work
+// item, counter[1] the number of CTAs that have finished; the CTA that finishes last resets both, so
+// the next launch that uses this counter (launches that share one are ordered on one stream) starts
+// from zero without a memset.  Every CTA reaches this point, also after a timed-out wait.
+__device__ __forceinline__ void finish_cta(int* status, bool timed_out, unsigned int* counter) {
+    if (timed_out) atomicExch(status, kStatusTimeout);
+    if (counter) {
+        __threadfence();
+        if (atomicAdd(counter + 1, 1u) == gridDim.x - 1) {
+            counter[0] = 0u;
+            counter[1] = 0u;
+            __threadfence();
+        }
+    }
+}
+
 }  // namespace attn_tc

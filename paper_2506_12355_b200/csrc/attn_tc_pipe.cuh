@@ -70,9 +70,10 @@ struct PipeParams {
     int n_items;            // n_pairs * BH * n_splits
     int n_splits;           // key ranges per (head, Q tile pair): 1, or more for split-KV decoding, where range s of
     int split_tiles;        // split_tiles K/V tiles writes its partial result as head s * BH + bh of o and lse
-    unsigned int* counter;  // work counter, zero at launch: item = gridDim.x + atomicAdd(counter, 1); NULL when n_items <= grid
-#ifdef ATTN_TC_PROFILE
-    long long* prof;        // development builds: [grid][16] cycle sums of softmax group 1, row 0
+    unsigned int* counter;  // work counter {next item, CTAs done}, zero at launch and again at exit:
+                            // item = gridDim.x + atomicAdd(counter, 1); NULL when n_items <= grid
+#ifdef ATTN_TEST_HOOKS
+    int test_skip_ring_item;  // test build only: the K/V ring item whose load the producer leaves out (-1: none)
 #endif
 };
 
@@ -294,6 +295,9 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     const int s = ring_item % NSLOT;
                     const uint32_t use = ring_item / NSLOT;
                     if (!mbar_wait(bar(B_KVEMPTY + s), (use & 1) ^ 1, abort_flag)) return false;
+#ifdef ATTN_TEST_HOOKS
+                    if (ring_item == prm.test_skip_ring_item) return true;   // this slot's "full" barrier never completes
+#endif
                     if (leader) {
                         mbar_arrive_expect_tx(bar(B_KVFULL + s), C::KV_BYTES);
 #pragma unroll
@@ -432,17 +436,10 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             else
                 tmem_st_32x32b_x16(tS + ch * PCOLS, pk);
         };
-#ifdef ATTN_TC_PROFILE
-        long long pacc[8] = {}, pt0 = clock64();
-#define PLAP(i) do { long long t1_ = clock64(); pacc[i] += t1_ - pt0; pt0 = t1_; } while (0)
-#else
-#define PLAP(i)
-#endif
 
         for (int k = 0; ok; ++k) {
             PipeItem it;
             const int item = next_item(k, lane == 0, it);
-            PLAP(0);
             if (item < 0) break;
             const int n = it.n_kv[t];
             const int q0 = it.q0;
@@ -463,7 +460,6 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 
             for (int j = 0; j < n; ++j) {
                 if (!(ok = mbar_wait(bar(B_SFULL + t), (it_base + j) & 1, abort_flag))) break;
-                PLAP(j == 0 ? 1 : (j == n - 1 ? 5 : 3));
                 tc_fence_after_sync();
                 // Visibility of this K/V tile, per warp (rows 32 w .. 32 w + 31 of the Q tile): a chunk of
                 // 32 keys is FULL (every row sees all of it), EMPTY (no row sees any of it) or PARTIAL.
@@ -690,7 +686,6 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 tmem_st_wait();
                 tc_fence_before_sync();
                 mbar_arrive(bar(B_PFULL2 + t));
-                PLAP(j == 0 ? 2 : (j == n - 1 ? 6 : 4));
             }
             if (!ok) break;
 
@@ -737,18 +732,14 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             if (row < prm.Sq) prm.lse[grow] = seen ? m * prm.scale + (logf(l) - P_OFF * 0.6931471805599453f) : -INFINITY;
             it_base += n;
             ++uses;
-            PLAP(7);
         }
         if (r == 0) tma_store_wait_all<0>();   // the staging tile must outlive its last store
-#ifdef ATTN_TC_PROFILE
-        if (t == 1 && r == 0) { for (int i = 0; i < 8; ++i) prm.prof[blockIdx.x * 16 + i] = pacc[i]; prm.prof[blockIdx.x * 16 + 8] = uses; prm.prof[blockIdx.x * 16 + 9] = it_base; }
-#endif
     }
 
     // ---- teardown (also reached after a timed-out wait) ----
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0 && *abort_flag != 0) atomicExch(prm.status, kStatusTimeout);
+    if (tid == 0) finish_cta(prm.status, *abort_flag != 0, prm.counter);
     if (warp == 8) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 

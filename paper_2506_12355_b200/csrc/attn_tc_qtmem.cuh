@@ -67,7 +67,7 @@ struct QTmemParams {
     int H, Hkv;
     int k_offset;           // global index of key 0 of this K/V shard; enters the causal mask
     int n_items;            // n_qtiles * BH
-    unsigned int* counter;  // work counter, zero at launch; NULL when n_items <= grid
+    unsigned int* counter;  // work counter {next item, CTAs done}, zero at launch and again at exit; NULL when n_items <= grid
 };
 
 // One work item, decoded identically by every role.
@@ -592,7 +592,7 @@ attn_fwd_tc_qtmem_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     // ---- teardown (also reached after a timed-out wait) ----
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0 && *abort_flag != 0) atomicExch(prm.status, kStatusTimeout);
+    if (tid == 0) finish_cta(prm.status, *abort_flag != 0, prm.counter);
     if (warp == 4) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 

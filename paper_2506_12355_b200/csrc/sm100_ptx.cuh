@@ -69,8 +69,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Longest time any single wait may take before the CTA gives up (nanoseconds).
+// Longest time any single wait may take before the CTA gives up (nanoseconds): one second of wall
+// clock.  ATTN_TEST_WAIT_LIMIT_NS shortens it in the separate test build that makes a wait run out.
+#ifdef ATTN_TEST_WAIT_LIMIT_NS
+constexpr uint64_t kWaitLimitNs = ATTN_TEST_WAIT_LIMIT_NS;
+#else
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+#endif
 
 // Bounded wait.  Returns false (and raises *abort_flag) when the limit expires or
 // another thread of the CTA has already given up.

@@ -434,6 +434,72 @@ def test_cuda_graph_capture_and_replay():
     assert torch.equal(o.view(torch.int16), ref_o.view(torch.int16)) and torch.equal(lse, ref_l)
 
 
+def test_many_launches_on_one_stream_while_a_long_launch_runs_on_another():
+    # work counters belong to streams: 1100 counted launches on one stream (more than any ring of counters
+    # would hold) next to one long launch on another stream; every result must be bit-equal to a quiet run
+    dev = torch.device("cuda:0")
+    ql, kl, vl = (t.to(dev) for t in inputs.make_qkv(1, 4, 16384, 16384, 128, inputs.DTYPE_BF16, seed=140))
+    qs, ks, vs = (t.to(dev) for t in inputs.make_qkv(2, 40, 512, 512, 64, inputs.DTYPE_FP16, seed=141))   # 160 items
+    ref_long = api.attn_fwd(ql, kl, vl, 0.09, True)
+    ref_short = api.attn_fwd(qs, ks, vs, 0.125, False)
+    torch.cuda.synchronize()
+    s_long, s_short = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    o_long = torch.empty_like(ql)
+    l_long = torch.empty(1, 4, 16384, dtype=torch.float32, device=dev)
+    o_short = torch.empty_like(qs)
+    l_short = torch.empty(2, 40, 512, dtype=torch.float32, device=dev)
+    mismatches = torch.zeros(1, dtype=torch.int64, device=dev)
+    for rep in range(4):
+        for _ in range(3):
+            api.attn_fwd(ql, kl, vl, 0.09, True, out=o_long, lse=l_long, stream=s_long)
+        with torch.cuda.stream(s_short):
+            for i in range(275):
+                api.attn_fwd(qs, ks, vs, 0.125, False, out=o_short, lse=l_short, stream=s_short)
+                if i % 25 == 0:
+                    mismatches += (o_short.view(torch.int16) != ref_short[0].view(torch.int16)).sum() + (l_short != ref_short[1]).sum()
+        s_long.synchronize()
+        assert torch.equal(o_long.view(torch.int16), ref_long[0].view(torch.int16)) and torch.equal(l_long, ref_long[1])
+    torch.cuda.synchronize()
+    assert api.attn_last_device_status() == 0
+    assert int(mismatches.item()) == 0
+    assert torch.equal(o_short.view(torch.int16), ref_short[0].view(torch.int16)) and torch.equal(l_short, ref_short[1])
+
+
+def test_graph_of_a_counted_launch_replays_next_to_eager_launches():
+    # a captured launch with more work items than SMs keeps a work counter of its own: replayed on one stream
+    # while eager launches of another problem run on a second stream, all results stay bit-equal
+    dev = torch.device("cuda:0")
+    cfg = inputs.CONFIGS["C3"]
+    q, k, v = (t.to(dev) for t in inputs.make_config_inputs(cfg))
+    q2, k2, v2 = (t.to(dev) for t in inputs.make_qkv(2, 40, 512, 512, 64, inputs.DTYPE_FP16, seed=151))
+    ref = api.attn_fwd(q, k, v, cfg.scale, cfg.causal)
+    ref2 = api.attn_fwd(q2, k2, v2, 0.125, False)
+    torch.cuda.synchronize()
+    o = torch.empty_like(q)
+    lse = torch.empty(cfg.B, cfg.H, cfg.Sq, dtype=torch.float32, device=dev)
+    st, st2 = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            api.attn_fwd(q, k, v, cfg.scale, cfg.causal, out=o, lse=lse, stream=st)
+    o2 = torch.empty_like(q2)
+    l2 = torch.empty(2, 40, 512, dtype=torch.float32, device=dev)
+    bad = torch.zeros(1, dtype=torch.int64, device=dev)      # one tally per stream
+    bad2 = torch.zeros(1, dtype=torch.int64, device=dev)
+    for rep in range(20):
+        with torch.cuda.stream(st):
+            o.zero_()
+            g.replay()
+            bad += (o.view(torch.int16) != ref[0].view(torch.int16)).sum() + (lse != ref[1]).sum()
+        with torch.cuda.stream(st2):
+            for _ in range(60):
+                api.attn_fwd(q2, k2, v2, 0.125, False, out=o2, lse=l2, stream=st2)
+            bad2 += (o2.view(torch.int16) != ref2[0].view(torch.int16)).sum() + (l2 != ref2[1]).sum()
+    torch.cuda.synchronize()
+    assert api.attn_last_device_status() == 0
+    assert int(bad.item()) == 0 and int(bad2.item()) == 0
+
+
 # ------------------------------------------------------------------ merge of parts behind separate pointers
 
 @pytest.mark.parametrize("n_parts,dtype,D", [(1, 1, 128), (2, 0, 64), (5, 1, 128), (8, 0, 256)])

@@ -456,6 +456,104 @@ int attn_oracle_rows_e4m3(const uint8_t *q, const uint8_t *k, const uint8_t *v, 
     return failed ? -1 : 0;
 }
 
+/* ---- backward pass: gradients of the same operator ----------------------- */
+
+/* Gradients of O = Softmax(Mask(scale Q K^T)) V (the operator of Section 2.2; the paper measures the forward
+ * pass only, so this is the plain chain rule applied to that definition) with respect to Q, K and V,
+ * given dO = dL/dO.  One query row at a time, nothing reused from a forward pass:
+ *
+ *     s_j  = scale <q_i, k_j>             p_j = exp(s_j - m) / sum_j' exp(s_j' - m)      (visible j)
+ *     dp_j = <dO_i, v_j>                  (O_i = sum_j p_j v_j       =>  dL/dp_j)
+ *     ds_j = p_j (dp_j - sum_j' p_j' dp_j')                          (softmax Jacobian)
+ *     dq_i = scale sum_j ds_j k_j         dk_j += scale ds_j q_i     dv_j += p_j dO_i
+ *
+ * q, dout, dq: [B,H,Sq,D]; k, v, dk, dv: [B,Hkv,Sk,D] with H % Hkv == 0 (query head h reads K/V head
+ * h / (H / Hkv), so dk and dv collect the contributions of all query heads of their group).
+ * Top-left causal mask as in the forward pass.  Rows without a visible key contribute nothing.
+ * Returns 0, -1 when scratch cannot be allocated, -2 for bad head counts.
+ * Parallel over (batch, K/V head): each thread owns the dk, dv rows it accumulates into. */
+int attn_oracle_bwd_f64(const double *q, const double *k, const double *v, const double *dout, double *dq,
+                        double *dk, double *dv, int B, int H, int Hkv, int Sq, int Sk, int D, double scale,
+                        int causal)
+{
+    if (Hkv <= 0 || H % Hkv != 0)
+        return -2;
+    int group = H / Hkv;
+    int64_t n_kv_heads = (int64_t)B * Hkv;
+    int failed = 0;
+    int64_t g;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (g = 0; g < n_kv_heads; ++g) {
+        size_t nk = (size_t)(Sk > 0 ? Sk : 1);
+        double *p = (double *)malloc(sizeof(double) * nk);
+        double *dp = (double *)malloc(sizeof(double) * nk);
+        if (!p || !dp) {
+#pragma omp atomic write
+            failed = 1;
+            free(p);
+            free(dp);
+            continue;
+        }
+        int64_t b = g / Hkv, hk = g % Hkv;
+        const double *kh = k + g * Sk * D, *vh = v + g * Sk * D;
+        double *dkh = dk + g * Sk * D, *dvh = dv + g * Sk * D;
+        int64_t j, i;
+        int d, hq;
+        for (j = 0; j < (int64_t)Sk * D; ++j) {
+            dkh[j] = 0.0;
+            dvh[j] = 0.0;
+        }
+        for (hq = 0; hq < group; ++hq) {
+            int64_t bh = b * H + hk * group + hq;
+            for (i = 0; i < Sq; ++i) {
+                const double *qi = q + (bh * Sq + i) * D, *doi = dout + (bh * Sq + i) * D;
+                double *dqi = dq + (bh * Sq + i) * D;
+                int64_t n_vis = visible_keys(i, Sk, causal);
+                for (d = 0; d < D; ++d)
+                    dqi[d] = 0.0;
+                if (n_vis <= 0)
+                    continue;
+                /* forward quantities of this row: p_j */
+                double m = -INFINITY, l = 0.0;
+                for (j = 0; j < n_vis; ++j) {
+                    double acc = 0.0;
+                    for (d = 0; d < D; ++d)
+                        acc += qi[d] * kh[j * D + d];
+                    p[j] = scale * acc;
+                    if (p[j] > m)
+                        m = p[j];
+                }
+                for (j = 0; j < n_vis; ++j) {
+                    p[j] = exp(p[j] - m);
+                    l += p[j];
+                }
+                for (j = 0; j < n_vis; ++j)
+                    p[j] /= l;
+                /* dp_j = <dO_i, v_j>, and the row's sum_j p_j dp_j */
+                double pdp = 0.0;
+                for (j = 0; j < n_vis; ++j) {
+                    double acc = 0.0;
+                    for (d = 0; d < D; ++d)
+                        acc += doi[d] * vh[j * D + d];
+                    dp[j] = acc;
+                    pdp += p[j] * acc;
+                }
+                for (j = 0; j < n_vis; ++j) {
+                    double ds = p[j] * (dp[j] - pdp);
+                    for (d = 0; d < D; ++d) {
+                        dqi[d] += scale * ds * kh[j * D + d];
+                        dkh[j * D + d] += scale * ds * qi[d];
+                        dvh[j * D + d] += p[j] * doi[d];
+                    }
+                }
+            }
+        }
+        free(p);
+        free(dp);
+    }
+    return failed ? -1 : 0;
+}
+
 int oracle_num_threads(void)
 {
 #ifdef _OPENMP

@@ -70,6 +70,8 @@ def _load():
                                               i64p, ctypes.c_int64, dp, dp] + [ctypes.c_int] * 6 + [
                                                   ctypes.c_double, ctypes.c_int]
         lib.attn_oracle_rows_e4m3.restype = ctypes.c_int
+        lib.attn_oracle_bwd_f64.restype = ctypes.c_int
+        lib.attn_oracle_bwd_f64.argtypes = [dp] * 7 + [ctypes.c_int] * 6 + [ctypes.c_double, ctypes.c_int]
         lib.oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -183,6 +185,26 @@ def combine(o_parts, lse_parts):
     lse = np.empty(lse_parts.shape[1:], dtype=np.float64)
     _load().attn_oracle_combine_f64(_dptr(o_parts), _dptr(lse_parts), n, _dptr(o), _dptr(lse), rows, D)
     return o, lse
+
+
+def attention_bwd(q, k, v, dout, scale: float, causal: bool):
+    """Gradients (dq, dk, dv) of the attention output with respect to q, k, v for the upstream gradient
+    dout = dL/dO, by the chain rule on the definition.  q, dout: [B,H,Sq,D]; k, v: [B,Hkv,Sk,D] (float64)."""
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    k = np.ascontiguousarray(k, dtype=np.float64)
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    dout = np.ascontiguousarray(dout, dtype=np.float64)
+    B, H, Sq, D = q.shape
+    Hkv, Sk = k.shape[1], k.shape[2]
+    assert k.shape == (B, Hkv, Sk, D) and v.shape == (B, Hkv, Sk, D) and dout.shape == q.shape
+    dq, dk, dv = np.empty_like(q), np.empty_like(k), np.empty_like(v)
+    rc = _load().attn_oracle_bwd_f64(_dptr(q), _dptr(k), _dptr(v), _dptr(dout), _dptr(dq), _dptr(dk), _dptr(dv),
+                                     B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)))
+    if rc == -2:
+        raise ValueError("H must be a multiple of Hkv")
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return dq, dk, dv
 
 
 def attention_rows_16(q_bits, k_bits, v_bits, dtype: int, rows, scale: float, causal: bool):

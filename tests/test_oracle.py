@@ -410,3 +410,108 @@ def test_fp8_input_generator_is_seeded_clamped_and_rounded():
     assert np.all(err <= np.maximum(np.abs(x.numpy()) * 2.0 ** -4, 2.0 ** -10))
     big = inputs.randn8((1000,), 5, sigma=1000.0)
     assert np.nanmax(np.abs(orc.widen_e4m3(big.numpy()))) == 448.0
+
+
+# ------------------------------------------------------------------ backward pass (gradients of the same operator)
+
+def _loss(q, k, v, dout, scale, causal, gqa):
+    """sum(O * dout) through the oracle's FORWARD entries: its gradients are what attention_bwd must return."""
+    o, _ = (orc.attention_gqa if gqa else orc.attention)(q, k, v, scale, causal)
+    return float((o * dout).sum())
+
+
+@pytest.mark.parametrize("mode", ["noncausal", "causal"])
+def test_bwd_hand_case_2x2(mode):
+    g = json.load(open(GOLDEN))
+    c, b = g["case_2x2"], g["case_2x2_bwd"]
+    q, k, v, dout = (_mat(m)[None, None] for m in (c["Q"], c["K"], c["V"], b["dO"]))
+    dq, dk, dv = orc.attention_bwd(q, k, v, dout, c["scale"], mode == "causal")
+    np.testing.assert_allclose(dq[0, 0], _mat(b[mode]["dQ"]), rtol=0, atol=1e-14)
+    np.testing.assert_allclose(dk[0, 0], _mat(b[mode]["dK"]), rtol=0, atol=1e-14)
+    np.testing.assert_allclose(dv[0, 0], _mat(b[mode]["dV"]), rtol=0, atol=1e-14)
+    if mode == "noncausal":   # digits worked out separately: 2e/(e+1)^2
+        np.testing.assert_allclose(dq[0, 0, 0, 1], b["literal_g"], rtol=0, atol=1e-15)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("shape", [(1, 1, 1, 3, 5, 4), (2, 2, 2, 4, 4, 3), (1, 4, 2, 5, 3, 2), (1, 2, 1, 3, 7, 4)])
+def test_bwd_matches_central_finite_differences(shape, causal):
+    # every entry of dq, dk, dv against (L(x + h) - L(x - h)) / 2h of the forward oracle, L = sum(O * dout)
+    B, H, Hkv, Sq, Sk, D = shape
+    q, k, v, dout = rand((B, H, Sq, D), 1), rand((B, Hkv, Sk, D), 2), rand((B, Hkv, Sk, D), 3), rand((B, H, Sq, D), 4)
+    scale = 0.7
+    dq, dk, dv = orc.attention_bwd(q, k, v, dout, scale, causal)
+    h = 1e-6
+    for name, x, grad in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        num = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            keep = x[idx]
+            x[idx] = keep + h
+            up = _loss(q, k, v, dout, scale, causal, True)
+            x[idx] = keep - h
+            dn = _loss(q, k, v, dout, scale, causal, True)
+            x[idx] = keep
+            num[idx] = (up - dn) / (2 * h)
+        np.testing.assert_allclose(grad, num, rtol=0, atol=2e-8, err_msg="d" + name)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("H,Hkv", [(3, 3), (4, 2), (4, 1)])
+def test_bwd_against_torch_autograd_fp64(H, Hkv, causal):
+    B, Sq, Sk, D = 2, 33, 47, 16
+    q, k, v, dout = rand((B, H, Sq, D), 11), rand((B, Hkv, Sk, D), 12), rand((B, Hkv, Sk, D), 13), rand((B, H, Sq, D), 14)
+    scale = 0.31
+    dq, dk, dv = orc.attention_bwd(q, k, v, dout, scale, causal)
+    tq, tk, tv = (torch.from_numpy(x).clone().requires_grad_(True) for x in (q, k, v))
+    # library attention in fp64 with an explicit top-left mask (Sq != Sk), K/V heads repeated for the groups
+    rep = H // Hkv
+    s = torch.einsum("bhid,bhjd->bhij", tq, tk.repeat_interleave(rep, dim=1)) * scale
+    if causal:
+        mask = torch.arange(Sk)[None, :] > torch.arange(Sq)[:, None]
+        s = s.masked_fill(mask, float("-inf"))
+    o = torch.einsum("bhij,bhjd->bhid", torch.softmax(s, dim=-1), tv.repeat_interleave(rep, dim=1))
+    o.backward(torch.from_numpy(dout))
+    np.testing.assert_allclose(dq, tq.grad.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(dk, tk.grad.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(dv, tv.grad.numpy(), rtol=0, atol=1e-12)
+
+
+def test_bwd_invariants():
+    B, H, Sq, Sk, D = 1, 2, 9, 11, 4
+    q, k, v, dout = rand((B, H, Sq, D), 21), rand((B, H, Sk, D), 22), rand((B, H, Sk, D), 23), rand((B, H, Sq, D), 24)
+    # constant V: O does not depend on the probabilities, so no gradient reaches Q and K, and the
+    # probability rows sum to one: sum_j dv_j = sum_i dO_i
+    vc = np.broadcast_to(rand((B, H, 1, D), 25), (B, H, Sk, D)).copy()
+    dq, dk, dv = orc.attention_bwd(q, k, vc, dout, 0.5, True)
+    assert np.abs(dq).max() < 1e-14 and np.abs(dk).max() < 1e-14
+    np.testing.assert_allclose(dv.sum(axis=2), dout.sum(axis=2), atol=1e-13)
+    # identical keys: the scores of a row are all equal, dq_i = scale * (sum_j ds_j) * k0 = 0
+    kc = np.broadcast_to(rand((B, H, 1, D), 26), (B, H, Sk, D)).copy()
+    dq, _, dv = orc.attention_bwd(q, kc, v, dout, 0.5, False)
+    assert np.abs(dq).max() < 1e-14
+    np.testing.assert_allclose(dv, np.broadcast_to(dout.sum(axis=2, keepdims=True) / Sk, dv.shape), atol=1e-13)
+    # causal, Sq == Sk: the last key is seen by the last row only; rows see nothing beyond themselves
+    q2, d2 = rand((B, H, Sk, D), 27), rand((B, H, Sk, D), 28)
+    dq, dk, dv = orc.attention_bwd(q2, k, v, d2, 0.5, True)
+    assert np.abs(dq[:, :, 0]).max() < 1e-14          # row 0 sees one key: constant softmax
+    # dv of the last key = p(last row, last key) * dO(last row), with p written out here
+    s_last = 0.5 * np.einsum("bhd,bhjd->bhj", q2[:, :, -1], k)
+    p_last = np.exp(s_last - s_last.max(-1, keepdims=True))
+    p_last /= p_last.sum(-1, keepdims=True)
+    np.testing.assert_allclose(dv[:, :, -1], p_last[:, :, -1:] * d2[:, :, -1], atol=1e-14)
+    # scaling the loss scales every gradient; zero upstream gradient gives zero gradients
+    g1 = orc.attention_bwd(q, k, v, dout, 0.5, True)
+    g3 = orc.attention_bwd(q, k, v, 3.0 * dout, 0.5, True)
+    for a, b3 in zip(g1, g3):
+        np.testing.assert_allclose(3.0 * a, b3, atol=1e-13)
+    for a in orc.attention_bwd(q, k, v, np.zeros_like(dout), 0.5, True):
+        assert np.abs(a).max() == 0.0
+
+
+def test_bwd_rejects_indivisible_heads_and_handles_no_keys():
+    with pytest.raises(ValueError):
+        orc.attention_bwd(rand((1, 3, 2, 2), 1), rand((1, 2, 2, 2), 2), rand((1, 2, 2, 2), 3), rand((1, 3, 2, 2), 4), 1.0, False)
+    dq, dk, dv = orc.attention_bwd(rand((1, 1, 3, 2), 1), np.zeros((1, 1, 0, 2)), np.zeros((1, 1, 0, 2)), rand((1, 1, 3, 2), 4), 1.0, True)
+    assert dq.shape == (1, 1, 3, 2) and np.abs(dq).max() == 0.0 and dk.size == 0 and dv.size == 0

@@ -210,6 +210,37 @@ int attn_fwd_fp8(const void* q, const void* k, const void* v, void* o, float* ls
                  void* stream);
 
 /*
+ * attn_bwd -- backward pass: the gradients of the operator of Section 2.2,
+ * O = Softmax(Mask(scale Q K^T)) V, with respect to Q, K and V for an upstream gradient dO = dL/dO.
+ * (The paper measures the forward pass only; this is the chain rule applied to its definition.)
+ *
+ *     P = exp(scale Q K^T - LSE)  (visible keys; 0 elsewhere)      dP = dO V^T
+ *     dS = P o (dP - rowsum(dO o O))       dV = P^T dO       dQ = scale dS K       dK = scale dS^T Q
+ *
+ * q, o, dout : device, [B,H,Sq,D] (`dtype`), 16-byte aligned; o and lse are the OUTPUTS of the forward call
+ *              (attn_fwd / attn_fwd_gqa) on the same q, k, v, scale and mask.
+ * k, v       : device, [B,Hkv,Sk,D]; H % Hkv == 0 (grouped heads as in attn_fwd_gqa).
+ * lse        : device, [B,H,Sq] fp32.
+ * dq         : device, [B,H,Sq,D] (written);  dk, dv: device, [B,Hkv,Sk,D] (written; with grouped heads
+ *              they hold the sum over the query heads of the group).  Same 16-bit type as the inputs.
+ * D in {64, 128} (otherwise ATTN_ERR_UNSUPPORTED_HEAD_DIM); top-left causal mask as in attn_fwd.
+ * workspace  : device, 256-byte aligned, at least attn_bwd_workspace_bytes(B,H,Sq) bytes (it holds
+ *              rowsum(dO o O) in fp32); owned by the caller, may be reused as soon as the stream has
+ *              passed this call.  Missing, misaligned or too small: ATTN_ERR_WORKSPACE.
+ * Rows of dq whose query sees no key, and rows of dk, dv whose key no query sees, are zero.  Empty
+ * tensors may come with NULL pointers.  Three kernels are enqueued on `stream` (the row sums, the dQ
+ * pass, the dK/dV pass); nothing is synchronised; the results are deterministic (no atomics).
+ * Accumulation is fp32; P and dS are rounded to the 16-bit type before their second products.
+ * Errors: as attn_fwd_gqa, plus the above.
+ */
+int attn_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout,
+             void* dq, void* dk, void* dv, int B, int H, int Hkv, int Sq, int Sk, int D, float scale, int causal,
+             int dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of device workspace attn_bwd needs (0 for an invalid shape). */
+size_t attn_bwd_workspace_bytes(int B, int H, int Sq);
+
+/*
  * attn_fwd_simt -- same operator, same arguments, same conventions, computed by a plain
  * CUDA-core kernel (one warp per query row, fp32 arithmetic, online softmax).  It is one to
  * two orders of magnitude slower than attn_fwd and exists as an on-device cross-check that

@@ -25,7 +25,7 @@ STATUS_NAMES = {
 }
 
 # every symbol include/attn_fwd.h declares
-EXPORTS = ["attn_fwd", "attn_fwd_gqa", "attn_fwd_partial", "attn_combine", "attn_combine_gather", "attn_fwd_qkv_dims", "attn_fwd_splitkv", "attn_fwd_splitkv_workspace_bytes", "attn_fwd_fp8", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
+EXPORTS = ["attn_bwd", "attn_bwd_workspace_bytes", "attn_fwd", "attn_fwd_gqa", "attn_fwd_partial", "attn_combine", "attn_combine_gather", "attn_fwd_qkv_dims", "attn_fwd_splitkv", "attn_fwd_splitkv_workspace_bytes", "attn_fwd_fp8", "attn_fwd_simt", "attn_fwd_host", "attn_fwd_host_workspace_bytes",
            "attn_fwd_host_static", "attn_fwd_host_static_capacity",
            "attn_query_support", "attn_last_device_status", "attn_status_string"]
 
@@ -72,6 +72,10 @@ def load() -> ctypes.CDLL:
     lib.attn_fwd_splitkv_workspace_bytes.argtypes = [i] * 5
     lib.attn_fwd_fp8.restype = i
     lib.attn_fwd_fp8.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, f, f, f, f, i, i, vp]
+    lib.attn_bwd.restype = i
+    lib.attn_bwd.argtypes = [vp] * 9 + [i] * 6 + [f, i, i, vp, ctypes.c_size_t, vp]
+    lib.attn_bwd_workspace_bytes.restype = ctypes.c_size_t
+    lib.attn_bwd_workspace_bytes.argtypes = [i] * 3
     lib.attn_fwd_simt.restype = i
     lib.attn_fwd_simt.argtypes = sig
     lib.attn_fwd_host.restype = i
@@ -321,6 +325,43 @@ def attn_fwd_fp8(q, k, v, scale: float, q_factor: float = 1.0, k_factor: float =
     if rc != 0:
         raise AttnError(rc, "attn_fwd_fp8")
     return out, lse
+
+
+def attn_bwd_workspace_bytes(B, H, Sq) -> int:
+    return int(load().attn_bwd_workspace_bytes(B, H, Sq))
+
+
+def attn_bwd(q, k, v, o, lse, dout, scale: float, causal: bool = False, dq=None, dk=None, dv=None, workspace=None,
+             stream=None):
+    """Gradients (dq, dk, dv) of the attention output for the upstream gradient dout: q, o, dout [B,H,Sq,D];
+    k, v [B,Hkv,Sk,D]; lse [B,H,Sq] fp32; o and lse from the forward call on the same inputs.  D in {64, 128}.
+    `workspace`: CUDA uint8 tensor of at least attn_bwd_workspace_bytes(B, H, Sq) bytes (allocated here when None)."""
+    if q.dim() != 4 or k.dim() != 4 or tuple(v.shape) != tuple(k.shape):
+        raise ValueError("q must be [B,H,Sq,D]; k, v must be [B,Hkv,Sk,D]")
+    B, H, Sq, D = q.shape
+    Hkv, Sk = k.shape[1], k.shape[2]
+    if k.shape[0] != B or k.shape[3] != D or tuple(o.shape) != tuple(q.shape) or tuple(dout.shape) != tuple(q.shape):
+        raise ValueError("k, v must match q's B and D; o and dout must have q's shape")
+    if tuple(lse.shape) != (B, H, Sq) or lse.dtype != torch.float32:
+        raise ValueError("lse must be fp32 [B,H,Sq]")
+    for t in (q, k, v, o, dout, lse):
+        if not (t.is_cuda and t.is_contiguous()):
+            raise ValueError("all tensors must be contiguous CUDA tensors")
+    if not (q.dtype == k.dtype == v.dtype == o.dtype == dout.dtype):
+        raise TypeError("q, k, v, o, dout must share one dtype")
+    dt = _dtype_code(q)
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    if workspace is None:
+        workspace = torch.empty(max(attn_bwd_workspace_bytes(B, H, Sq), 256), dtype=torch.uint8, device=q.device)
+    with torch.cuda.device(q.device):
+        rc = load().attn_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dout.data_ptr(),
+                             dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, H, Hkv, Sq, Sk, D, float(scale),
+                             int(bool(causal)), dt, workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_bwd")
+    return dq, dk, dv
 
 
 def attn_fwd_simt(q, k, v, scale: float, causal: bool = False, out=None, lse=None, stream=None):

@@ -15,6 +15,7 @@
 #include <vector>
 
 #include "../../include/attn_fwd.h"
+#include "attn_bwd.cuh"
 #include "attn_combine.cuh"
 #include "attn_simt.cuh"
 #include "attn_tc_qtmem.cuh"
@@ -788,6 +789,93 @@ int attn_fwd_fp8(const void* q, const void* k, const void* v, void* o, float* ls
     if (impl == 1)
         return launch_simt<128, ATTN_DTYPE_FP8_E4M3>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, s_eff, causal, 0, st, v_factor);
     return launch_tc_pipe<128, ATTN_DTYPE_FP8_E4M3>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, s_eff, causal, 0, st, v_factor);
+}
+
+size_t attn_bwd_workspace_bytes(int B, int H, int Sq) {
+    if (B < 0 || H < 0 || Sq < 0) return 0;
+    return align256(static_cast<size_t>(B) * H * Sq * sizeof(float));
+}
+
+int attn_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout, void* dq,
+             void* dk, void* dv, int B, int H, int Hkv, int Sq, int Sk, int D, float scale, int causal, int dtype,
+             void* workspace, size_t workspace_bytes, void* stream) {
+    if (D != 64 && D != 128) {
+        if (B < 0 || H < 0 || Hkv < 0 || Sq < 0 || Sk < 0 || D < 0) return ATTN_ERR_BAD_SHAPE;
+        return ATTN_ERR_UNSUPPORTED_HEAD_DIM;
+    }
+    // the shared checks on q, k, v (dq stands in for o, the caller's lse is checked as a float pointer)
+    int rc = validate(q, k, v, dq, lse, B, H, Hkv, Sq, Sk, D, scale, dtype, true);
+    if (rc != ATTN_OK) return rc;
+    const size_t n_q = static_cast<size_t>(B) * H * Sq, n_kv = static_cast<size_t>(B) * Hkv * Sk;
+    if (n_q > 0 && (!o || !dout)) return ATTN_ERR_NULL_POINTER;
+    if (n_kv > 0 && (!dk || !dv)) return ATTN_ERR_NULL_POINTER;
+    if ((reinterpret_cast<uintptr_t>(o) | reinterpret_cast<uintptr_t>(dout) | reinterpret_cast<uintptr_t>(dk) |
+         reinterpret_cast<uintptr_t>(dv)) & 15u)
+        return ATTN_ERR_MISALIGNED;
+    if (n_q == 0 && n_kv == 0) return ATTN_OK;
+    if (n_q > 0 && n_kv > 0 &&
+        (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < attn_bwd_workspace_bytes(B, H, Sq)))
+        return ATTN_ERR_WORKSPACE;
+    rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // no queries: nothing reaches K and V; no keys: nothing reaches Q
+    if (n_q == 0 || n_kv == 0) {
+        if (n_kv > 0 && (cudaMemsetAsync(dk, 0, n_kv * D * 2, st) != cudaSuccess || cudaMemsetAsync(dv, 0, n_kv * D * 2, st) != cudaSuccess))
+            return ATTN_ERR_CUDA;
+        if (n_q > 0 && cudaMemsetAsync(dq, 0, n_q * D * 2, st) != cudaSuccess) return ATTN_ERR_CUDA;
+        return ATTN_OK;
+    }
+    const int64_t BH = static_cast<int64_t>(B) * H, BHkv = static_cast<int64_t>(B) * Hkv;
+    const int64_t n_qtiles = (static_cast<int64_t>(Sq) + 127) / 128, n_ktiles = (static_cast<int64_t>(Sk) + 127) / 128;
+    if (n_qtiles * BH > 2147483647LL || n_ktiles * BHkv > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
+    float* delta = static_cast<float*>(workspace);
+    attn_grad::BwdParams prm;
+    prm.lse = lse;
+    prm.delta = delta;
+    prm.Sq = Sq;
+    prm.Sk = Sk;
+    prm.scale = scale;
+    prm.scale_log2 = scale * 1.4426950408889634f;
+    prm.causal = causal ? 1 : 0;
+    prm.H = H;
+    prm.Hkv = Hkv;
+    prm.n_qtiles = static_cast<int>(n_qtiles);
+    prm.n_ktiles = static_cast<int>(n_ktiles);
+    prm.status = device_status_ptr();
+    if (!prm.status) return ATTN_ERR_CUDA;
+    CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
+    if (!make_map(&mq, q, dtype, BH, Sq, D, 128) || !make_map(&mdo, dout, dtype, BH, Sq, D, 128) ||
+        !make_map(&mdq, dq, dtype, BH, Sq, D, 128) || !make_map(&mk, k, dtype, BHkv, Sk, D, 128) ||
+        !make_map(&mv, v, dtype, BHkv, Sk, D, 128) || !make_map(&mdk, dk, dtype, BHkv, Sk, D, 128) ||
+        !make_map(&mdv, dv, dtype, BHkv, Sk, D, 128))
+        return ATTN_ERR_CUDA;
+#define ATTN_BWD_CASE(DD, TT)                                                                                              \
+    if (D == DD && dtype == TT) {                                                                                          \
+        using C = attn_grad::BwdCfg<DD>;                                                                                    \
+        auto kq = attn_grad::attn_bwd_kernel<DD, TT, 0>;                                                                    \
+        auto kkv = attn_grad::attn_bwd_kernel<DD, TT, 1>;                                                                   \
+        if (!allow_dynamic_smem(reinterpret_cast<const void*>(kq), C::SMEM_BYTES) ||                                       \
+            !allow_dynamic_smem(reinterpret_cast<const void*>(kkv), C::SMEM_BYTES))                                        \
+            return ATTN_ERR_CUDA;                                                                                          \
+        const int64_t rows = BH * Sq;                                                                                      \
+        int64_t blocks = (rows + 7) / 8;                                                                                   \
+        if (blocks > 148 * 16) blocks = 148 * 16;                                                                          \
+        attn_grad::attn_bwd_delta_kernel<DD, TT><<<static_cast<unsigned>(blocks), 256, 0, st>>>(o, dout, delta, rows);        \
+        prm.out0 = dq;                                                                                                     \
+        prm.out1 = nullptr;                                                                                                \
+        kq<<<static_cast<unsigned>(n_qtiles * BH), C::THREADS, C::SMEM_BYTES, st>>>(mq, mdo, mk, mv, mdq, mdq, prm);       \
+        prm.out0 = dv;                                                                                                     \
+        prm.out1 = dk;                                                                                                     \
+        kkv<<<static_cast<unsigned>(n_ktiles * BHkv), C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mq, mdo, mdv, mdk, prm);    \
+        return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;                                                \
+    }
+    ATTN_BWD_CASE(64, 0)
+    ATTN_BWD_CASE(64, 1)
+    ATTN_BWD_CASE(128, 0)
+    ATTN_BWD_CASE(128, 1)
+#undef ATTN_BWD_CASE
+    return ATTN_ERR_UNSUPPORTED_DTYPE;
 }
 
 int attn_fwd_simt(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int Sq, int Sk,

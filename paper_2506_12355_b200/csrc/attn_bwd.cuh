@@ -1,0 +1,442 @@
+// Backward pass of the attention operator on tcgen05 tensor cores (head dims 64 and 128).
+//
+// Gradients of O = Softmax(Mask(scale Q K^T)) V (Section 2.2 of the paper; the paper itself measures the
+// forward pass only) for an upstream gradient dO, from Q, K, V, O, dO and the forward pass's per-row
+// logsumexp L:
+//
+//     P  = exp(scale Q K^T - L)           dP = dO V^T            delta_i = sum_d dO_id O_id
+//     dS = P o (dP - delta)               dV = P^T dO            dQ = scale dS K        dK = scale dS^T Q
+//
+// Two passes over the score tiles, each the forward loop of Appendix C's listings with other operands (one
+// tile resident, the other side streamed through a TMA ring, the S x S matrices never leave the SM):
+//
+//   MODE 0 (dQ):      CTA = one 128-row Q tile; Q_i, dO_i resident; K_j, V_j streamed.
+//                     S = Q_i K_j^T and dP = dO_i V_j^T (both operands in shared memory) -> tensor memory;
+//                     one thread per query row turns them into dS (16-bit, written over S);
+//                     dQ += dS K_j with dS read from tensor memory, K_j as the MN-major operand.
+//   MODE 1 (dK, dV):  CTA = one 128-key K/V tile; K_j, V_j resident; Q_i, dO_i streamed (all query heads of
+//                     the K/V head's group).  The TRANSPOSED tiles S^T = K_j Q_i^T and dP^T = V_j dO_i^T are
+//                     computed, so that P^T and dS^T land in tensor memory with keys on the lanes, which is
+//                     the A operand that dV += P^T dO_i and dK += dS^T Q_i need; one thread per key row, the
+//                     per-query L and delta come from shared memory.
+//
+// Recomputing S and dP in both passes costs 7 tile products instead of 5 but needs no atomics and no
+// cross-CTA reduction, so the results are deterministic.  delta is computed by a small kernel first.
+//
+//   warps 0-3  element-wise group (one thread per tensor-memory lane), then the epilogue
+//   warp  4    MMA issuer
+//   warp  5    TMA producer
+//
+// Every wait is bounded (see sm100_ptx.cuh); a timed-out wait ends the CTA through the normal exit.
+#pragma once
+#include "attn_tc_common.cuh"
+
+namespace attn_grad {
+
+using namespace sm100;
+using attn_tc::finish_cta;
+
+template <int D>
+struct BwdCfg {
+    static constexpr int BT = 128;                          // rows of every tile (queries or keys)
+    static constexpr int NBOX = D / 64;                     // 128-byte wide TMA boxes per tile row
+    static constexpr int TILE_BYTES1 = BT * D * 2;          // one operand tile
+    static constexpr int NSTAGE = D == 128 ? 2 : 4;         // ring stages, each holds the two streamed tiles
+    static constexpr int OST_BYTES = BT * 128;              // epilogue staging: 128 rows x 64 columns
+    static constexpr int VEC_BYTES = 2 * 2 * BT * 4;        // MODE 1: L and delta of the streamed Q tile, two buffers
+    static constexpr int TILE_BYTES = 2 * TILE_BYTES1 + NSTAGE * 2 * TILE_BYTES1 + OST_BYTES + VEC_BYTES;
+    static constexpr int MISC_BYTES = 256;
+    static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
+    static constexpr int THREADS = 192;
+    static constexpr int S_COL = 0, DP_COL = 128, ACC0_COL = 256, ACC1_COL = 256 + D;
+    static constexpr int TMEM_COLS = 512;
+    static_assert(D == 64 || D == 128, "head dims 64 and 128");
+};
+
+struct BwdParams {
+    const float* lse;       // [B,H,Sq] natural-log logsumexp of the scaled scores, from the forward pass
+    const float* delta;     // [B,H,Sq] rowsum(dO o O)
+    void* out0;             // plain pointers of the outputs, for tiles that no step touches (zero fill):
+    void* out1;             //   MODE 0: dq, unused;  MODE 1: dv, dk
+    int Sq, Sk;
+    float scale, scale_log2;
+    int causal;
+    int H, Hkv;
+    int n_qtiles, n_ktiles;
+    int* status;
+};
+
+__device__ __forceinline__ void zero_rows(void* base, int64_t first_row, int rows, int D, int tid, int nthreads) {
+    uint4* p = reinterpret_cast<uint4*>(static_cast<uint8_t*>(base) + first_row * D * 2);
+    const int n = rows * D / 8;
+    for (int i = tid; i < n; i += nthreads) p[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+// delta_i = sum_d dO_id * O_id, one warp per row.
+template <int D, int DTYPE>
+__global__ void attn_bwd_delta_kernel(const void* __restrict__ o, const void* __restrict__ dout, float* __restrict__ delta,
+                                      int64_t rows) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = static_cast<int64_t>(gridDim.x) * (blockDim.x >> 5);
+    for (int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); row < rows; row += warps) {
+        float acc = 0.f;
+        if constexpr (D == 128) {
+            const uint2 a = reinterpret_cast<const uint2*>(static_cast<const uint8_t*>(o) + row * D * 2)[lane];
+            const uint2 b = reinterpret_cast<const uint2*>(static_cast<const uint8_t*>(dout) + row * D * 2)[lane];
+            const uint32_t aw[2] = {a.x, a.y}, bw[2] = {b.x, b.y};
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                float a0, a1, b0, b1;
+                if constexpr (DTYPE == 0) {
+                    const float2 fa = __half22float2(*reinterpret_cast<const __half2*>(&aw[i]));
+                    const float2 fb = __half22float2(*reinterpret_cast<const __half2*>(&bw[i]));
+                    a0 = fa.x; a1 = fa.y; b0 = fb.x; b1 = fb.y;
+                } else {
+                    const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[i]));
+                    const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[i]));
+                    a0 = fa.x; a1 = fa.y; b0 = fb.x; b1 = fb.y;
+                }
+                acc = fmaf(a0, b0, acc);
+                acc = fmaf(a1, b1, acc);
+            }
+        } else {
+            const uint32_t a = reinterpret_cast<const uint32_t*>(static_cast<const uint8_t*>(o) + row * D * 2)[lane];
+            const uint32_t b = reinterpret_cast<const uint32_t*>(static_cast<const uint8_t*>(dout) + row * D * 2)[lane];
+            float2 fa, fb;
+            if constexpr (DTYPE == 0) {
+                fa = __half22float2(*reinterpret_cast<const __half2*>(&a));
+                fb = __half22float2(*reinterpret_cast<const __half2*>(&b));
+            } else {
+                fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a));
+                fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
+            }
+            acc = fmaf(fa.x, fb.x, fa.y * fb.y);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (lane == 0) delta[row] = acc;
+    }
+}
+
+// tmR0 / tmR1: maps of the resident tiles (MODE 0: Q, dO; MODE 1: K, V); tmT0 / tmT1: maps of the streamed
+// tiles (MODE 0: K, V; MODE 1: Q, dO); tmOut0 / tmOut1: MODE 0: dQ, unused; MODE 1: dV, dK.
+template <int D, int DTYPE, int MODE>
+__global__ void __launch_bounds__(192, 1)
+attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant__ CUtensorMap tmR1,
+                const __grid_constant__ CUtensorMap tmT0, const __grid_constant__ CUtensorMap tmT1,
+                const __grid_constant__ CUtensorMap tmOut0, const __grid_constant__ CUtensorMap tmOut1,
+                const BwdParams prm) {
+    using C = BwdCfg<D>;
+    constexpr int BT = C::BT, NBOX = C::NBOX, NSTAGE = C::NSTAGE, T1B = C::TILE_BYTES1;
+    constexpr float LOG2E = 1.4426950408889634f;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    auto sR = [&](int w) { return smem_base + w * T1B; };                              // resident tile w (0 / 1)
+    auto sT = [&](int stage, int w) { return smem_base + (2 + 2 * stage + w) * T1B; };   // streamed tile w of a stage
+    const uint32_t sOst = smem_base + (2 + 2 * NSTAGE) * T1B;
+    float* vec = reinterpret_cast<float*>(smem_gen + (2 + 2 * NSTAGE) * T1B + C::OST_BYTES);   // [2 buffers][L2 | delta][BT]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
+    const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
+    enum { B_RFULL = 0, B_SFULL = 1, B_PFULL = 2, B_ACCFINAL = 3, B_GSYNC = 4, B_TFULL = 5, B_TEMPTY = 5 + NSTAGE, B_COUNT = 5 + 2 * NSTAGE };
+    auto bar = [&](int i) { return bars_u32 + i * 8; };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 1;
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+
+    // ---- this CTA's tile and its steps ----
+    // The grid is one-dimensional, tiles of one head next to each other (their streamed tiles are shared in L2).
+    // MODE 0: Q tile (causal: longest first) of a (batch, query head); steps = K/V tiles.
+    // MODE 1: K/V tile (the first has the most steps) of a (batch, K/V head);
+    //         steps = (query head of the group, Q tile) pairs.
+    const int group = prm.H / prm.Hkv;
+    const int tiles_per_head = MODE == 0 ? prm.n_qtiles : prm.n_ktiles;
+    const int bid_tile = static_cast<int>(blockIdx.x % static_cast<unsigned>(tiles_per_head));
+    int tile, bh_res, step_lo, step_hi, n_steps;
+    bh_res = static_cast<int>(blockIdx.x / static_cast<unsigned>(tiles_per_head));
+    if constexpr (MODE == 0) {
+        tile = prm.causal ? prm.n_qtiles - 1 - bid_tile : bid_tile;
+        const int last_key = attn_tc::last_visible_key(tile * BT + BT - 1, prm.Sk, prm.causal, 0);
+        step_lo = 0;
+        step_hi = last_key < 0 ? 0 : last_key / BT + 1;
+        n_steps = step_hi - step_lo;
+    } else {
+        tile = bid_tile;
+        step_lo = prm.causal ? tile : 0;     // first Q tile with a row that sees key tile * BT
+        step_hi = prm.n_qtiles;
+        if (step_lo > step_hi) step_lo = step_hi;
+        n_steps = (step_hi - step_lo) * group;
+    }
+    const int kv_bh_of_q = (bh_res / prm.H) * prm.Hkv + (bh_res % prm.H) / group;   // MODE 0: K/V head of this query head
+    // streamed tile of step s: (head index in its tensor, tile index)
+    auto step_head = [&](int s) {
+        if constexpr (MODE == 0) return kv_bh_of_q;
+        else return (bh_res / prm.Hkv) * prm.H + (bh_res % prm.Hkv) * group + s / (step_hi - step_lo);
+    };
+    auto step_tile = [&](int s) {
+        if constexpr (MODE == 0) return step_lo + s;
+        else return step_lo + s % (step_hi - step_lo);
+    };
+
+    if (n_steps == 0) {
+        // nothing reaches this tile (keys that no query sees, or no keys at all): the gradients are zero
+        const int rows_total = MODE == 0 ? prm.Sq : prm.Sk;
+        const int rows = rows_total - tile * BT < BT ? rows_total - tile * BT : BT;
+        if (rows > 0) {
+            const int64_t first = static_cast<int64_t>(bh_res) * rows_total + tile * BT;
+            zero_rows(prm.out0, first, rows, D, tid, C::THREADS);
+            if constexpr (MODE == 1) zero_rows(prm.out1, first, rows, D, tid, C::THREADS);
+        }
+        return;
+    }
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(B_RFULL), 1);
+        mbar_init(bar(B_SFULL), 1);
+        mbar_init(bar(B_PFULL), 128);
+        mbar_init(bar(B_ACCFINAL), 1);
+        mbar_init(bar(B_GSYNC), 128);
+        for (int s = 0; s < NSTAGE; ++s) {
+            mbar_init(bar(B_TFULL + s), 1);
+            mbar_init(bar(B_TEMPTY + s), 1);
+        }
+        fence_barrier_init();
+        fence_proxy_async_smem();
+    }
+    if (warp == 4) {
+        tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    if (warp == 5 && elect_one()) {
+        prefetch_tensormap(&tmR0);
+        prefetch_tensormap(&tmR1);
+        prefetch_tensormap(&tmT0);
+        prefetch_tensormap(&tmT1);
+        prefetch_tensormap(&tmOut0);
+        if constexpr (MODE == 1) prefetch_tensormap(&tmOut1);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 5) {
+        // =========================== TMA producer ===========================
+        const bool leader = elect_one();
+        if (leader) {
+            mbar_arrive_expect_tx(bar(B_RFULL), 2 * T1B);
+#pragma unroll
+            for (int bx = 0; bx < NBOX; ++bx) {
+                tma_load_3d(sR(0) + bx * BT * 128, &tmR0, bar(B_RFULL), bx * 64, tile * BT, bh_res);
+                tma_load_3d(sR(1) + bx * BT * 128, &tmR1, bar(B_RFULL), bx * 64, tile * BT, bh_res);
+            }
+        }
+        for (int s = 0; s < n_steps; ++s) {
+            const int st = s % NSTAGE;
+            if (!mbar_wait(bar(B_TEMPTY + st), ((s / NSTAGE) & 1) ^ 1, abort_flag)) break;
+            if (leader) {
+                mbar_arrive_expect_tx(bar(B_TFULL + st), 2 * T1B);
+                const int head = step_head(s), row0 = step_tile(s) * BT;
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx) {
+                    tma_load_3d(sT(st, 0) + bx * BT * 128, &tmT0, bar(B_TFULL + st), bx * 64, row0, head);
+                    tma_load_3d(sT(st, 1) + bx * BT * 128, &tmT1, bar(B_TFULL + st), bx * 64, row0, head);
+                }
+            }
+        }
+    } else if (warp == 4) {
+        // =========================== MMA issuer ===========================
+        const bool leader = elect_one();
+        constexpr uint32_t IDESC_S = make_idesc_f16(BT, BT, DTYPE, 0, 0);    // both operands K-major (contraction over D)
+        constexpr uint32_t IDESC_ACC = make_idesc_f16(BT, D, DTYPE, 0, 1);   // A from tensor memory, B MN-major (N = D)
+        constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
+        const uint32_t r_lo[2] = {smem_desc_lo(sR(0), 16), smem_desc_lo(sR(1), 16)};
+        bool ok = mbar_wait(bar(B_RFULL), 0, abort_flag);
+        for (int s = 0; s < n_steps && ok; ++s) {
+            const int st = s % NSTAGE;
+            if (!(ok = mbar_wait(bar(B_TFULL + st), (s / NSTAGE) & 1, abort_flag))) break;
+            tc_fence_after_sync();
+            if (leader) {
+                // S (or S^T) = R0 T0^T, dP (or dP^T) = R1 T1^T : D / 16 instructions each
+#pragma unroll
+                for (int w = 0; w < 2; ++w) {
+                    const uint32_t b0 = smem_desc_lo(sT(st, w), 16);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = ((kk >> 2) * BT * 128 + (kk & 3) * 32) >> 4;
+                        mma_f16_ss_lohi(tmem + (w == 0 ? C::S_COL : C::DP_COL), r_lo[w] + off, b0 + off, DESC_HI, IDESC_S, kk > 0);
+                    }
+                }
+                mma_commit(bar(B_SFULL));
+            }
+            if (!(ok = mbar_wait(bar(B_PFULL), s & 1, abort_flag))) break;
+            tc_fence_after_sync();
+            if (leader) {
+                if constexpr (MODE == 0) {
+                    // dQ += dS K_j : dS from tensor memory (over S), K_j MN-major
+                    const uint32_t b0 = smem_desc_lo(sT(st, 0), BT * 128);
+#pragma unroll
+                    for (int kk = 0; kk < BT / 16; ++kk)
+                        mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::S_COL + kk * 8, b0 + ((kk * 16 * 128) >> 4), DESC_HI,
+                                        IDESC_ACC, (s > 0 || kk > 0) ? 1u : 0u);
+                } else {
+                    // dV += P^T dO_i (P^T over S^T), dK += dS^T Q_i (dS^T over dP^T); dO_i and Q_i MN-major
+                    const uint32_t bdo = smem_desc_lo(sT(st, 1), BT * 128), bq = smem_desc_lo(sT(st, 0), BT * 128);
+#pragma unroll
+                    for (int kk = 0; kk < BT / 16; ++kk)
+                        mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::S_COL + kk * 8, bdo + ((kk * 16 * 128) >> 4), DESC_HI,
+                                        IDESC_ACC, (s > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int kk = 0; kk < BT / 16; ++kk)
+                        mma_f16_ts_lohi(tmem + C::ACC1_COL, tmem + C::DP_COL + kk * 8, bq + ((kk * 16 * 128) >> 4), DESC_HI,
+                                        IDESC_ACC, (s > 0 || kk > 0) ? 1u : 0u);
+                }
+                mma_commit(bar(B_TEMPTY + st));
+                if (s + 1 == n_steps) mma_commit(bar(B_ACCFINAL));
+            }
+        }
+    } else {
+        // =========================== element-wise group + epilogue ===========================
+        const int r = tid;                                   // tensor-memory lane: query row (MODE 0) / key row (MODE 1)
+        const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
+        const uint32_t tS = tmem + C::S_COL + lane_off, tDP = tmem + C::DP_COL + lane_off;
+        const float c = prm.scale_log2;
+        const int my_row = tile * BT + r;                    // global query row (MODE 0) or key index (MODE 1)
+        float my_l2 = 0.f, my_delta = 0.f;                   // MODE 0: this row's L * log2(e) and delta
+        if constexpr (MODE == 0) {
+            if (my_row < prm.Sq) {
+                const float l = prm.lse[static_cast<int64_t>(bh_res) * prm.Sq + my_row];
+                my_l2 = (l == -INFINITY) ? INFINITY : l * LOG2E;   // a row without visible keys has P = 0
+                my_delta = prm.delta[static_cast<int64_t>(bh_res) * prm.Sq + my_row];
+            }
+        }
+        bool ok = true;
+        // Barrier among the 128 threads of this group, bounded like every other wait (a plain bar.sync would
+        // wait forever for a thread that has left through the time-out path).
+        uint32_t gsync_phase = 0;
+        auto group_sync = [&]() -> bool {
+            mbar_arrive(bar(B_GSYNC));
+            const bool done = mbar_wait(bar(B_GSYNC), gsync_phase & 1, abort_flag);
+            ++gsync_phase;
+            return done;
+        };
+        for (int s = 0; s < n_steps && ok; ++s) {
+            const int t = step_tile(s);
+            float* vl2 = vec + (s & 1) * 2 * BT;
+            float* vdl = vl2 + BT;
+            if constexpr (MODE == 1) {
+                // L and delta of the streamed Q tile: one row per thread into shared memory
+                const int qr = t * BT + r;
+                float l2 = 0.f, dl = 0.f;
+                if (qr < prm.Sq) {
+                    const int64_t g = static_cast<int64_t>(step_head(s)) * prm.Sq + qr;
+                    const float l = prm.lse[g];
+                    l2 = (l == -INFINITY) ? INFINITY : l * LOG2E;
+                    dl = prm.delta[g];
+                }
+                vl2[r] = l2;
+                vdl[r] = dl;
+                if (!(ok = group_sync())) break;
+            }
+            if (!(ok = mbar_wait(bar(B_SFULL), s & 1, abort_flag))) break;
+            tc_fence_after_sync();
+            // does any element of this tile need the mask?  (uniform over the CTA)
+            //   MODE 0: rows tile*BT.., keys t*BT..;  MODE 1: keys tile*BT.., rows t*BT..
+            const int key0 = MODE == 0 ? t * BT : tile * BT;
+            const int row0 = MODE == 0 ? tile * BT : t * BT;
+            const bool partial = (key0 + BT > prm.Sk) || (prm.causal && key0 + BT - 1 > row0);
+#pragma unroll
+            for (int ch = 0; ch < BT / 32; ++ch) {
+                uint32_t sr[32], dpr[32], pk_p[16], pk_ds[16];
+                tmem_ld_32x32b_x32(tS + ch * 32, sr);
+                tmem_ld_32x32b_x32(tDP + ch * 32, dpr);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    float p[2], ds[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int col = ch * 32 + e + h;
+                        float l2, dl;
+                        bool vis = true;
+                        if constexpr (MODE == 0) {
+                            l2 = my_l2;
+                            dl = my_delta;
+                            if (partial) {
+                                const int key = key0 + col;
+                                vis = key < prm.Sk && (!prm.causal || key <= my_row);
+                            }
+                        } else {
+                            l2 = vl2[col];
+                            dl = vdl[col];
+                            if (partial) vis = my_row < prm.Sk && (!prm.causal || my_row <= row0 + col);
+                        }
+                        const float x = fmaf(__uint_as_float(sr[e + h]), c, -l2);
+                        p[h] = vis ? ex2_approx(x) : 0.f;
+                        ds[h] = p[h] * (__uint_as_float(dpr[e + h]) - dl);
+                    }
+                    pk_p[e / 2] = pack2<DTYPE>(p[0], p[1]);
+                    pk_ds[e / 2] = pack2<DTYPE>(ds[0], ds[1]);
+                }
+                // 16-bit results over the columns already read: chunk ch lands in columns [16 ch, 16 ch + 16)
+                if constexpr (MODE == 0) {
+                    tmem_st_32x32b_x16(tS + ch * 16, pk_ds);
+                } else {
+                    tmem_st_32x32b_x16(tS + ch * 16, pk_p);
+                    tmem_st_32x32b_x16(tDP + ch * 16, pk_ds);
+                }
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(bar(B_PFULL));
+        }
+
+        // ---- epilogue: accumulators -> 16-bit -> swizzled staging tile -> TMA store (rows beyond the tensor clipped) ----
+        if (ok && (ok = mbar_wait(bar(B_ACCFINAL), 0, abort_flag))) {
+            tc_fence_after_sync();
+            constexpr int NACC = MODE == 0 ? 1 : 2;
+#pragma unroll
+            for (int a = 0; a < NACC && ok; ++a) {
+                // MODE 0: dQ (x scale).  MODE 1: accumulator 0 = dV, accumulator 1 = dK (x scale).
+                const float f = (MODE == 0 || a == 1) ? prm.scale : 1.f;
+                const uint32_t tA = tmem + (a == 0 ? C::ACC0_COL : C::ACC1_COL) + lane_off;
+#pragma unroll
+                for (int h = 0; h < D / 64 && ok; ++h) {
+                    uint32_t acc[64];
+                    tmem_ld_32x32b_x32(tA + h * 64, acc);
+                    tmem_ld_32x32b_x32(tA + h * 64 + 32, acc + 32);
+                    tmem_ld_wait();
+                    if (r == 0) tma_store_wait_read<0>();          // the previous store has read the staging tile
+                    if (!(ok = group_sync())) break;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        const uint32_t w0 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 0]) * f, __uint_as_float(acc[g * 8 + 1]) * f);
+                        const uint32_t w1 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 2]) * f, __uint_as_float(acc[g * 8 + 3]) * f);
+                        const uint32_t w2 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 4]) * f, __uint_as_float(acc[g * 8 + 5]) * f);
+                        const uint32_t w3 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 6]) * f, __uint_as_float(acc[g * 8 + 7]) * f);
+                        const uint32_t dst = sOst + r * 128 + ((g ^ (r & 7)) << 4);   // 128-byte swizzle
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+                    }
+                    fence_proxy_async_smem();
+                    if (!(ok = group_sync())) break;
+                    if (r == 0) {
+                        tma_store_3d(a == 0 ? &tmOut0 : &tmOut1, sOst, h * 64, tile * BT, bh_res);
+                        tma_store_commit();
+                    }
+                }
+            }
+        }
+        if (r == 0) tma_store_wait_all<0>();   // the staging tile must outlive its last store
+    }
+
+    // ---- teardown (also reached after a timed-out wait) ----
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) finish_cta(prm.status, *abort_flag != 0, nullptr);
+    if (warp == 4) tmem_dealloc(tmem, C::TMEM_COLS);
+}
+
+}  // namespace attn_grad

@@ -3,7 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C5] [--impl ours|reference]
                     [--kernel-only] [--no-cpu-baseline] [--no-configs] [--sustained-s SEC]
-                    [--sweep grid|configs|shards|decode ...]
+                    [--sweep grid|configs|shards|decode|bwd ...]
 
 A step is one pass of the whole hot path (one attn_fwd call) over one batch of synthetic input of the
 named configuration (default C5, the configuration the target is quoted on).  Rank 0 prints ONE JSON line:
@@ -701,13 +701,40 @@ def sweep_grid(api, args, dev, flush):
                                               "causal" if causal else "none", " | ".join(cells)), flush=True)
 
 
+def sweep_bwd(api, args, dev, flush):
+    """The backward pass (attn_bwd: row sums + dQ pass + dK/dV pass) on the grid of sweep_grid for head dims 64 and
+    128; FLOPs counted as 2.5 x the forward count (five tile products: S, dP, dV, dQ, dK; the kernels execute
+    seven, S and dP once per pass)."""
+    dt = inputs.DTYPE_BF16 if args.dtype == "bf16" else inputs.DTYPE_FP16
+    seqs = [args.seq] if args.seq else [512, 1024, 2048, 4096, 8192, 16384]
+    print("| heads x dim | mask | " + " | ".join("%d: ms (TFLOP/s)" % s for s in seqs) + " |")
+    print("|---|---|" + "---|" * len(seqs))
+    for H, D in ((32, 64), (16, 128)):
+        for causal in (True, False):
+            cells = []
+            for S in seqs:
+                B = max(1, 16384 // S)
+                q, k, v = (t.to(dev) for t in inputs.make_qkv(B, H, S, S, D, dt, 1))
+                dout = inputs.randn16((B, H, S, D), 4, dt).to(dev)
+                scale = D ** -0.5
+                o, lse = api.attn_fwd(q, k, v, scale, causal)
+                dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+                ws = torch.empty(api.attn_bwd_workspace_bytes(B, H, S), dtype=torch.uint8, device=dev)
+                ms = sweep_time(lambda: api.attn_bwd(q, k, v, o, lse, dout, scale, causal, dq=dq, dk=dk, dv=dv, workspace=ws),
+                                flush, args.iters)
+                flops = 2.5 * 4.0 * B * H * S * S * D / (2 if causal else 1)
+                cells.append("%.3f (%.0f)" % (ms, flops / ms / 1e9))
+                del q, k, v, dout, o, lse, dq, dk, dv, ws
+            print("| %d x %d | %s | %s |" % (H, D, "causal" if causal else "none", " | ".join(cells)), flush=True)
+
+
 def run_sweep(args):
     from paper_2506_12355_b200 import api
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
     dev = torch.device("cuda:0")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    {"grid": sweep_grid, "configs": sweep_configs, "shards": sweep_shards, "decode": sweep_decode}[args.sweep](
+    {"grid": sweep_grid, "configs": sweep_configs, "shards": sweep_shards, "decode": sweep_decode, "bwd": sweep_bwd}[args.sweep](
         api, args, dev, flush)
     if api.attn_last_device_status() != 0:
         raise SystemExit("device timeout status")
@@ -726,7 +753,7 @@ def main(argv=None):
     ap.add_argument("--no-configs", action="store_true", help="skip the C1..C5 block")
     ap.add_argument("--sustained-s", type=float, default=2.0, help="length of the back-to-back run (0: skip)")
     ap.add_argument("--kernel-only", action="store_true", help="warm-up and timed steps only (for profiler runs)")
-    ap.add_argument("--sweep", default=None, choices=["grid", "configs", "shards", "decode"])
+    ap.add_argument("--sweep", default=None, choices=["grid", "configs", "shards", "decode", "bwd"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16", "fp8"], help="--sweep grid")
     ap.add_argument("--gqa", type=int, default=0, help="--sweep grid: number of K/V heads (0: same as query heads)")
     ap.add_argument("--iters", type=int, default=15, help="--sweep: timed launches per cell")

@@ -23,9 +23,10 @@
 // Recomputing S and dP in both passes costs 7 tile products instead of 5 but needs no atomics and no
 // cross-CTA reduction, so the results are deterministic.  delta is computed by a small kernel first.
 //
-//   warps 0-3  element-wise group (one thread per tensor-memory lane), then the epilogue
-//   warp  4    MMA issuer
-//   warp  5    TMA producer
+//   warps 0-7  element-wise group, then the epilogue: warp w works on tensor-memory lanes 32 (w % 4) .. + 31
+//              (the lanes a warp may touch) and on columns 64 (w / 4) .. + 63 of the score tile
+//   warp  8    MMA issuer
+//   warp  9    TMA producer
 //
 // Every wait is bounded (see sm100_ptx.cuh); a timed-out wait ends the CTA through the normal exit.
 #pragma once
@@ -47,7 +48,7 @@ struct BwdCfg {
     static constexpr int TILE_BYTES = 2 * TILE_BYTES1 + NSTAGE * 2 * TILE_BYTES1 + OST_BYTES + VEC_BYTES;
     static constexpr int MISC_BYTES = 256;
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
-    static constexpr int THREADS = 192;
+    static constexpr int THREADS = 320;
     static constexpr int S_COL = 0, DP_COL = 128, ACC0_COL = 256, ACC1_COL = 256 + D;
     static constexpr int TMEM_COLS = 512;
     static_assert(D == 64 || D == 128, "head dims 64 and 128");
@@ -121,7 +122,7 @@ __global__ void attn_bwd_delta_kernel(const void* __restrict__ o, const void* __
 // tmR0 / tmR1: maps of the resident tiles (MODE 0: Q, dO; MODE 1: K, V); tmT0 / tmT1: maps of the streamed
 // tiles (MODE 0: K, V; MODE 1: Q, dO); tmOut0 / tmOut1: MODE 0: dQ, unused; MODE 1: dV, dK.
 template <int D, int DTYPE, int MODE>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(320, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant__ CUtensorMap tmR1,
                 const __grid_constant__ CUtensorMap tmT0, const __grid_constant__ CUtensorMap tmT1,
                 const __grid_constant__ CUtensorMap tmOut0, const __grid_constant__ CUtensorMap tmOut1,
@@ -144,7 +145,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 1;
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // ---- this CTA's tile and its steps ----
     // The grid is one-dimensional, tiles of one head next to each other (their streamed tiles are shared in L2).
@@ -196,9 +197,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         *abort_flag = 0;
         mbar_init(bar(B_RFULL), 1);
         mbar_init(bar(B_SFULL), 1);
-        mbar_init(bar(B_PFULL), 128);
+        mbar_init(bar(B_PFULL), 256);
         mbar_init(bar(B_ACCFINAL), 1);
-        mbar_init(bar(B_GSYNC), 128);
+        mbar_init(bar(B_GSYNC), 256);
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(bar(B_TFULL + s), 1);
             mbar_init(bar(B_TEMPTY + s), 1);
@@ -206,11 +207,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         fence_barrier_init();
         fence_proxy_async_smem();
     }
-    if (warp == 4) {
+    if (warp == 8) {
         tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
         tmem_relinquish();
     }
-    if (warp == 5 && elect_one()) {
+    if (warp == 9 && elect_one()) {
         prefetch_tensormap(&tmR0);
         prefetch_tensormap(&tmR1);
         prefetch_tensormap(&tmT0);
@@ -223,7 +224,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 5) {
+    if (warp == 9) {
         // =========================== TMA producer ===========================
         const bool leader = elect_one();
         if (leader) {
@@ -247,7 +248,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 }
             }
         }
-    } else if (warp == 4) {
+    } else if (warp == 8) {
         // =========================== MMA issuer ===========================
         const bool leader = elect_one();
         constexpr uint32_t IDESC_S = make_idesc_f16(BT, BT, DTYPE, 0, 0);    // both operands K-major (contraction over D)
@@ -275,23 +276,27 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             if (!(ok = mbar_wait(bar(B_PFULL), s & 1, abort_flag))) break;
             tc_fence_after_sync();
             if (leader) {
+                // The 16-bit A operands lie over the fp32 tiles they were made from: the values of columns
+                // 64 h .. 64 h + 63 occupy columns 64 h .. 64 h + 31 (each half of the tile is rewritten by the
+                // warps that read it), so contraction step kk (16 values = 8 columns) starts at this column:
+                auto a_col = [](int kk) { return 64 * (kk >> 2) + (kk & 3) * 8; };
                 if constexpr (MODE == 0) {
                     // dQ += dS K_j : dS from tensor memory (over S), K_j MN-major
                     const uint32_t b0 = smem_desc_lo(sT(st, 0), BT * 128);
 #pragma unroll
                     for (int kk = 0; kk < BT / 16; ++kk)
-                        mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::S_COL + kk * 8, b0 + ((kk * 16 * 128) >> 4), DESC_HI,
+                        mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::S_COL + a_col(kk), b0 + ((kk * 16 * 128) >> 4), DESC_HI,
                                         IDESC_ACC, (s > 0 || kk > 0) ? 1u : 0u);
                 } else {
                     // dV += P^T dO_i (P^T over S^T), dK += dS^T Q_i (dS^T over dP^T); dO_i and Q_i MN-major
                     const uint32_t bdo = smem_desc_lo(sT(st, 1), BT * 128), bq = smem_desc_lo(sT(st, 0), BT * 128);
 #pragma unroll
                     for (int kk = 0; kk < BT / 16; ++kk)
-                        mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::S_COL + kk * 8, bdo + ((kk * 16 * 128) >> 4), DESC_HI,
+                        mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::S_COL + a_col(kk), bdo + ((kk * 16 * 128) >> 4), DESC_HI,
                                         IDESC_ACC, (s > 0 || kk > 0) ? 1u : 0u);
 #pragma unroll
                     for (int kk = 0; kk < BT / 16; ++kk)
-                        mma_f16_ts_lohi(tmem + C::ACC1_COL, tmem + C::DP_COL + kk * 8, bq + ((kk * 16 * 128) >> 4), DESC_HI,
+                        mma_f16_ts_lohi(tmem + C::ACC1_COL, tmem + C::DP_COL + a_col(kk), bq + ((kk * 16 * 128) >> 4), DESC_HI,
                                         IDESC_ACC, (s > 0 || kk > 0) ? 1u : 0u);
                 }
                 mma_commit(bar(B_TEMPTY + st));
@@ -300,8 +305,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         }
     } else {
         // =========================== element-wise group + epilogue ===========================
-        const int r = tid;                                   // tensor-memory lane: query row (MODE 0) / key row (MODE 1)
-        const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
+        const int half = warp >> 2;                          // which 64 columns of the score tile
+        const int r = (warp & 3) * 32 + lane;                // tensor-memory lane: query row (MODE 0) / key row (MODE 1)
+        const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + C::S_COL + lane_off, tDP = tmem + C::DP_COL + lane_off;
         const float c = prm.scale_log2;
         const int my_row = tile * BT + r;                    // global query row (MODE 0) or key index (MODE 1)
@@ -314,7 +320,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             }
         }
         bool ok = true;
-        // Barrier among the 128 threads of this group, bounded like every other wait (a plain bar.sync would
+        // Barrier among the 256 threads of this group, bounded like every other wait (a plain bar.sync would
         // wait forever for a thread that has left through the time-out path).
         uint32_t gsync_phase = 0;
         auto group_sync = [&]() -> bool {
@@ -328,17 +334,20 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             float* vl2 = vec + (s & 1) * 2 * BT;
             float* vdl = vl2 + BT;
             if constexpr (MODE == 1) {
-                // L and delta of the streamed Q tile: one row per thread into shared memory
+                // L and delta of the streamed Q tile into shared memory: one value per thread (the threads of
+                // the first column half fetch L, those of the second delta)
                 const int qr = t * BT + r;
-                float l2 = 0.f, dl = 0.f;
+                float val = 0.f;
                 if (qr < prm.Sq) {
                     const int64_t g = static_cast<int64_t>(step_head(s)) * prm.Sq + qr;
-                    const float l = prm.lse[g];
-                    l2 = (l == -INFINITY) ? INFINITY : l * LOG2E;
-                    dl = prm.delta[g];
+                    if (half == 0) {
+                        const float l = prm.lse[g];
+                        val = (l == -INFINITY) ? INFINITY : l * LOG2E;   // a row without visible keys has P = 0
+                    } else {
+                        val = prm.delta[g];
+                    }
                 }
-                vl2[r] = l2;
-                vdl[r] = dl;
+                (half == 0 ? vl2 : vdl)[r] = val;
                 if (!(ok = group_sync())) break;
             }
             if (!(ok = mbar_wait(bar(B_SFULL), s & 1, abort_flag))) break;
@@ -349,7 +358,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             const int row0 = MODE == 0 ? tile * BT : t * BT;
             const bool partial = (key0 + BT > prm.Sk) || (prm.causal && key0 + BT - 1 > row0);
 #pragma unroll
-            for (int ch = 0; ch < BT / 32; ++ch) {
+            for (int cc = 0; cc < 2; ++cc) {
+                const int ch = 2 * half + cc;                // 32-column chunk of the tile
                 uint32_t sr[32], dpr[32], pk_p[16], pk_ds[16];
                 tmem_ld_32x32b_x32(tS + ch * 32, sr);
                 tmem_ld_32x32b_x32(tDP + ch * 32, dpr);
@@ -381,12 +391,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                     pk_p[e / 2] = pack2<DTYPE>(p[0], p[1]);
                     pk_ds[e / 2] = pack2<DTYPE>(ds[0], ds[1]);
                 }
-                // 16-bit results over the columns already read: chunk ch lands in columns [16 ch, 16 ch + 16)
+                // 16-bit results over columns this warp has already read: its two chunks (columns 64 half + 32 cc ..)
+                // land in columns 64 half + 16 cc .. + 15
                 if constexpr (MODE == 0) {
-                    tmem_st_32x32b_x16(tS + ch * 16, pk_ds);
+                    tmem_st_32x32b_x16(tS + 64 * half + 16 * cc, pk_ds);
                 } else {
-                    tmem_st_32x32b_x16(tS + ch * 16, pk_p);
-                    tmem_st_32x32b_x16(tDP + ch * 16, pk_ds);
+                    tmem_st_32x32b_x16(tS + 64 * half + 16 * cc, pk_p);
+                    tmem_st_32x32b_x16(tDP + 64 * half + 16 * cc, pk_ds);
                 }
             }
             tmem_st_wait();
@@ -405,38 +416,38 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 const uint32_t tA = tmem + (a == 0 ? C::ACC0_COL : C::ACC1_COL) + lane_off;
 #pragma unroll
                 for (int h = 0; h < D / 64 && ok; ++h) {
-                    uint32_t acc[64];
-                    tmem_ld_32x32b_x32(tA + h * 64, acc);
-                    tmem_ld_32x32b_x32(tA + h * 64 + 32, acc + 32);
+                    // 64 output columns per round; this thread converts the 32 of its column half
+                    uint32_t acc[32];
+                    tmem_ld_32x32b_x32(tA + h * 64 + 32 * half, acc);
                     tmem_ld_wait();
-                    if (r == 0) tma_store_wait_read<0>();          // the previous store has read the staging tile
+                    if (tid == 0) tma_store_wait_read<0>();        // the previous store has read the staging tile
                     if (!(ok = group_sync())) break;
 #pragma unroll
-                    for (int g = 0; g < 8; ++g) {
+                    for (int g = 0; g < 4; ++g) {
                         const uint32_t w0 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 0]) * f, __uint_as_float(acc[g * 8 + 1]) * f);
                         const uint32_t w1 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 2]) * f, __uint_as_float(acc[g * 8 + 3]) * f);
                         const uint32_t w2 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 4]) * f, __uint_as_float(acc[g * 8 + 5]) * f);
                         const uint32_t w3 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 6]) * f, __uint_as_float(acc[g * 8 + 7]) * f);
-                        const uint32_t dst = sOst + r * 128 + ((g ^ (r & 7)) << 4);   // 128-byte swizzle
+                        const uint32_t dst = sOst + r * 128 + (((4 * half + g) ^ (r & 7)) << 4);   // 128-byte swizzle
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
                     }
                     fence_proxy_async_smem();
                     if (!(ok = group_sync())) break;
-                    if (r == 0) {
+                    if (tid == 0) {
                         tma_store_3d(a == 0 ? &tmOut0 : &tmOut1, sOst, h * 64, tile * BT, bh_res);
                         tma_store_commit();
                     }
                 }
             }
         }
-        if (r == 0) tma_store_wait_all<0>();   // the staging tile must outlive its last store
+        if (tid == 0) tma_store_wait_all<0>();   // the staging tile must outlive its last store
     }
 
     // ---- teardown (also reached after a timed-out wait) ----
     tc_fence_before_sync();
     __syncthreads();
     if (tid == 0) finish_cta(prm.status, *abort_flag != 0, nullptr);
-    if (warp == 4) tmem_dealloc(tmem, C::TMEM_COLS);
+    if (warp == 8) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 }  // namespace attn_grad

@@ -844,10 +844,13 @@ int attn_bwd(const void* q, const void* k, const void* v, const void* o, const f
     prm.n_ktiles = static_cast<int>(n_ktiles);
     prm.status = device_status_ptr();
     if (!prm.status) return ATTN_ERR_CUDA;
-    CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
+    // resident tiles and outputs move in boxes of 128 rows, streamed tiles in boxes of 64 rows
+    CUtensorMap mq, mk, mv, mdo, mq64, mk64, mv64, mdo64, mdq, mdk, mdv;
     if (!make_map(&mq, q, dtype, BH, Sq, D, 128) || !make_map(&mdo, dout, dtype, BH, Sq, D, 128) ||
+        !make_map(&mq64, q, dtype, BH, Sq, D, 64) || !make_map(&mdo64, dout, dtype, BH, Sq, D, 64) ||
         !make_map(&mdq, dq, dtype, BH, Sq, D, 128) || !make_map(&mk, k, dtype, BHkv, Sk, D, 128) ||
-        !make_map(&mv, v, dtype, BHkv, Sk, D, 128) || !make_map(&mdk, dk, dtype, BHkv, Sk, D, 128) ||
+        !make_map(&mv, v, dtype, BHkv, Sk, D, 128) || !make_map(&mk64, k, dtype, BHkv, Sk, D, 64) ||
+        !make_map(&mv64, v, dtype, BHkv, Sk, D, 64) || !make_map(&mdk, dk, dtype, BHkv, Sk, D, 128) ||
         !make_map(&mdv, dv, dtype, BHkv, Sk, D, 128))
         return ATTN_ERR_CUDA;
 #define ATTN_BWD_CASE(DD, TT)                                                                                              \
@@ -864,10 +867,10 @@ int attn_bwd(const void* q, const void* k, const void* v, const void* o, const f
         attn_grad::attn_bwd_delta_kernel<DD, TT><<<static_cast<unsigned>(blocks), 256, 0, st>>>(o, dout, delta, rows);        \
         prm.out0 = dq;                                                                                                     \
         prm.out1 = nullptr;                                                                                                \
-        kq<<<static_cast<unsigned>(n_qtiles * BH), C::THREADS, C::SMEM_BYTES, st>>>(mq, mdo, mk, mv, mdq, mdq, prm);       \
+        kq<<<static_cast<unsigned>(n_qtiles * BH), C::THREADS, C::SMEM_BYTES, st>>>(mq, mdo, mk64, mv64, mdq, mdq, prm);       \
         prm.out0 = dv;                                                                                                     \
         prm.out1 = dk;                                                                                                     \
-        kkv<<<static_cast<unsigned>(n_ktiles * BHkv), C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mq, mdo, mdv, mdk, prm);    \
+        kkv<<<static_cast<unsigned>(n_ktiles * BHkv), C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mq64, mdo64, mdv, mdk, prm);    \
         return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;                                                \
     }
     ATTN_BWD_CASE(64, 0)

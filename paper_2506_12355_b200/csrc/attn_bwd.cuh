@@ -23,6 +23,10 @@
 // Recomputing S and dP in both passes costs 7 tile products instead of 5 but needs no atomics and no
 // cross-CTA reduction, so the results are deterministic.  delta is computed by a small kernel first.
 //
+// The streamed side advances 64 rows per step, and the S / dP tiles of a step (128 lanes x 64 columns each)
+// are double-buffered in tensor memory: while the element-wise warps work on step u, the tensor core
+// already computes S and dP of step u + 1 and the accumulating products of step u - 1.
+//
 //   warps 0-7  element-wise group, then the epilogue: warp w works on tensor-memory lanes 32 (w % 4) .. + 31
 //              (the lanes a warp may touch) and on columns 64 (w / 4) .. + 63 of the score tile
 //   warp  8    MMA issuer
@@ -39,17 +43,22 @@ using attn_tc::finish_cta;
 
 template <int D>
 struct BwdCfg {
-    static constexpr int BT = 128;                          // rows of every tile (queries or keys)
+    static constexpr int BT = 128;                          // rows of the resident tiles = tensor-memory lanes
+    static constexpr int BS = 64;                           // rows of the streamed tiles = columns of one step
     static constexpr int NBOX = D / 64;                     // 128-byte wide TMA boxes per tile row
-    static constexpr int TILE_BYTES1 = BT * D * 2;          // one operand tile
-    static constexpr int NSTAGE = D == 128 ? 2 : 4;         // ring stages, each holds the two streamed tiles
+    static constexpr int RES_BYTES = BT * D * 2;            // one resident tile
+    static constexpr int STR_BYTES = BS * D * 2;            // one streamed tile
+    static constexpr int NSTAGE = D == 128 ? 4 : 6;           // ring stages, each holds the two streamed tiles
     static constexpr int OST_BYTES = BT * 128;              // epilogue staging: 128 rows x 64 columns
-    static constexpr int VEC_BYTES = 2 * 2 * BT * 4;        // MODE 1: L and delta of the streamed Q tile, two buffers
-    static constexpr int TILE_BYTES = 2 * TILE_BYTES1 + NSTAGE * 2 * TILE_BYTES1 + OST_BYTES + VEC_BYTES;
+    static constexpr int VEC_BYTES = 2 * 2 * BS * 4;        // MODE 1: L and delta of the streamed rows, two buffers
+    static constexpr int TILE_BYTES = 2 * RES_BYTES + NSTAGE * 2 * STR_BYTES + OST_BYTES + VEC_BYTES;
     static constexpr int MISC_BYTES = 256;
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
     static constexpr int THREADS = 320;
-    static constexpr int S_COL = 0, DP_COL = 128, ACC0_COL = 256, ACC1_COL = 256 + D;
+    // tensor memory: step buffer b holds S in columns 128 b .. + 63 and dP in 128 b + 64 .. + 63
+    __host__ __device__ static constexpr int s_col(int b) { return 128 * b; }
+    __host__ __device__ static constexpr int dp_col(int b) { return 128 * b + 64; }
+    static constexpr int ACC0_COL = 256, ACC1_COL = 256 + D;
     static constexpr int TMEM_COLS = 512;
     static_assert(D == 64 || D == 128, "head dims 64 and 128");
 };
@@ -63,7 +72,7 @@ struct BwdParams {
     float scale, scale_log2;
     int causal;
     int H, Hkv;
-    int n_qtiles, n_ktiles;
+    int n_qtiles, n_ktiles; // 128-row tiles of the query and of the key axis
     int* status;
 };
 
@@ -119,8 +128,9 @@ __global__ void attn_bwd_delta_kernel(const void* __restrict__ o, const void* __
     }
 }
 
-// tmR0 / tmR1: maps of the resident tiles (MODE 0: Q, dO; MODE 1: K, V); tmT0 / tmT1: maps of the streamed
-// tiles (MODE 0: K, V; MODE 1: Q, dO); tmOut0 / tmOut1: MODE 0: dQ, unused; MODE 1: dV, dK.
+// tmR0 / tmR1: maps of the resident tiles, boxes of 128 rows (MODE 0: Q, dO; MODE 1: K, V); tmT0 / tmT1: maps of
+// the streamed tiles, boxes of 64 rows (MODE 0: K, V; MODE 1: Q, dO); tmOut0 / tmOut1: MODE 0: dQ, unused;
+// MODE 1: dV, dK (boxes of 128 rows).
 template <int D, int DTYPE, int MODE>
 __global__ void __launch_bounds__(320, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant__ CUtensorMap tmR1,
@@ -128,19 +138,29 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 const __grid_constant__ CUtensorMap tmOut0, const __grid_constant__ CUtensorMap tmOut1,
                 const BwdParams prm) {
     using C = BwdCfg<D>;
-    constexpr int BT = C::BT, NBOX = C::NBOX, NSTAGE = C::NSTAGE, T1B = C::TILE_BYTES1;
+    constexpr int BT = C::BT, BS = C::BS, NBOX = C::NBOX, NSTAGE = C::NSTAGE;
     constexpr float LOG2E = 1.4426950408889634f;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    auto sR = [&](int w) { return smem_base + w * T1B; };                              // resident tile w (0 / 1)
-    auto sT = [&](int stage, int w) { return smem_base + (2 + 2 * stage + w) * T1B; };   // streamed tile w of a stage
-    const uint32_t sOst = smem_base + (2 + 2 * NSTAGE) * T1B;
-    float* vec = reinterpret_cast<float*>(smem_gen + (2 + 2 * NSTAGE) * T1B + C::OST_BYTES);   // [2 buffers][L2 | delta][BT]
+    auto sR = [&](int w) { return smem_base + w * C::RES_BYTES; };                                          // resident tile w
+    auto sT = [&](int stage, int w) { return smem_base + 2 * C::RES_BYTES + (2 * stage + w) * C::STR_BYTES; };  // streamed tile w
+    constexpr int OST_OFF = 2 * C::RES_BYTES + 2 * NSTAGE * C::STR_BYTES;
+    const uint32_t sOst = smem_base + OST_OFF;
+    float* vec = reinterpret_cast<float*>(smem_gen + OST_OFF + C::OST_BYTES);   // [2 buffers][L * log2 e | delta][BS]
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
     const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
-    enum { B_RFULL = 0, B_SFULL = 1, B_PFULL = 2, B_ACCFINAL = 3, B_GSYNC = 4, B_TFULL = 5, B_TEMPTY = 5 + NSTAGE, B_COUNT = 5 + 2 * NSTAGE };
+    enum {
+        B_RFULL = 0,      // resident tiles loaded (TMA bytes)
+        B_SFULL = 1,      // [2] S and dP of a step are in buffer b (MMA commit)
+        B_PFULL = 3,      // [2] the 16-bit operands of a step are in buffer b (256 element-wise threads)
+        B_ACCFINAL = 5,   // the last accumulating product has finished
+        B_GSYNC = 6,      // barrier among the element-wise threads
+        B_TFULL = 7,      // [NSTAGE] streamed tiles loaded
+        B_TEMPTY = 7 + NSTAGE,
+        B_COUNT = 7 + 2 * NSTAGE
+    };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 1;
@@ -149,36 +169,36 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
 
     // ---- this CTA's tile and its steps ----
     // The grid is one-dimensional, tiles of one head next to each other (their streamed tiles are shared in L2).
-    // MODE 0: Q tile (causal: longest first) of a (batch, query head); steps = K/V tiles.
-    // MODE 1: K/V tile (the first has the most steps) of a (batch, K/V head);
-    //         steps = (query head of the group, Q tile) pairs.
+    // MODE 0: 128-row Q tile (causal: longest first) of a (batch, query head); steps = 64-key K/V tiles.
+    // MODE 1: 128-key K/V tile (the first has the most steps) of a (batch, K/V head);
+    //         steps = (query head of the group, 64-row Q tile) pairs.
     const int group = prm.H / prm.Hkv;
     const int tiles_per_head = MODE == 0 ? prm.n_qtiles : prm.n_ktiles;
     const int bid_tile = static_cast<int>(blockIdx.x % static_cast<unsigned>(tiles_per_head));
-    int tile, bh_res, step_lo, step_hi, n_steps;
-    bh_res = static_cast<int>(blockIdx.x / static_cast<unsigned>(tiles_per_head));
+    const int bh_res = static_cast<int>(blockIdx.x / static_cast<unsigned>(tiles_per_head));
+    int tile, sub_lo, sub_hi, n_steps;
     if constexpr (MODE == 0) {
         tile = prm.causal ? prm.n_qtiles - 1 - bid_tile : bid_tile;
         const int last_key = attn_tc::last_visible_key(tile * BT + BT - 1, prm.Sk, prm.causal, 0);
-        step_lo = 0;
-        step_hi = last_key < 0 ? 0 : last_key / BT + 1;
-        n_steps = step_hi - step_lo;
+        sub_lo = 0;
+        sub_hi = last_key < 0 ? 0 : last_key / BS + 1;
+        n_steps = sub_hi;
     } else {
         tile = bid_tile;
-        step_lo = prm.causal ? tile : 0;     // first Q tile with a row that sees key tile * BT
-        step_hi = prm.n_qtiles;
-        if (step_lo > step_hi) step_lo = step_hi;
-        n_steps = (step_hi - step_lo) * group;
+        sub_lo = prm.causal ? (tile * BT) / BS : 0;     // first 64-row Q tile with a row that sees key tile * BT
+        sub_hi = (prm.Sq + BS - 1) / BS;
+        if (sub_lo > sub_hi) sub_lo = sub_hi;
+        n_steps = (sub_hi - sub_lo) * group;
     }
     const int kv_bh_of_q = (bh_res / prm.H) * prm.Hkv + (bh_res % prm.H) / group;   // MODE 0: K/V head of this query head
-    // streamed tile of step s: (head index in its tensor, tile index)
-    auto step_head = [&](int s) {
+    // streamed tile of step u: (head index in its tensor, index of the 64-row tile)
+    auto step_head = [&](int u) {
         if constexpr (MODE == 0) return kv_bh_of_q;
-        else return (bh_res / prm.Hkv) * prm.H + (bh_res % prm.Hkv) * group + s / (step_hi - step_lo);
+        else return (bh_res / prm.Hkv) * prm.H + (bh_res % prm.Hkv) * group + u / (sub_hi - sub_lo);
     };
-    auto step_tile = [&](int s) {
-        if constexpr (MODE == 0) return step_lo + s;
-        else return step_lo + s % (step_hi - step_lo);
+    auto step_sub = [&](int u) {
+        if constexpr (MODE == 0) return u;
+        else return sub_lo + u % (sub_hi - sub_lo);
     };
 
     if (n_steps == 0) {
@@ -196,8 +216,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
     if (tid == 0) {
         *abort_flag = 0;
         mbar_init(bar(B_RFULL), 1);
-        mbar_init(bar(B_SFULL), 1);
-        mbar_init(bar(B_PFULL), 256);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(B_SFULL + b), 1);
+            mbar_init(bar(B_PFULL + b), 256);
+        }
         mbar_init(bar(B_ACCFINAL), 1);
         mbar_init(bar(B_GSYNC), 256);
         for (int s = 0; s < NSTAGE; ++s) {
@@ -228,87 +250,94 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         // =========================== TMA producer ===========================
         const bool leader = elect_one();
         if (leader) {
-            mbar_arrive_expect_tx(bar(B_RFULL), 2 * T1B);
+            mbar_arrive_expect_tx(bar(B_RFULL), 2 * C::RES_BYTES);
 #pragma unroll
             for (int bx = 0; bx < NBOX; ++bx) {
                 tma_load_3d(sR(0) + bx * BT * 128, &tmR0, bar(B_RFULL), bx * 64, tile * BT, bh_res);
                 tma_load_3d(sR(1) + bx * BT * 128, &tmR1, bar(B_RFULL), bx * 64, tile * BT, bh_res);
             }
         }
-        for (int s = 0; s < n_steps; ++s) {
-            const int st = s % NSTAGE;
-            if (!mbar_wait(bar(B_TEMPTY + st), ((s / NSTAGE) & 1) ^ 1, abort_flag)) break;
+        for (int u = 0; u < n_steps; ++u) {
+            const int st = u % NSTAGE;
+            if (!mbar_wait(bar(B_TEMPTY + st), ((u / NSTAGE) & 1) ^ 1, abort_flag)) break;
             if (leader) {
-                mbar_arrive_expect_tx(bar(B_TFULL + st), 2 * T1B);
-                const int head = step_head(s), row0 = step_tile(s) * BT;
+                mbar_arrive_expect_tx(bar(B_TFULL + st), 2 * C::STR_BYTES);
+                const int head = step_head(u), row0 = step_sub(u) * BS;
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx) {
-                    tma_load_3d(sT(st, 0) + bx * BT * 128, &tmT0, bar(B_TFULL + st), bx * 64, row0, head);
-                    tma_load_3d(sT(st, 1) + bx * BT * 128, &tmT1, bar(B_TFULL + st), bx * 64, row0, head);
+                    tma_load_3d(sT(st, 0) + bx * BS * 128, &tmT0, bar(B_TFULL + st), bx * 64, row0, head);
+                    tma_load_3d(sT(st, 1) + bx * BS * 128, &tmT1, bar(B_TFULL + st), bx * 64, row0, head);
                 }
             }
         }
     } else if (warp == 8) {
         // =========================== MMA issuer ===========================
         const bool leader = elect_one();
-        constexpr uint32_t IDESC_S = make_idesc_f16(BT, BT, DTYPE, 0, 0);    // both operands K-major (contraction over D)
+        constexpr uint32_t IDESC_S = make_idesc_f16(BT, BS, DTYPE, 0, 0);    // both operands K-major (contraction over D)
         constexpr uint32_t IDESC_ACC = make_idesc_f16(BT, D, DTYPE, 0, 1);   // A from tensor memory, B MN-major (N = D)
         constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
         const uint32_t r_lo[2] = {smem_desc_lo(sR(0), 16), smem_desc_lo(sR(1), 16)};
+        // The 16-bit A operands lie over the fp32 tiles they were made from: the values of columns 32 h .. 32 h + 31
+        // of a step buffer occupy its columns 32 h .. 32 h + 15 (each half is rewritten by the warps that read it),
+        // so contraction step kk (16 values = 8 columns) starts at this column:
+        auto a_col = [](int kk) { return 32 * (kk >> 1) + (kk & 1) * 8; };
         bool ok = mbar_wait(bar(B_RFULL), 0, abort_flag);
-        for (int s = 0; s < n_steps && ok; ++s) {
-            const int st = s % NSTAGE;
-            if (!(ok = mbar_wait(bar(B_TFULL + st), (s / NSTAGE) & 1, abort_flag))) break;
-            tc_fence_after_sync();
-            if (leader) {
-                // S (or S^T) = R0 T0^T, dP (or dP^T) = R1 T1^T : D / 16 instructions each
+        // software pipeline: iteration u issues S, dP of step u, then the accumulating products of step u - 1
+        for (int u = 0; u <= n_steps && ok; ++u) {
+            if (u < n_steps) {
+                const int st = u % NSTAGE, b = u & 1;
+                if (!(ok = mbar_wait(bar(B_TFULL + st), (u / NSTAGE) & 1, abort_flag))) break;
+                tc_fence_after_sync();
+                if (leader) {
+                    // S (or S^T) = R0 T0^T, dP (or dP^T) = R1 T1^T : D / 16 instructions each (M 128, N 64, K 16).
+                    // Buffer b was last read by the accumulating products of step u - 2, issued before these.
 #pragma unroll
-                for (int w = 0; w < 2; ++w) {
-                    const uint32_t b0 = smem_desc_lo(sT(st, w), 16);
+                    for (int w = 0; w < 2; ++w) {
+                        const uint32_t b0 = smem_desc_lo(sT(st, w), 16);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = ((kk >> 2) * BT * 128 + (kk & 3) * 32) >> 4;
-                        mma_f16_ss_lohi(tmem + (w == 0 ? C::S_COL : C::DP_COL), r_lo[w] + off, b0 + off, DESC_HI, IDESC_S, kk > 0);
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint32_t offa = ((kk >> 2) * BT * 128 + (kk & 3) * 32) >> 4;
+                            const uint32_t offb = ((kk >> 2) * BS * 128 + (kk & 3) * 32) >> 4;
+                            mma_f16_ss_lohi(tmem + (w == 0 ? C::s_col(b) : C::dp_col(b)), r_lo[w] + offa, b0 + offb, DESC_HI, IDESC_S, kk > 0);
+                        }
                     }
+                    mma_commit(bar(B_SFULL + b));
                 }
-                mma_commit(bar(B_SFULL));
             }
-            if (!(ok = mbar_wait(bar(B_PFULL), s & 1, abort_flag))) break;
-            tc_fence_after_sync();
-            if (leader) {
-                // The 16-bit A operands lie over the fp32 tiles they were made from: the values of columns
-                // 64 h .. 64 h + 63 occupy columns 64 h .. 64 h + 31 (each half of the tile is rewritten by the
-                // warps that read it), so contraction step kk (16 values = 8 columns) starts at this column:
-                auto a_col = [](int kk) { return 64 * (kk >> 2) + (kk & 3) * 8; };
-                if constexpr (MODE == 0) {
-                    // dQ += dS K_j : dS from tensor memory (over S), K_j MN-major
-                    const uint32_t b0 = smem_desc_lo(sT(st, 0), BT * 128);
+            if (u >= 1) {
+                const int v = u - 1, st = v % NSTAGE, b = v & 1;
+                if (!(ok = mbar_wait(bar(B_PFULL + b), (v >> 1) & 1, abort_flag))) break;
+                tc_fence_after_sync();
+                if (leader) {
+                    if constexpr (MODE == 0) {
+                        // dQ += dS K_j : dS from tensor memory (over S), K_j MN-major
+                        const uint32_t b0 = smem_desc_lo(sT(st, 0), BS * 128);
 #pragma unroll
-                    for (int kk = 0; kk < BT / 16; ++kk)
-                        mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::S_COL + a_col(kk), b0 + ((kk * 16 * 128) >> 4), DESC_HI,
-                                        IDESC_ACC, (s > 0 || kk > 0) ? 1u : 0u);
-                } else {
-                    // dV += P^T dO_i (P^T over S^T), dK += dS^T Q_i (dS^T over dP^T); dO_i and Q_i MN-major
-                    const uint32_t bdo = smem_desc_lo(sT(st, 1), BT * 128), bq = smem_desc_lo(sT(st, 0), BT * 128);
+                        for (int kk = 0; kk < BS / 16; ++kk)
+                            mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::s_col(b) + a_col(kk), b0 + ((kk * 16 * 128) >> 4), DESC_HI,
+                                            IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
+                    } else {
+                        // dV += P^T dO_i (P^T over S^T), dK += dS^T Q_i (dS^T over dP^T); dO_i and Q_i MN-major
+                        const uint32_t bdo = smem_desc_lo(sT(st, 1), BS * 128), bq = smem_desc_lo(sT(st, 0), BS * 128);
 #pragma unroll
-                    for (int kk = 0; kk < BT / 16; ++kk)
-                        mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::S_COL + a_col(kk), bdo + ((kk * 16 * 128) >> 4), DESC_HI,
-                                        IDESC_ACC, (s > 0 || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < BS / 16; ++kk)
+                            mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::s_col(b) + a_col(kk), bdo + ((kk * 16 * 128) >> 4), DESC_HI,
+                                            IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
 #pragma unroll
-                    for (int kk = 0; kk < BT / 16; ++kk)
-                        mma_f16_ts_lohi(tmem + C::ACC1_COL, tmem + C::DP_COL + a_col(kk), bq + ((kk * 16 * 128) >> 4), DESC_HI,
-                                        IDESC_ACC, (s > 0 || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < BS / 16; ++kk)
+                            mma_f16_ts_lohi(tmem + C::ACC1_COL, tmem + C::dp_col(b) + a_col(kk), bq + ((kk * 16 * 128) >> 4), DESC_HI,
+                                            IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    mma_commit(bar(B_TEMPTY + st));
+                    if (v + 1 == n_steps) mma_commit(bar(B_ACCFINAL));
                 }
-                mma_commit(bar(B_TEMPTY + st));
-                if (s + 1 == n_steps) mma_commit(bar(B_ACCFINAL));
             }
         }
     } else {
         // =========================== element-wise group + epilogue ===========================
-        const int half = warp >> 2;                          // which 64 columns of the score tile
+        const int half = warp >> 2;                          // which 32 columns of a step buffer
         const int r = (warp & 3) * 32 + lane;                // tensor-memory lane: query row (MODE 0) / key row (MODE 1)
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + C::S_COL + lane_off, tDP = tmem + C::DP_COL + lane_off;
         const float c = prm.scale_log2;
         const int my_row = tile * BT + r;                    // global query row (MODE 0) or key index (MODE 1)
         float my_l2 = 0.f, my_delta = 0.f;                   // MODE 0: this row's L * log2(e) and delta
@@ -329,47 +358,47 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             ++gsync_phase;
             return done;
         };
-        for (int s = 0; s < n_steps && ok; ++s) {
-            const int t = step_tile(s);
-            float* vl2 = vec + (s & 1) * 2 * BT;
-            float* vdl = vl2 + BT;
+        for (int u = 0; u < n_steps && ok; ++u) {
+            const int t = step_sub(u), b = u & 1;
+            const uint32_t tS = tmem + C::s_col(b) + lane_off, tDP = tmem + C::dp_col(b) + lane_off;
+            float* vl2 = vec + b * 2 * BS;
+            float* vdl = vl2 + BS;
             if constexpr (MODE == 1) {
-                // L and delta of the streamed Q tile into shared memory: one value per thread (the threads of
-                // the first column half fetch L, those of the second delta)
-                const int qr = t * BT + r;
-                float val = 0.f;
-                if (qr < prm.Sq) {
-                    const int64_t g = static_cast<int64_t>(step_head(s)) * prm.Sq + qr;
-                    if (half == 0) {
-                        const float l = prm.lse[g];
-                        val = (l == -INFINITY) ? INFINITY : l * LOG2E;   // a row without visible keys has P = 0
-                    } else {
-                        val = prm.delta[g];
+                // L and delta of the 64 streamed query rows into shared memory: threads 0..63 fetch L, 64..127 delta
+                if (tid < 2 * BS) {
+                    const int qr = t * BS + (tid & (BS - 1));
+                    float val = 0.f;
+                    if (qr < prm.Sq) {
+                        const int64_t g = static_cast<int64_t>(step_head(u)) * prm.Sq + qr;
+                        if (tid < BS) {
+                            const float l = prm.lse[g];
+                            val = (l == -INFINITY) ? INFINITY : l * LOG2E;   // a row without visible keys has P = 0
+                        } else {
+                            val = prm.delta[g];
+                        }
                     }
+                    (tid < BS ? vl2 : vdl)[tid & (BS - 1)] = val;
                 }
-                (half == 0 ? vl2 : vdl)[r] = val;
                 if (!(ok = group_sync())) break;
             }
-            if (!(ok = mbar_wait(bar(B_SFULL), s & 1, abort_flag))) break;
+            if (!(ok = mbar_wait(bar(B_SFULL + b), (u >> 1) & 1, abort_flag))) break;
             tc_fence_after_sync();
-            // does any element of this tile need the mask?  (uniform over the CTA)
-            //   MODE 0: rows tile*BT.., keys t*BT..;  MODE 1: keys tile*BT.., rows t*BT..
-            const int key0 = MODE == 0 ? t * BT : tile * BT;
-            const int row0 = MODE == 0 ? tile * BT : t * BT;
-            const bool partial = (key0 + BT > prm.Sk) || (prm.causal && key0 + BT - 1 > row0);
-#pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-                const int ch = 2 * half + cc;                // 32-column chunk of the tile
+            // does any element of this step need the mask?  (uniform over the CTA)
+            //   MODE 0: rows tile*128 .. +127, keys t*64 .. +63;  MODE 1: keys tile*128 .. +127, rows t*64 .. +63
+            const int key0 = MODE == 0 ? t * BS : tile * BT, nkeys = MODE == 0 ? BS : BT;
+            const int row0 = MODE == 0 ? tile * BT : t * BS;
+            const bool partial = (key0 + nkeys > prm.Sk) || (prm.causal && key0 + nkeys - 1 > row0);
+            {
                 uint32_t sr[32], dpr[32], pk_p[16], pk_ds[16];
-                tmem_ld_32x32b_x32(tS + ch * 32, sr);
-                tmem_ld_32x32b_x32(tDP + ch * 32, dpr);
+                tmem_ld_32x32b_x32(tS + 32 * half, sr);
+                tmem_ld_32x32b_x32(tDP + 32 * half, dpr);
                 tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
                     float p[2], ds[2];
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const int col = ch * 32 + e + h;
+                        const int col = 32 * half + e + h;
                         float l2, dl;
                         bool vis = true;
                         if constexpr (MODE == 0) {
@@ -391,18 +420,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                     pk_p[e / 2] = pack2<DTYPE>(p[0], p[1]);
                     pk_ds[e / 2] = pack2<DTYPE>(ds[0], ds[1]);
                 }
-                // 16-bit results over columns this warp has already read: its two chunks (columns 64 half + 32 cc ..)
-                // land in columns 64 half + 16 cc .. + 15
+                // 16-bit results over the columns this thread has just read: 32 values -> 16 columns
                 if constexpr (MODE == 0) {
-                    tmem_st_32x32b_x16(tS + 64 * half + 16 * cc, pk_ds);
+                    tmem_st_32x32b_x16(tS + 32 * half, pk_ds);
                 } else {
-                    tmem_st_32x32b_x16(tS + 64 * half + 16 * cc, pk_p);
-                    tmem_st_32x32b_x16(tDP + 64 * half + 16 * cc, pk_ds);
+                    tmem_st_32x32b_x16(tS + 32 * half, pk_p);
+                    tmem_st_32x32b_x16(tDP + 32 * half, pk_ds);
                 }
             }
             tmem_st_wait();
             tc_fence_before_sync();
-            mbar_arrive(bar(B_PFULL));
+            mbar_arrive(bar(B_PFULL + b));
         }
 
         // ---- epilogue: accumulators -> 16-bit -> swizzled staging tile -> TMA store (rows beyond the tensor clipped) ----

@@ -27,8 +27,8 @@
 // are double-buffered in tensor memory: while the element-wise warps work on step u, the tensor core
 // already computes S and dP of step u + 1 and the accumulating products of step u - 1.
 //
-//   warps 0-7  element-wise group, then the epilogue: warp w works on tensor-memory lanes 32 (w % 4) .. + 31
-//              (the lanes a warp may touch) and on columns 64 (w / 4) .. + 63 of the score tile
+//   warps 0-3  element-wise group of the even steps (one thread per tensor-memory lane), then the epilogue
+//   warps 4-7  element-wise group of the odd steps
 //   warp  8    MMA issuer
 //   warp  9    TMA producer
 //
@@ -50,7 +50,7 @@ struct BwdCfg {
     static constexpr int STR_BYTES = BS * D * 2;            // one streamed tile
     static constexpr int NSTAGE = D == 128 ? 4 : 6;           // ring stages, each holds the two streamed tiles
     static constexpr int OST_BYTES = BT * 128;              // epilogue staging: 128 rows x 64 columns
-    static constexpr int VEC_BYTES = 2 * 2 * BS * 4;        // MODE 1: L and delta of the streamed rows, two buffers
+    static constexpr int VEC_BYTES = 2 * 2 * 2 * BS * 4;    // MODE 1: L and delta of the streamed rows: two groups x two buffers
     static constexpr int TILE_BYTES = 2 * RES_BYTES + NSTAGE * 2 * STR_BYTES + OST_BYTES + VEC_BYTES;
     static constexpr int MISC_BYTES = 256;
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
@@ -148,18 +148,19 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
     auto sT = [&](int stage, int w) { return smem_base + 2 * C::RES_BYTES + (2 * stage + w) * C::STR_BYTES; };  // streamed tile w
     constexpr int OST_OFF = 2 * C::RES_BYTES + 2 * NSTAGE * C::STR_BYTES;
     const uint32_t sOst = smem_base + OST_OFF;
-    float* vec = reinterpret_cast<float*>(smem_gen + OST_OFF + C::OST_BYTES);   // [2 buffers][L * log2 e | delta][BS]
+    float* vec = reinterpret_cast<float*>(smem_gen + OST_OFF + C::OST_BYTES);   // [group][buffer][-L log2 e | -delta][BS]
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
     const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
     enum {
         B_RFULL = 0,      // resident tiles loaded (TMA bytes)
         B_SFULL = 1,      // [2] S and dP of a step are in buffer b (MMA commit)
-        B_PFULL = 3,      // [2] the 16-bit operands of a step are in buffer b (256 element-wise threads)
+        B_PFULL = 3,      // [2] the 16-bit operands of a step are in buffer b (the 128 threads of group b)
         B_ACCFINAL = 5,   // the last accumulating product has finished
-        B_GSYNC = 6,      // barrier among the element-wise threads
-        B_TFULL = 7,      // [NSTAGE] streamed tiles loaded
-        B_TEMPTY = 7 + NSTAGE,
-        B_COUNT = 7 + 2 * NSTAGE
+        B_GSYNC = 6,      // [2] barrier among the 128 threads of a group
+        B_ESYNC = 8,      // barrier among all 256 element-wise threads (epilogue)
+        B_TFULL = 9,      // [NSTAGE] streamed tiles loaded
+        B_TEMPTY = 9 + NSTAGE,
+        B_COUNT = 9 + 2 * NSTAGE
     };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
@@ -218,10 +219,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         mbar_init(bar(B_RFULL), 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(B_SFULL + b), 1);
-            mbar_init(bar(B_PFULL + b), 256);
+            mbar_init(bar(B_PFULL + b), 128);
+            mbar_init(bar(B_GSYNC + b), 128);
         }
         mbar_init(bar(B_ACCFINAL), 1);
-        mbar_init(bar(B_GSYNC), 256);
+        mbar_init(bar(B_ESYNC), 256);
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(bar(B_TFULL + s), 1);
             mbar_init(bar(B_TEMPTY + s), 1);
@@ -277,10 +279,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         constexpr uint32_t IDESC_ACC = make_idesc_f16(BT, D, DTYPE, 0, 1);   // A from tensor memory, B MN-major (N = D)
         constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
         const uint32_t r_lo[2] = {smem_desc_lo(sR(0), 16), smem_desc_lo(sR(1), 16)};
-        // The 16-bit A operands lie over the fp32 tiles they were made from: the values of columns 32 h .. 32 h + 31
-        // of a step buffer occupy its columns 32 h .. 32 h + 15 (each half is rewritten by the warps that read it),
-        // so contraction step kk (16 values = 8 columns) starts at this column:
-        auto a_col = [](int kk) { return 32 * (kk >> 1) + (kk & 1) * 8; };
+        // The 16-bit A operands lie over the fp32 tiles they were made from: the 64 values of a step occupy the
+        // first 32 columns of its S (or dP) columns, so contraction step kk (16 values) starts at column 8 kk.
+        auto a_col = [](int kk) { return kk * 8; };
         bool ok = mbar_wait(bar(B_RFULL), 0, abort_flag);
         // software pipeline: iteration u issues S, dP of step u, then the accumulating products of step u - 1
         for (int u = 0; u <= n_steps && ok; ++u) {
@@ -334,103 +335,123 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             }
         }
     } else {
-        // =========================== element-wise group + epilogue ===========================
-        const int half = warp >> 2;                          // which 32 columns of a step buffer
+        // =========================== element-wise groups + epilogue ===========================
+        // Group g (warps 4g .. 4g+3) takes the steps u = g, g + 2, ...: always step buffer g.  While one group
+        // waits for its tile or for tensor memory, the other computes.
+        const int grp = warp >> 2;
+        const int half = grp;                                // epilogue: which 32 of every 64 output columns
         const int r = (warp & 3) * 32 + lane;                // tensor-memory lane: query row (MODE 0) / key row (MODE 1)
+        const int gt = tid & 127;                            // thread index inside the group
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + C::s_col(grp) + lane_off, tDP = tmem + C::dp_col(grp) + lane_off;
         const float c = prm.scale_log2;
+        const uint64_t c2 = pack_f32x2(c, c);
         const int my_row = tile * BT + r;                    // global query row (MODE 0) or key index (MODE 1)
-        float my_l2 = 0.f, my_delta = 0.f;                   // MODE 0: this row's L * log2(e) and delta
+        float my_nl2 = 0.f, my_ndelta = 0.f;                 // MODE 0: minus this row's L * log2(e), minus its delta
         if constexpr (MODE == 0) {
             if (my_row < prm.Sq) {
                 const float l = prm.lse[static_cast<int64_t>(bh_res) * prm.Sq + my_row];
-                my_l2 = (l == -INFINITY) ? INFINITY : l * LOG2E;   // a row without visible keys has P = 0
-                my_delta = prm.delta[static_cast<int64_t>(bh_res) * prm.Sq + my_row];
+                my_nl2 = (l == -INFINITY) ? -INFINITY : -l * LOG2E;   // a row without visible keys has P = 0
+                my_ndelta = -prm.delta[static_cast<int64_t>(bh_res) * prm.Sq + my_row];
             }
         }
         bool ok = true;
-        // Barrier among the 256 threads of this group, bounded like every other wait (a plain bar.sync would
-        // wait forever for a thread that has left through the time-out path).
-        uint32_t gsync_phase = 0;
+        // Barriers among element-wise threads are mbarriers with the same bounded wait as everything else (a plain
+        // bar.sync would wait forever for a thread that has left through the time-out path).
+        uint32_t gsync_phase = 0, esync_phase = 0;
         auto group_sync = [&]() -> bool {
-            mbar_arrive(bar(B_GSYNC));
-            const bool done = mbar_wait(bar(B_GSYNC), gsync_phase & 1, abort_flag);
+            mbar_arrive(bar(B_GSYNC + grp));
+            const bool done = mbar_wait(bar(B_GSYNC + grp), gsync_phase & 1, abort_flag);
             ++gsync_phase;
             return done;
         };
-        for (int u = 0; u < n_steps && ok; ++u) {
-            const int t = step_sub(u), b = u & 1;
-            const uint32_t tS = tmem + C::s_col(b) + lane_off, tDP = tmem + C::dp_col(b) + lane_off;
-            float* vl2 = vec + b * 2 * BS;
-            float* vdl = vl2 + BS;
+        auto all_sync = [&]() -> bool {
+            mbar_arrive(bar(B_ESYNC));
+            const bool done = mbar_wait(bar(B_ESYNC), esync_phase & 1, abort_flag);
+            ++esync_phase;
+            return done;
+        };
+        for (int u = grp; u < n_steps && ok; u += 2) {
+            const int t = step_sub(u);
+            // MODE 1: -L * log2(e) and -delta of the step's 64 query rows, in one of the group's two buffers
+            float* vnl2 = vec + (grp * 2 + ((u >> 1) & 1)) * 2 * BS;
+            float* vndl = vnl2 + BS;
             if constexpr (MODE == 1) {
-                // L and delta of the 64 streamed query rows into shared memory: threads 0..63 fetch L, 64..127 delta
-                if (tid < 2 * BS) {
-                    const int qr = t * BS + (tid & (BS - 1));
-                    float val = 0.f;
-                    if (qr < prm.Sq) {
-                        const int64_t g = static_cast<int64_t>(step_head(u)) * prm.Sq + qr;
-                        if (tid < BS) {
-                            const float l = prm.lse[g];
-                            val = (l == -INFINITY) ? INFINITY : l * LOG2E;   // a row without visible keys has P = 0
-                        } else {
-                            val = prm.delta[g];
-                        }
+                // this group's 128 threads fetch one value each: threads 0..63 L, 64..127 delta.  A thread that
+                // writes buffer x for step u has passed the barrier of step u - 2, which every thread of the group
+                // reaches only after its reads of buffer x for step u - 4.
+                const int qr = t * BS + (gt & (BS - 1));
+                float val = 0.f;
+                if (qr < prm.Sq) {
+                    const int64_t g = static_cast<int64_t>(step_head(u)) * prm.Sq + qr;
+                    if (gt < BS) {
+                        const float l = prm.lse[g];
+                        val = (l == -INFINITY) ? -INFINITY : -l * LOG2E;
+                    } else {
+                        val = -prm.delta[g];
                     }
-                    (tid < BS ? vl2 : vdl)[tid & (BS - 1)] = val;
                 }
+                (gt < BS ? vnl2 : vndl)[gt & (BS - 1)] = val;
                 if (!(ok = group_sync())) break;
             }
-            if (!(ok = mbar_wait(bar(B_SFULL + b), (u >> 1) & 1, abort_flag))) break;
+            if (!(ok = mbar_wait(bar(B_SFULL + grp), (u >> 1) & 1, abort_flag))) break;
             tc_fence_after_sync();
             // does any element of this step need the mask?  (uniform over the CTA)
             //   MODE 0: rows tile*128 .. +127, keys t*64 .. +63;  MODE 1: keys tile*128 .. +127, rows t*64 .. +63
             const int key0 = MODE == 0 ? t * BS : tile * BT, nkeys = MODE == 0 ? BS : BT;
             const int row0 = MODE == 0 ? tile * BT : t * BS;
             const bool partial = (key0 + nkeys > prm.Sk) || (prm.causal && key0 + nkeys - 1 > row0);
-            {
+#pragma unroll
+            for (int ch = 0; ch < BS / 32; ++ch) {
                 uint32_t sr[32], dpr[32], pk_p[16], pk_ds[16];
-                tmem_ld_32x32b_x32(tS + 32 * half, sr);
-                tmem_ld_32x32b_x32(tDP + 32 * half, dpr);
+                tmem_ld_32x32b_x32(tS + 32 * ch, sr);
+                tmem_ld_32x32b_x32(tDP + 32 * ch, dpr);
                 tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
-                    float p[2], ds[2];
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int col = 32 * half + e + h;
-                        float l2, dl;
-                        bool vis = true;
-                        if constexpr (MODE == 0) {
-                            l2 = my_l2;
-                            dl = my_delta;
-                            if (partial) {
-                                const int key = key0 + col;
-                                vis = key < prm.Sk && (!prm.causal || key <= my_row);
-                            }
-                        } else {
-                            l2 = vl2[col];
-                            dl = vdl[col];
-                            if (partial) vis = my_row < prm.Sk && (!prm.causal || my_row <= row0 + col);
-                        }
-                        const float x = fmaf(__uint_as_float(sr[e + h]), c, -l2);
-                        p[h] = vis ? ex2_approx(x) : 0.f;
-                        ds[h] = p[h] * (__uint_as_float(dpr[e + h]) - dl);
+                    const int col = 32 * ch + e;
+                    uint64_t nl2_2, ndl_2;
+                    if constexpr (MODE == 0) {
+                        nl2_2 = pack_f32x2(my_nl2, my_nl2);
+                        ndl_2 = pack_f32x2(my_ndelta, my_ndelta);
+                    } else {
+                        const float2 a = *reinterpret_cast<const float2*>(vnl2 + col);
+                        const float2 d = *reinterpret_cast<const float2*>(vndl + col);
+                        nl2_2 = pack_f32x2(a.x, a.y);
+                        ndl_2 = pack_f32x2(d.x, d.y);
                     }
-                    pk_p[e / 2] = pack2<DTYPE>(p[0], p[1]);
-                    pk_ds[e / 2] = pack2<DTYPE>(ds[0], ds[1]);
+                    float x0, x1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), c2, nl2_2), x0, x1);
+                    float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                    if (partial) {
+                        bool v0, v1;
+                        if constexpr (MODE == 0) {
+                            v0 = key0 + col < prm.Sk && (!prm.causal || key0 + col <= my_row);
+                            v1 = key0 + col + 1 < prm.Sk && (!prm.causal || key0 + col + 1 <= my_row);
+                        } else {
+                            v0 = my_row < prm.Sk && (!prm.causal || my_row <= row0 + col);
+                            v1 = my_row < prm.Sk && (!prm.causal || my_row <= row0 + col + 1);
+                        }
+                        p0 = v0 ? p0 : 0.f;
+                        p1 = v1 ? p1 : 0.f;
+                    }
+                    float d0, d1;
+                    unpack_f32x2(mul_f32x2(pack_f32x2(p0, p1),
+                                           add_f32x2(pack_f32x2(__uint_as_float(dpr[e]), __uint_as_float(dpr[e + 1])), ndl_2)), d0, d1);
+                    if constexpr (MODE == 1) pk_p[e / 2] = pack2<DTYPE>(p0, p1);
+                    pk_ds[e / 2] = pack2<DTYPE>(d0, d1);
                 }
-                // 16-bit results over the columns this thread has just read: 32 values -> 16 columns
+                // 16-bit results over columns this thread has already read: 32 values -> 16 columns
                 if constexpr (MODE == 0) {
-                    tmem_st_32x32b_x16(tS + 32 * half, pk_ds);
+                    tmem_st_32x32b_x16(tS + 16 * ch, pk_ds);
                 } else {
-                    tmem_st_32x32b_x16(tS + 32 * half, pk_p);
-                    tmem_st_32x32b_x16(tDP + 32 * half, pk_ds);
+                    tmem_st_32x32b_x16(tS + 16 * ch, pk_p);
+                    tmem_st_32x32b_x16(tDP + 16 * ch, pk_ds);
                 }
             }
             tmem_st_wait();
             tc_fence_before_sync();
-            mbar_arrive(bar(B_PFULL + b));
+            mbar_arrive(bar(B_PFULL + grp));
         }
 
         // ---- epilogue: accumulators -> 16-bit -> swizzled staging tile -> TMA store (rows beyond the tensor clipped) ----
@@ -449,7 +470,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                     tmem_ld_32x32b_x32(tA + h * 64 + 32 * half, acc);
                     tmem_ld_wait();
                     if (tid == 0) tma_store_wait_read<0>();        // the previous store has read the staging tile
-                    if (!(ok = group_sync())) break;
+                    if (!(ok = all_sync())) break;
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         const uint32_t w0 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 0]) * f, __uint_as_float(acc[g * 8 + 1]) * f);
@@ -460,7 +481,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
                     }
                     fence_proxy_async_smem();
-                    if (!(ok = group_sync())) break;
+                    if (!(ok = all_sync())) break;
                     if (tid == 0) {
                         tma_store_3d(a == 0 ? &tmOut0 : &tmOut1, sOst, h * 64, tile * BT, bh_res);
                         tma_store_commit();

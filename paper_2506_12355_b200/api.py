@@ -124,15 +124,38 @@ def _check_qkv(q, k, v):
     return B, H, Sq, Sk, D
 
 
+def _check_grouped(q, k, v, same_v_dim=True):
+    """The shared checks of the device entry points with grouped K/V heads: q [B,H,Sq,D], k [B,Hkv,Sk,D],
+    v [B,Hkv,Sk,Dv] (Dv == D unless same_v_dim is False), contiguous CUDA tensors of one dtype.
+    Returns (B, H, Hkv, Sq, Sk, D, Dv)."""
+    if q.dim() != 4 or k.dim() != 4 or v.dim() != 4:
+        raise ValueError("q must be [B,H,Sq,D]; k, v must be [B,Hkv,Sk,D]")
+    B, H, Sq, D = q.shape
+    Hkv, Sk, Dv = k.shape[1], k.shape[2], v.shape[3]
+    if tuple(k.shape) != (B, Hkv, Sk, D) or tuple(v.shape) != (B, Hkv, Sk, Dv) or (same_v_dim and Dv != D):
+        raise ValueError("k must be [B,Hkv,Sk,D] and v [B,Hkv,Sk,%s] matching q's B and D" % ("D" if same_v_dim else "Dv"))
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
+        raise ValueError("q, k, v must be contiguous")
+    if not (q.is_cuda and k.is_cuda and v.is_cuda) or not (q.dtype == k.dtype == v.dtype):
+        raise ValueError("q, k, v must be CUDA tensors of one dtype")
+    return B, H, Hkv, Sq, Sk, D, Dv
+
+
+def _outputs(q, B, H, Sq, Dv, out, lse, dtype=None):
+    """O [B,H,Sq,Dv] and LSE [B,H,Sq] (fp32), allocated on q's device when not given."""
+    if out is None:
+        out = torch.empty((B, H, Sq, Dv), dtype=q.dtype if dtype is None else dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    return out, lse
+
+
 def _call_device(fn_name, q, k, v, scale, causal, out, lse, stream):
     B, H, Sq, Sk, D = _check_qkv(q, k, v)
     if not (q.is_cuda and k.is_cuda and v.is_cuda):
         raise ValueError("q, k, v must be CUDA tensors")
     dt = _dtype_code(q)
-    if out is None:
-        out = torch.empty_like(q)
-    if lse is None:
-        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    out, lse = _outputs(q, B, H, Sq, D, out, lse)
     with torch.cuda.device(q.device):
         rc = getattr(load(), fn_name)(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                       lse.data_ptr(), B, H, Sq, Sk, D, float(scale),
@@ -152,21 +175,9 @@ def attn_fwd(q, k, v, scale: float, causal: bool = False, out=None, lse=None, st
 
 def attn_fwd_gqa(q, k, v, scale: float, causal: bool = False, out=None, lse=None, stream=None):
     """Grouped-query / multi-query attention: q [B,H,Sq,D], k, v [B,Hkv,Sk,D] with H % Hkv == 0."""
-    if q.dim() != 4 or k.dim() != 4 or tuple(v.shape) != tuple(k.shape):
-        raise ValueError("q must be [B,H,Sq,D]; k, v must be [B,Hkv,Sk,D]")
-    B, H, Sq, D = q.shape
-    Hkv, Sk = k.shape[1], k.shape[2]
-    if k.shape[0] != B or k.shape[3] != D:
-        raise ValueError("k, v must match q's B and D")
-    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
-        raise ValueError("q, k, v must be contiguous")
-    if not (q.is_cuda and k.is_cuda and v.is_cuda) or not (q.dtype == k.dtype == v.dtype):
-        raise ValueError("q, k, v must be CUDA tensors of one dtype")
+    B, H, Hkv, Sq, Sk, D, _ = _check_grouped(q, k, v)
     dt = _dtype_code(q)
-    if out is None:
-        out = torch.empty_like(q)
-    if lse is None:
-        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    out, lse = _outputs(q, B, H, Sq, D, out, lse)
     with torch.cuda.device(q.device):
         rc = load().attn_fwd_gqa(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
                                  B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)), dt, _stream_ptr(stream))
@@ -178,19 +189,9 @@ def attn_fwd_gqa(q, k, v, scale: float, causal: bool = False, out=None, lse=None
 def attn_fwd_partial(q, k, v, scale: float, causal: bool, k_offset: int, out=None, lse=None, stream=None):
     """Attention over one K/V shard whose first key has global index k_offset: q [B,H,Sq,D],
     k, v [B,Hkv,Sk_shard,D].  Returns the shard's normalised O_r and LSE_r (merge with attn_combine)."""
-    B, H, Sq, D = q.shape
-    Hkv, Sk = k.shape[1], k.shape[2]
-    if tuple(k.shape) != (B, Hkv, Sk, D) or tuple(v.shape) != tuple(k.shape):
-        raise ValueError("k, v must be [B,Hkv,Sk,D]")
-    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
-        raise ValueError("q, k, v must be contiguous")
-    if not (q.is_cuda and k.is_cuda and v.is_cuda) or not (q.dtype == k.dtype == v.dtype):
-        raise ValueError("q, k, v must be CUDA tensors of one dtype")
+    B, H, Hkv, Sq, Sk, D, _ = _check_grouped(q, k, v)
     dt = _dtype_code(q)
-    if out is None:
-        out = torch.empty_like(q)
-    if lse is None:
-        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    out, lse = _outputs(q, B, H, Sq, D, out, lse)
     with torch.cuda.device(q.device):
         rc = load().attn_fwd_partial(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
                                      B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)), int(k_offset), dt,
@@ -246,19 +247,9 @@ def attn_combine_gather(o_part_ptrs, lse_part_ptrs, shape, dtype, out, lse, row_
 def attn_fwd_qkv_dims(q, k, v, scale: float, causal: bool = False, out=None, lse=None, stream=None):
     """Attention with separate Q/K and V head dims (the 192/128 MLA head shape): q [B,H,Sq,Dqk],
     k [B,Hkv,Sk,Dqk], v [B,Hkv,Sk,Dv]; returns o [B,H,Sq,Dv] and lse [B,H,Sq]."""
-    B, H, Sq, Dqk = q.shape
-    Hkv, Sk, Dv = k.shape[1], k.shape[2], v.shape[3]
-    if tuple(k.shape) != (B, Hkv, Sk, Dqk) or tuple(v.shape) != (B, Hkv, Sk, Dv):
-        raise ValueError("k must be [B,Hkv,Sk,Dqk] and v [B,Hkv,Sk,Dv]")
-    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
-        raise ValueError("q, k, v must be contiguous")
-    if not (q.is_cuda and k.is_cuda and v.is_cuda) or not (q.dtype == k.dtype == v.dtype):
-        raise ValueError("q, k, v must be CUDA tensors of one dtype")
+    B, H, Hkv, Sq, Sk, Dqk, Dv = _check_grouped(q, k, v, same_v_dim=False)
     dt = _dtype_code(q)
-    if out is None:
-        out = torch.empty((B, H, Sq, Dv), dtype=q.dtype, device=q.device)
-    if lse is None:
-        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    out, lse = _outputs(q, B, H, Sq, Dv, out, lse)
     with torch.cuda.device(q.device):
         rc = load().attn_fwd_qkv_dims(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
                                       B, H, Hkv, Sq, Sk, Dqk, Dv, float(scale), int(bool(causal)), dt,
@@ -276,21 +267,11 @@ def attn_fwd_splitkv(q, k, v, scale: float, causal: bool, n_splits: int, workspa
     """attn_fwd_gqa with the keys split into n_splits ranges that run concurrently, then merged (split-KV
     decoding).  `workspace`: CUDA uint8 tensor of at least attn_fwd_splitkv_workspace_bytes(...) bytes
     (allocated here when None)."""
-    B, H, Sq, D = q.shape
-    Hkv, Sk = k.shape[1], k.shape[2]
-    if tuple(k.shape) != (B, Hkv, Sk, D) or tuple(v.shape) != tuple(k.shape):
-        raise ValueError("k, v must be [B,Hkv,Sk,D]")
-    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous()):
-        raise ValueError("q, k, v must be contiguous")
-    if not (q.is_cuda and k.is_cuda and v.is_cuda) or not (q.dtype == k.dtype == v.dtype):
-        raise ValueError("q, k, v must be CUDA tensors of one dtype")
+    B, H, Hkv, Sq, Sk, D, _ = _check_grouped(q, k, v)
     dt = _dtype_code(q)
     if workspace is None:
         workspace = torch.empty(attn_fwd_splitkv_workspace_bytes(B, H, Sq, D, n_splits), dtype=torch.uint8, device=q.device)
-    if out is None:
-        out = torch.empty((B, H, Sq, D), dtype=q.dtype, device=q.device)
-    if lse is None:
-        lse = torch.empty((B, H, Sq), dtype=torch.float32, device=q.device)
+    out, lse = _outputs(q, B, H, Sq, D, out, lse)
     with torch.cuda.device(q.device):
         rc = load().attn_fwd_splitkv(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
                                      B, H, Hkv, Sq, Sk, D, float(scale), int(bool(causal)), dt, int(n_splits),
@@ -336,18 +317,15 @@ def attn_bwd(q, k, v, o, lse, dout, scale: float, causal: bool = False, dq=None,
     """Gradients (dq, dk, dv) of the attention output for the upstream gradient dout: q, o, dout [B,H,Sq,D];
     k, v [B,Hkv,Sk,D]; lse [B,H,Sq] fp32; o and lse from the forward call on the same inputs.  D in {64, 128}.
     `workspace`: CUDA uint8 tensor of at least attn_bwd_workspace_bytes(B, H, Sq) bytes (allocated here when None)."""
-    if q.dim() != 4 or k.dim() != 4 or tuple(v.shape) != tuple(k.shape):
-        raise ValueError("q must be [B,H,Sq,D]; k, v must be [B,Hkv,Sk,D]")
-    B, H, Sq, D = q.shape
-    Hkv, Sk = k.shape[1], k.shape[2]
-    if k.shape[0] != B or k.shape[3] != D or tuple(o.shape) != tuple(q.shape) or tuple(dout.shape) != tuple(q.shape):
-        raise ValueError("k, v must match q's B and D; o and dout must have q's shape")
+    B, H, Hkv, Sq, Sk, D, _ = _check_grouped(q, k, v)
+    if tuple(o.shape) != tuple(q.shape) or tuple(dout.shape) != tuple(q.shape):
+        raise ValueError("o and dout must have q's shape")
     if tuple(lse.shape) != (B, H, Sq) or lse.dtype != torch.float32:
         raise ValueError("lse must be fp32 [B,H,Sq]")
-    for t in (q, k, v, o, dout, lse):
+    for t in (o, dout, lse):
         if not (t.is_cuda and t.is_contiguous()):
-            raise ValueError("all tensors must be contiguous CUDA tensors")
-    if not (q.dtype == k.dtype == v.dtype == o.dtype == dout.dtype):
+            raise ValueError("o, dout, lse must be contiguous CUDA tensors")
+    if not (q.dtype == o.dtype == dout.dtype):
         raise TypeError("q, k, v, o, dout must share one dtype")
     dt = _dtype_code(q)
     dq = torch.empty_like(q) if dq is None else dq

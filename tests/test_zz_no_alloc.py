@@ -9,9 +9,11 @@ a caller-allocated workspace) on two calls in a row that share the built-in buff
 size limit is enforced.  It is collected last on purpose: a run that stops at the first failure has
 then already run every other test.  It passes alone in a fresh process and after the other tests.
 """
+import numpy as np
 import pytest
 import torch
 
+from oracle import attn_oracle as orc
 from paper_2506_12355_b200 import api, inputs
 
 CASES = [
@@ -40,7 +42,7 @@ def test_static_entry_matches_host_entry_on_two_calls_in_a_row():
     for idx, (B, H, Sq, Sk, D, dtype, causal) in enumerate(CASES):
         q, k, v = inputs.make_qkv(B, H, Sq, Sk, D, dtype, seed=900 + idx)
         q, k, v = q.pin_memory(), k.pin_memory(), v.pin_memory()
-        scale = 1.0 / D ** 0.5
+        scale = float(np.float32(1.0) / np.sqrt(np.float32(D)))   # the fp32 value the library receives
         prepared.append((q, k, v, scale, causal, _host_reference(q, k, v, scale, causal)))
 
     # two calls back to back on one stream, both through the built-in buffer; nothing is allocated
@@ -50,9 +52,14 @@ def test_static_entry_matches_host_entry_on_two_calls_in_a_row():
         o = torch.full_like(q, float("nan")).pin_memory()
         lse = torch.full((q.shape[0], q.shape[1], q.shape[2]), float("nan"), dtype=torch.float32).pin_memory()
         outs.append((o, lse))
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
     for (q, k, v, scale, causal, _), (o, lse) in zip(prepared, outs):
         api.attn_fwd_host_static(q, k, v, scale, causal, o, lse)
     assert api.attn_last_device_status() == 0     # synchronises the stream
+    free_after, _ = torch.cuda.mem_get_info()
+    # the driver's own count of free device memory: the two calls took none (this process is the GPU's only user)
+    assert free_after == free_before
 
     for (q, k, v, scale, causal, (o_ref, lse_ref)), (o, lse) in zip(prepared, outs):
         tol = 1e-2 if q.dtype == torch.float16 else 2e-2
@@ -61,6 +68,11 @@ def test_static_entry_matches_host_entry_on_two_calls_in_a_row():
         assert float((lse - lse_ref).abs().max()) <= 1e-3
         # same kernel, same inputs: in fact the bytes are identical
         assert torch.equal(o.view(torch.int16), o_ref.view(torch.int16)) and torch.equal(lse, lse_ref)
+        # and, like every other entry point, against the fp64 oracle itself
+        dtype = inputs.DTYPE_FP16 if q.dtype == torch.float16 else inputs.DTYPE_BF16
+        want_o, want_l = orc.attention(*(orc.widen(inputs.bits(t), dtype) for t in (q, k, v)), scale, causal)
+        assert np.abs(o.double().numpy() - want_o).max() <= tol
+        assert np.abs(lse.double().numpy() - want_l).max() <= 1e-3
 
 
 @pytest.mark.gpu

@@ -13,6 +13,7 @@ named configuration (default C5, the configuration the target is quoted on).  Ra
   errors                the timed output against the fp64 oracle rows that the cpu_baseline leg computes
   configs               C1..C5, each timed as isolated launches (L2 flushed in between) with its own errors
   sustained             the same launch back to back for a few seconds, with the sampled SM clock
+  backward              attn_bwd on the two causal configurations (time, TFLOP/s) and its errors on a small problem
   e2e                   host buffers through attn_fwd_host, copies inside the timed region
   cpu_baseline          the oracle timed on this machine's host cores on a bounded row sample
 
@@ -349,6 +350,44 @@ def sustained_block(prob, sampler_index, peaks, seconds, ms_guess):
             "power_w_max": clocks.get("power_w_max"), "reasons": clocks.get("reasons"), "clock_samples": clocks.get("samples")}
 
 
+def backward_block(api, dev, peaks, flush, with_errors):
+    """The backward pass (attn_bwd: row sums, dQ pass, dK/dV pass) on the two causal bf16 configurations, timed as
+    isolated calls; FLOPs counted as 2.5 x the forward count (five tile products, of which the two passes execute
+    seven).  Errors: a small problem against the oracle's fp64 gradients."""
+    out = {"flops_counted": "2.5 x forward (S, dP, dV, dQ, dK); the kernels execute 3.5 x (S and dP once per pass)"}
+    for name in ("C3", "C5"):
+        cfg = inputs.CONFIGS[name]
+        prob = Problem(api, cfg, dev)
+        prob.step()
+        dout = inputs.randn16((cfg.B, cfg.H, cfg.Sq, cfg.D), inputs.BASE_SEED + 1000 * cfg.index + 3, cfg.dtype).to(dev)
+        dq, dk, dv = torch.empty_like(prob.qd), torch.empty_like(prob.kd), torch.empty_like(prob.vd)
+        ws = torch.empty(api.attn_bwd_workspace_bytes(cfg.B, cfg.H, cfg.Sq), dtype=torch.uint8, device=dev)
+        ms = time_isolated(lambda: api.attn_bwd(prob.qd, prob.kd, prob.vd, prob.o, prob.lse, dout, cfg.scale, cfg.causal,
+                                                dq=dq, dk=dk, dv=dv, workspace=ws), flush, 20, warmup=3)
+        med = float(np.median(ms))
+        tf = 2.5 * cfg.flops / med / 1e9
+        out[name] = {"workload": cfg.workload.replace("fwd", "bwd"), "ms_median": med, "ms_min": min(ms), "tflops": tf,
+                     "frac_of_burst": tf / peaks["bf16_tflops"], "gpu_launches_per_call": 3}
+        del prob, dout, dq, dk, dv, ws
+    if with_errors:
+        from oracle import attn_oracle as orc   # oracle leg: gradients of a small problem
+        B, H, S, D, dt = 1, 4, 1024, 128, inputs.DTYPE_BF16
+        q, k, v = inputs.make_qkv(B, H, S, S, D, dt, inputs.BASE_SEED + 555)
+        dout = inputs.randn16((B, H, S, D), inputs.BASE_SEED + 558, dt)
+        scale = float(np.float32(1.0) / np.sqrt(np.float32(D)))
+        qd, kd, vd, dd = q.to(dev), k.to(dev), v.to(dev), dout.to(dev)
+        o, lse = api.attn_fwd(qd, kd, vd, scale, True)
+        got = api.attn_bwd(qd, kd, vd, o, lse, dd, scale, True)
+        ref = orc.attention_bwd(*(orc.widen(inputs.bits(t), dt) for t in (q, k, v, dout)), scale, True)
+        e = {"problem": "causal bf16 B=1 H=4 S=1024 D=128"}
+        for nm, g, r in zip(("dq", "dk", "dv"), got, ref):
+            err = np.abs(g.cpu().double().numpy() - r)
+            e[nm] = {"max_abs": float(err.max()), "rms_rel": float(math.sqrt((err ** 2).mean() / (r ** 2).mean())),
+                     "ref_rms": float(math.sqrt((r ** 2).mean()))}
+        out["errors"] = e
+    return out
+
+
 def kv_sharded_check(api, dev, rank, world):
     """A small K/V-sharded problem through dist.kv_sharded_attention with both exchange forms; rank 0 compares
     the merged result with the oracle (max-abs errors).  Every rank takes the same branches."""
@@ -485,7 +524,7 @@ def run_ours(args, cfg):
 
     # ---- single GPU only: the oracle on this machine's host cores, the errors of the timed output against it,
     # every configuration as isolated launches, and the sustained run ----
-    cpu = errors = configs = sustained = None
+    cpu = errors = configs = sustained = backward = None
     if world == 1 and not args.no_cpu_baseline:
         # calibrate on a small sample, then size the timed sample for roughly 15 s of CPU work
         cal_rph = max(1, ORACLE_ROWS_PER_HEAD[cfg.name] // 8)
@@ -502,6 +541,8 @@ def run_ours(args, cfg):
         configs = config_block(api, dev, peaks, flush, prob, errors, with_errors=not args.no_cpu_baseline)
     if world == 1 and args.sustained_s > 0:
         sustained = sustained_block(prob, local_rank, peaks, args.sustained_s, ms_per_step_local)
+    if world == 1 and not args.no_configs:
+        backward = backward_block(api, dev, peaks, flush, with_errors=not args.no_cpu_baseline)
     if api.attn_last_device_status() != 0:
         raise SystemExit("device timeout status after the timed region")
 
@@ -521,7 +562,7 @@ def run_ours(args, cfg):
                         "measured_sustained": 100 * value / world / peaks["bf16_tflops_sustained"]
                         if peaks["bf16_tflops_sustained"] else None,
                         "datasheet_2250": 100 * value / world / 2250.0},
-        "sustained": sustained, "configs": configs,
+        "sustained": sustained, "configs": configs, "backward": backward,
     }
     if kv_check is not None:
         line["kv_sharded_check"] = kv_check

@@ -23,17 +23,23 @@
 // Recomputing S and dP in both passes costs 7 tile products instead of 5 but needs no atomics and no
 // cross-CTA reduction, so the results are deterministic.  delta is computed by a small kernel first.
 //
-// The streamed side advances 64 rows per step, and the S / dP tiles of a step (128 lanes x 64 columns each)
-// are double-buffered in tensor memory: while the element-wise warps work on step u, the tensor core
-// already computes S and dP of step u + 1 and the accumulating products of step u - 1.
+// The streamed side advances 64 rows per step.  The fp32 S / dP tiles of a step (128 lanes x 64 columns each)
+// have ONE place in tensor memory, which an element-wise group frees as soon as it has the tile in registers;
+// the 16-bit operands it makes from them go to one of two small operand regions.  So while a group computes,
+// the tensor core already produces S and dP of the next step for the other group, and the accumulating products
+// of a step run whenever its operands are ready.
 //
 //   warps 0-3  element-wise group of the even steps (one thread per tensor-memory lane), then the epilogue
 //   warps 4-7  element-wise group of the odd steps
 //   warp  8    MMA issuer
 //   warp  9    TMA producer
+//   warps 10-11 idle (they complete the third warpgroup so that registers can be re-balanced: an element-wise
+//              thread holds a whole S and dP row of a step, 128 registers, while it computes)
 //
 // Every wait is bounded (see sm100_ptx.cuh); a timed-out wait ends the CTA through the normal exit.
 #pragma once
+#include <type_traits>
+
 #include "attn_tc_common.cuh"
 
 namespace attn_grad {
@@ -54,10 +60,11 @@ struct BwdCfg {
     static constexpr int TILE_BYTES = 2 * RES_BYTES + NSTAGE * 2 * STR_BYTES + OST_BYTES + VEC_BYTES;
     static constexpr int MISC_BYTES = 256;
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
-    static constexpr int THREADS = 320;
-    // tensor memory: step buffer b holds S in columns 128 b .. + 63 and dP in 128 b + 64 .. + 63
-    __host__ __device__ static constexpr int s_col(int b) { return 128 * b; }
-    __host__ __device__ static constexpr int dp_col(int b) { return 128 * b + 64; }
+    static constexpr int THREADS = 384;
+    // tensor memory: fp32 S in columns 0 .. 63, fp32 dP in 64 .. 127; operand region g (steps u = g mod 2) at
+    // 128 + 64 g: first 16-bit operand (dS in MODE 0, P^T in MODE 1) in its columns 0 .. 31, second (dS^T) in 32 .. 63
+    static constexpr int S_COL = 0, DP_COL = 64;
+    __host__ __device__ static constexpr int op_col(int g) { return 128 + 64 * g; }
     static constexpr int ACC0_COL = 256, ACC1_COL = 256 + D;
     static constexpr int TMEM_COLS = 512;
     static_assert(D == 64 || D == 128, "head dims 64 and 128");
@@ -132,7 +139,7 @@ __global__ void attn_bwd_delta_kernel(const void* __restrict__ o, const void* __
 // the streamed tiles, boxes of 64 rows (MODE 0: K, V; MODE 1: Q, dO); tmOut0 / tmOut1: MODE 0: dQ, unused;
 // MODE 1: dV, dK (boxes of 128 rows).
 template <int D, int DTYPE, int MODE>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(384, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant__ CUtensorMap tmR1,
                 const __grid_constant__ CUtensorMap tmT0, const __grid_constant__ CUtensorMap tmT1,
                 const __grid_constant__ CUtensorMap tmOut0, const __grid_constant__ CUtensorMap tmOut1,
@@ -153,14 +160,16 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
     const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
     enum {
         B_RFULL = 0,      // resident tiles loaded (TMA bytes)
-        B_SFULL = 1,      // [2] S and dP of a step are in buffer b (MMA commit)
-        B_PFULL = 3,      // [2] the 16-bit operands of a step are in buffer b (the 128 threads of group b)
-        B_ACCFINAL = 5,   // the last accumulating product has finished
-        B_GSYNC = 6,      // [2] barrier among the 128 threads of a group
-        B_ESYNC = 8,      // barrier among all 256 element-wise threads (epilogue)
-        B_TFULL = 9,      // [NSTAGE] streamed tiles loaded
-        B_TEMPTY = 9 + NSTAGE,
-        B_COUNT = 9 + 2 * NSTAGE
+        B_SFULL = 1,      // [2] S and dP of a step of group g are in tensor memory (MMA commit)
+        B_SREAD = 3,      // [2] group g has them in registers: S and dP may be overwritten (128 threads)
+        B_PFULL = 5,      // [2] the 16-bit operands of a step are in operand region g (128 threads)
+        B_OPFREE = 7,     // [2] the accumulating products of a step have read operand region g (MMA commit)
+        B_ACCFINAL = 9,   // the last accumulating product has finished
+        B_GSYNC = 10,     // [2] barrier among the 128 threads of a group
+        B_ESYNC = 12,     // barrier among all 256 element-wise threads (epilogue)
+        B_TFULL = 13,     // [NSTAGE] streamed tiles loaded
+        B_TEMPTY = 13 + NSTAGE,
+        B_COUNT = 13 + 2 * NSTAGE
     };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
@@ -219,7 +228,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         mbar_init(bar(B_RFULL), 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(B_SFULL + b), 1);
+            mbar_init(bar(B_SREAD + b), 128);
             mbar_init(bar(B_PFULL + b), 128);
+            mbar_init(bar(B_OPFREE + b), 1);
             mbar_init(bar(B_GSYNC + b), 128);
         }
         mbar_init(bar(B_ACCFINAL), 1);
@@ -248,7 +259,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 9) {
+    // Register re-balancing: 384 threads start with 168 registers each; the service warpgroup (warps 8-11) drops
+    // to 64 and the two element-wise warpgroups rise to 216.
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+      if (warp == 9) {
         // =========================== TMA producer ===========================
         const bool leader = elect_one();
         if (leader) {
@@ -272,69 +287,87 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 }
             }
         }
-    } else if (warp == 8) {
+      } else if (warp == 8) {
         // =========================== MMA issuer ===========================
         const bool leader = elect_one();
         constexpr uint32_t IDESC_S = make_idesc_f16(BT, BS, DTYPE, 0, 0);    // both operands K-major (contraction over D)
         constexpr uint32_t IDESC_ACC = make_idesc_f16(BT, D, DTYPE, 0, 1);   // A from tensor memory, B MN-major (N = D)
         constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
         const uint32_t r_lo[2] = {smem_desc_lo(sR(0), 16), smem_desc_lo(sR(1), 16)};
-        // The 16-bit A operands lie over the fp32 tiles they were made from: the 64 values of a step occupy the
-        // first 32 columns of its S (or dP) columns, so contraction step kk (16 values) starts at column 8 kk.
-        auto a_col = [](int kk) { return kk * 8; };
-        bool ok = mbar_wait(bar(B_RFULL), 0, abort_flag);
-        // software pipeline: iteration u issues S, dP of step u, then the accumulating products of step u - 1
+        // S (or S^T) = R0 T0^T, dP (or dP^T) = R1 T1^T of step u : D / 16 instructions each (M 128, N 64, K 16)
+        auto issue_s = [&](int u) {
+            if (leader) {
+                const int st = u % NSTAGE;
+#pragma unroll
+                for (int w = 0; w < 2; ++w) {
+                    const uint32_t b0 = smem_desc_lo(sT(st, w), 16);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t offa = ((kk >> 2) * BT * 128 + (kk & 3) * 32) >> 4;
+                        const uint32_t offb = ((kk >> 2) * BS * 128 + (kk & 3) * 32) >> 4;
+                        mma_f16_ss_lohi(tmem + (w == 0 ? C::S_COL : C::DP_COL), r_lo[w] + offa, b0 + offb, DESC_HI, IDESC_S, kk > 0);
+                    }
+                }
+                mma_commit(bar(B_SFULL + (u & 1)));
+            }
+        };
+        bool ok = mbar_wait(bar(B_RFULL), 0, abort_flag) && mbar_wait(bar(B_TFULL), 0, abort_flag);
+        if (ok) {
+            tc_fence_after_sync();
+            issue_s(0);
+        }
+        // accumulating products of step v (contraction step kk, 16 values = 8 columns, starts at column 8 kk of its
+        // operand); afterwards its streamed tiles and its operand region are free
+        auto issue_acc = [&](int v) {
+            if (leader) {
+                const int st = v % NSTAGE;
+                const uint32_t op = tmem + C::op_col(v & 1);
+                if constexpr (MODE == 0) {
+                    // dQ += dS K_j : dS from tensor memory, K_j MN-major
+                    const uint32_t b0 = smem_desc_lo(sT(st, 0), BS * 128);
+#pragma unroll
+                    for (int kk = 0; kk < BS / 16; ++kk)
+                        mma_f16_ts_lohi(tmem + C::ACC0_COL, op + kk * 8, b0 + ((kk * 16 * 128) >> 4), DESC_HI,
+                                        IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
+                } else {
+                    // dV += P^T dO_i, dK += dS^T Q_i; dO_i and Q_i MN-major
+                    const uint32_t bdo = smem_desc_lo(sT(st, 1), BS * 128), bq = smem_desc_lo(sT(st, 0), BS * 128);
+#pragma unroll
+                    for (int kk = 0; kk < BS / 16; ++kk)
+                        mma_f16_ts_lohi(tmem + C::ACC0_COL, op + kk * 8, bdo + ((kk * 16 * 128) >> 4), DESC_HI,
+                                        IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int kk = 0; kk < BS / 16; ++kk)
+                        mma_f16_ts_lohi(tmem + C::ACC1_COL, op + 32 + kk * 8, bq + ((kk * 16 * 128) >> 4), DESC_HI,
+                                        IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
+                }
+                mma_commit(bar(B_TEMPTY + st));
+                mma_commit(bar(B_OPFREE + (v & 1)));
+                if (v + 1 == n_steps) mma_commit(bar(B_ACCFINAL));
+            }
+        };
+        // Iteration u: S and dP of step u + 1 as soon as step u's are in its group's registers, then the
+        // accumulating products of step u - 1, whose operands have had a whole step to get ready: the tensor core
+        // does not wait for the element-wise warps unless they fall a full step behind.
         for (int u = 0; u <= n_steps && ok; ++u) {
             if (u < n_steps) {
-                const int st = u % NSTAGE, b = u & 1;
-                if (!(ok = mbar_wait(bar(B_TFULL + st), (u / NSTAGE) & 1, abort_flag))) break;
-                tc_fence_after_sync();
-                if (leader) {
-                    // S (or S^T) = R0 T0^T, dP (or dP^T) = R1 T1^T : D / 16 instructions each (M 128, N 64, K 16).
-                    // Buffer b was last read by the accumulating products of step u - 2, issued before these.
-#pragma unroll
-                    for (int w = 0; w < 2; ++w) {
-                        const uint32_t b0 = smem_desc_lo(sT(st, w), 16);
-#pragma unroll
-                        for (int kk = 0; kk < D / 16; ++kk) {
-                            const uint32_t offa = ((kk >> 2) * BT * 128 + (kk & 3) * 32) >> 4;
-                            const uint32_t offb = ((kk >> 2) * BS * 128 + (kk & 3) * 32) >> 4;
-                            mma_f16_ss_lohi(tmem + (w == 0 ? C::s_col(b) : C::dp_col(b)), r_lo[w] + offa, b0 + offb, DESC_HI, IDESC_S, kk > 0);
-                        }
-                    }
-                    mma_commit(bar(B_SFULL + b));
+                if (!(ok = mbar_wait(bar(B_SREAD + (u & 1)), (u >> 1) & 1, abort_flag))) break;
+                if (u + 1 < n_steps) {
+                    if (!(ok = mbar_wait(bar(B_TFULL + (u + 1) % NSTAGE), ((u + 1) / NSTAGE) & 1, abort_flag))) break;
+                    tc_fence_after_sync();
+                    issue_s(u + 1);
                 }
             }
             if (u >= 1) {
-                const int v = u - 1, st = v % NSTAGE, b = v & 1;
-                if (!(ok = mbar_wait(bar(B_PFULL + b), (v >> 1) & 1, abort_flag))) break;
+                const int v = u - 1;
+                if (!(ok = mbar_wait(bar(B_PFULL + (v & 1)), (v >> 1) & 1, abort_flag))) break;
                 tc_fence_after_sync();
-                if (leader) {
-                    if constexpr (MODE == 0) {
-                        // dQ += dS K_j : dS from tensor memory (over S), K_j MN-major
-                        const uint32_t b0 = smem_desc_lo(sT(st, 0), BS * 128);
-#pragma unroll
-                        for (int kk = 0; kk < BS / 16; ++kk)
-                            mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::s_col(b) + a_col(kk), b0 + ((kk * 16 * 128) >> 4), DESC_HI,
-                                            IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
-                    } else {
-                        // dV += P^T dO_i (P^T over S^T), dK += dS^T Q_i (dS^T over dP^T); dO_i and Q_i MN-major
-                        const uint32_t bdo = smem_desc_lo(sT(st, 1), BS * 128), bq = smem_desc_lo(sT(st, 0), BS * 128);
-#pragma unroll
-                        for (int kk = 0; kk < BS / 16; ++kk)
-                            mma_f16_ts_lohi(tmem + C::ACC0_COL, tmem + C::s_col(b) + a_col(kk), bdo + ((kk * 16 * 128) >> 4), DESC_HI,
-                                            IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
-#pragma unroll
-                        for (int kk = 0; kk < BS / 16; ++kk)
-                            mma_f16_ts_lohi(tmem + C::ACC1_COL, tmem + C::dp_col(b) + a_col(kk), bq + ((kk * 16 * 128) >> 4), DESC_HI,
-                                            IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
-                    }
-                    mma_commit(bar(B_TEMPTY + st));
-                    if (v + 1 == n_steps) mma_commit(bar(B_ACCFINAL));
-                }
+                issue_acc(v);
             }
         }
+      }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         // =========================== element-wise groups + epilogue ===========================
         // Group g (warps 4g .. 4g+3) takes the steps u = g, g + 2, ...: always step buffer g.  While one group
         // waits for its tile or for tensor memory, the other computes.
@@ -343,7 +376,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         const int r = (warp & 3) * 32 + lane;                // tensor-memory lane: query row (MODE 0) / key row (MODE 1)
         const int gt = tid & 127;                            // thread index inside the group
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + C::s_col(grp) + lane_off, tDP = tmem + C::dp_col(grp) + lane_off;
+        const uint32_t tS = tmem + C::S_COL + lane_off, tDP = tmem + C::DP_COL + lane_off;
+        const uint32_t tOP = tmem + C::op_col(grp) + lane_off;
         const float c = prm.scale_log2;
         const uint64_t c2 = pack_f32x2(c, c);
         const int my_row = tile * BT + r;                    // global query row (MODE 0) or key index (MODE 1)
@@ -371,28 +405,33 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             ++esync_phase;
             return done;
         };
+        // MODE 1: this group's 128 threads fetch one value of a step's 64 query rows each: threads 0..63 -L log2(e),
+        // 64..127 -delta.  The value for the group's NEXT step is fetched before the current step is computed, so the
+        // latency of the load is not on the path.
+        // (The loaded value is not touched until it is stored to shared memory one step later: any arithmetic on it
+        // here would make the thread wait for the load at once.)
+        auto fetch_vec = [&](int u) -> float {
+            float raw = 0.f;
+            if (u < n_steps) {
+                const int qr = step_sub(u) * BS + (gt & (BS - 1));
+                if (qr < prm.Sq) raw = (gt < BS ? prm.lse : prm.delta)[static_cast<int64_t>(step_head(u)) * prm.Sq + qr];
+            }
+            return raw;
+        };
+        float vec_next = 0.f;
+        if constexpr (MODE == 1) vec_next = fetch_vec(grp);
         for (int u = grp; u < n_steps && ok; u += 2) {
             const int t = step_sub(u);
-            // MODE 1: -L * log2(e) and -delta of the step's 64 query rows, in one of the group's two buffers
+            // MODE 1: the step's values in one of the group's two buffers
             float* vnl2 = vec + (grp * 2 + ((u >> 1) & 1)) * 2 * BS;
             float* vndl = vnl2 + BS;
             if constexpr (MODE == 1) {
-                // this group's 128 threads fetch one value each: threads 0..63 L, 64..127 delta.  A thread that
-                // writes buffer x for step u has passed the barrier of step u - 2, which every thread of the group
-                // reaches only after its reads of buffer x for step u - 4.
-                const int qr = t * BS + (gt & (BS - 1));
-                float val = 0.f;
-                if (qr < prm.Sq) {
-                    const int64_t g = static_cast<int64_t>(step_head(u)) * prm.Sq + qr;
-                    if (gt < BS) {
-                        const float l = prm.lse[g];
-                        val = (l == -INFINITY) ? -INFINITY : -l * LOG2E;
-                    } else {
-                        val = -prm.delta[g];
-                    }
-                }
-                (gt < BS ? vnl2 : vndl)[gt & (BS - 1)] = val;
+                // A thread that writes buffer x for step u has passed the barrier of step u - 2, which every thread
+                // of the group reaches only after its reads of buffer x for step u - 4.
+                // L = -inf: a row without visible keys, P = 0
+                (gt < BS ? vnl2 : vndl)[gt & (BS - 1)] = gt < BS ? (vec_next == -INFINITY ? -INFINITY : -vec_next * LOG2E) : -vec_next;
                 if (!(ok = group_sync())) break;
+                vec_next = fetch_vec(u + 2);
             }
             if (!(ok = mbar_wait(bar(B_SFULL + grp), (u >> 1) & 1, abort_flag))) break;
             tc_fence_after_sync();
@@ -401,12 +440,25 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             const int key0 = MODE == 0 ? t * BS : tile * BT, nkeys = MODE == 0 ? BS : BT;
             const int row0 = MODE == 0 ? tile * BT : t * BS;
             const bool partial = (key0 + nkeys > prm.Sk) || (prm.causal && key0 + nkeys - 1 > row0);
+            // the whole S and dP row of this step into registers, then tensor memory is free for the next step
+            uint32_t sr[BS], dpr[BS];
 #pragma unroll
             for (int ch = 0; ch < BS / 32; ++ch) {
-                uint32_t sr[32], dpr[32], pk_p[16], pk_ds[16];
-                tmem_ld_32x32b_x32(tS + 32 * ch, sr);
-                tmem_ld_32x32b_x32(tDP + 32 * ch, dpr);
-                tmem_ld_wait();
+                tmem_ld_32x32b_x32(tS + 32 * ch, sr + 32 * ch);
+                tmem_ld_32x32b_x32(tDP + 32 * ch, dpr + 32 * ch);
+            }
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            mbar_arrive(bar(B_SREAD + grp));
+            // operand region `grp` was last read by the accumulating products of step u - 2
+            bool op_free = u < 2;
+            // Two instances of the arithmetic: steps that need the mask (diagonal and ragged tiles) and all others,
+            // whose code then carries no trace of the mask (predicated-off mask code more than doubled its time).
+            auto make_operands = [&](auto masked_tag) {
+            constexpr bool MASKED = decltype(masked_tag)::value;
+#pragma unroll
+            for (int ch = 0; ch < BS / 32; ++ch) {
+                uint32_t pk_p[16], pk_ds[16];
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
                     const int col = 32 * ch + e;
@@ -421,9 +473,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                         ndl_2 = pack_f32x2(d.x, d.y);
                     }
                     float x0, x1;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), c2, nl2_2), x0, x1);
+                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[col]), __uint_as_float(sr[col + 1])), c2, nl2_2), x0, x1);
                     float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                    if (partial) {
+                    if constexpr (MASKED) {
                         bool v0, v1;
                         if constexpr (MODE == 0) {
                             v0 = key0 + col < prm.Sk && (!prm.causal || key0 + col <= my_row);
@@ -437,18 +489,26 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                     }
                     float d0, d1;
                     unpack_f32x2(mul_f32x2(pack_f32x2(p0, p1),
-                                           add_f32x2(pack_f32x2(__uint_as_float(dpr[e]), __uint_as_float(dpr[e + 1])), ndl_2)), d0, d1);
+                                           add_f32x2(pack_f32x2(__uint_as_float(dpr[col]), __uint_as_float(dpr[col + 1])), ndl_2)), d0, d1);
                     if constexpr (MODE == 1) pk_p[e / 2] = pack2<DTYPE>(p0, p1);
                     pk_ds[e / 2] = pack2<DTYPE>(d0, d1);
                 }
-                // 16-bit results over columns this thread has already read: 32 values -> 16 columns
+                // 32 values -> 16 columns of this group's operand region
+                if (!op_free) {
+                    if (!(ok = mbar_wait(bar(B_OPFREE + grp), ((u >> 1) - 1) & 1, abort_flag))) break;
+                    tc_fence_after_sync();
+                    op_free = true;
+                }
                 if constexpr (MODE == 0) {
-                    tmem_st_32x32b_x16(tS + 16 * ch, pk_ds);
+                    tmem_st_32x32b_x16(tOP + 16 * ch, pk_ds);
                 } else {
-                    tmem_st_32x32b_x16(tS + 16 * ch, pk_p);
-                    tmem_st_32x32b_x16(tDP + 16 * ch, pk_ds);
+                    tmem_st_32x32b_x16(tOP + 16 * ch, pk_p);
+                    tmem_st_32x32b_x16(tOP + 32 + 16 * ch, pk_ds);
                 }
             }
+            };
+            if (partial) make_operands(std::true_type{}); else make_operands(std::false_type{});
+            if (!ok) break;
             tmem_st_wait();
             tc_fence_before_sync();
             mbar_arrive(bar(B_PFULL + grp));

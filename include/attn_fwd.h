@@ -224,9 +224,10 @@ int attn_fwd_fp8(const void* q, const void* k, const void* v, void* o, float* ls
  * dq         : device, [B,H,Sq,D] (written);  dk, dv: device, [B,Hkv,Sk,D] (written; with grouped heads
  *              they hold the sum over the query heads of the group).  Same 16-bit type as the inputs.
  * D in {64, 128} (otherwise ATTN_ERR_UNSUPPORTED_HEAD_DIM); top-left causal mask as in attn_fwd.
- * workspace  : device, 256-byte aligned, at least attn_bwd_workspace_bytes(B,H,Sq) bytes (it holds
- *              rowsum(dO o O) in fp32); owned by the caller, may be reused as soon as the stream has
- *              passed this call.  Missing, misaligned or too small: ATTN_ERR_WORKSPACE.
+ * workspace  : device, 256-byte aligned, at least attn_bwd_workspace_bytes(B,H,Sq) bytes (it holds two
+ *              fp32 values per query row, -LSE log2(e) and -rowsum(dO o O), rows padded to a multiple
+ *              of 64 per head); owned by the caller, may be reused as soon as the stream has passed
+ *              this call.  Missing, misaligned or too small: ATTN_ERR_WORKSPACE.
  * Rows of dq whose query sees no key, and rows of dk, dv whose key no query sees, are zero.  Empty
  * tensors may come with NULL pointers.  Three kernels are enqueued on `stream` (the row sums, the dQ
  * pass, the dK/dV pass); nothing is synchronised; the results are deterministic (no atomics).

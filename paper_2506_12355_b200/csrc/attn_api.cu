@@ -791,9 +791,12 @@ int attn_fwd_fp8(const void* q, const void* k, const void* v, void* o, float* ls
     return launch_tc_pipe<128, ATTN_DTYPE_FP8_E4M3>(q, k, v, o, lse, B, H, Hkv, Sq, Sk, s_eff, causal, 0, st, v_factor);
 }
 
+// attn_bwd's workspace: two fp32 row vectors [B*H][Sq_pad], Sq_pad = Sq rounded up to a multiple of 64
+size_t bwd_sq_pad(int Sq) { return (static_cast<size_t>(Sq) + 63) / 64 * 64; }
+
 size_t attn_bwd_workspace_bytes(int B, int H, int Sq) {
     if (B < 0 || H < 0 || Sq < 0) return 0;
-    return align256(static_cast<size_t>(B) * H * Sq * sizeof(float));
+    return 2 * align256(static_cast<size_t>(B) * H * bwd_sq_pad(Sq) * sizeof(float));
 }
 
 int attn_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dout, void* dq,
@@ -829,10 +832,13 @@ int attn_bwd(const void* q, const void* k, const void* v, const void* o, const f
     const int64_t BH = static_cast<int64_t>(B) * H, BHkv = static_cast<int64_t>(B) * Hkv;
     const int64_t n_qtiles = (static_cast<int64_t>(Sq) + 127) / 128, n_ktiles = (static_cast<int64_t>(Sk) + 127) / 128;
     if (n_qtiles * BH > 2147483647LL || n_ktiles * BHkv > 2147483647LL) return ATTN_ERR_BAD_SHAPE;
-    float* delta = static_cast<float*>(workspace);
+    const int64_t sq_pad = static_cast<int64_t>(bwd_sq_pad(Sq));
+    float* nl2 = static_cast<float*>(workspace);
+    float* ndelta = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align256(static_cast<size_t>(BH) * sq_pad * sizeof(float)));
     attn_grad::BwdParams prm;
-    prm.lse = lse;
-    prm.delta = delta;
+    prm.nl2 = nl2;
+    prm.ndelta = ndelta;
+    prm.Sq_pad = static_cast<int>(sq_pad);
     prm.Sq = Sq;
     prm.Sk = Sk;
     prm.scale = scale;
@@ -861,10 +867,11 @@ int attn_bwd(const void* q, const void* k, const void* v, const void* o, const f
         if (!allow_dynamic_smem(reinterpret_cast<const void*>(kq), C::SMEM_BYTES) ||                                       \
             !allow_dynamic_smem(reinterpret_cast<const void*>(kkv), C::SMEM_BYTES))                                        \
             return ATTN_ERR_CUDA;                                                                                          \
-        const int64_t rows = BH * Sq;                                                                                      \
+        const int64_t rows = BH * sq_pad;                                                                                  \
         int64_t blocks = (rows + 7) / 8;                                                                                   \
         if (blocks > 148 * 16) blocks = 148 * 16;                                                                          \
-        attn_grad::attn_bwd_delta_kernel<DD, TT><<<static_cast<unsigned>(blocks), 256, 0, st>>>(o, dout, delta, rows);        \
+        attn_grad::attn_bwd_rows_kernel<DD, TT><<<static_cast<unsigned>(blocks), 256, 0, st>>>(o, dout, lse, nl2, ndelta, Sq, \
+                                                                                              prm.Sq_pad, rows);          \
         prm.out0 = dq;                                                                                                     \
         prm.out1 = nullptr;                                                                                                \
         kq<<<static_cast<unsigned>(n_qtiles * BH), C::THREADS, C::SMEM_BYTES, st>>>(mq, mdo, mk64, mv64, mdq, mdq, prm);       \

@@ -56,7 +56,7 @@ struct BwdCfg {
     static constexpr int STR_BYTES = BS * D * 2;            // one streamed tile
     static constexpr int NSTAGE = D == 128 ? 4 : 6;           // ring stages, each holds the two streamed tiles
     static constexpr int OST_BYTES = BT * 128;              // epilogue staging: 128 rows x 64 columns
-    static constexpr int VEC_BYTES = 2 * 2 * 2 * BS * 4;    // MODE 1: L and delta of the streamed rows: two groups x two buffers
+    static constexpr int VEC_BYTES = NSTAGE * 2 * BS * 4;   // MODE 1: -L log2(e) and -delta of a stage's 64 streamed query rows
     static constexpr int TILE_BYTES = 2 * RES_BYTES + NSTAGE * 2 * STR_BYTES + OST_BYTES + VEC_BYTES;
     static constexpr int MISC_BYTES = 256;
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
@@ -71,8 +71,11 @@ struct BwdCfg {
 };
 
 struct BwdParams {
-    const float* lse;       // [B,H,Sq] natural-log logsumexp of the scaled scores, from the forward pass
-    const float* delta;     // [B,H,Sq] rowsum(dO o O)
+    // Row vectors prepared by attn_bwd_rows_kernel, [B*H][Sq_pad] fp32 each (Sq_pad: Sq rounded up to a multiple
+    // of 64, the padding rows hold 0, so that 64 rows from any multiple of 64 are one aligned, in-bounds block):
+    const float* nl2;       // -LSE * log2(e)   (-inf for rows without a visible key: their P is 0)
+    const float* ndelta;    // -rowsum(dO o O)
+    int Sq_pad;
     void* out0;             // plain pointers of the outputs, for tiles that no step touches (zero fill):
     void* out1;             //   MODE 0: dq, unused;  MODE 1: dv, dk
     int Sq, Sk;
@@ -89,13 +92,24 @@ __device__ __forceinline__ void zero_rows(void* base, int64_t first_row, int row
     for (int i = tid; i < n; i += nthreads) p[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
-// delta_i = sum_d dO_id * O_id, one warp per row.
+// Per query row, one warp per row: ndelta = -sum_d dO_id * O_id and nl2 = -LSE * log2(e), written with the row
+// stride Sq_pad (padding rows: 0).  `rows` counts padded rows: B * H * Sq_pad.
 template <int D, int DTYPE>
-__global__ void attn_bwd_delta_kernel(const void* __restrict__ o, const void* __restrict__ dout, float* __restrict__ delta,
-                                      int64_t rows) {
+__global__ void attn_bwd_rows_kernel(const void* __restrict__ o, const void* __restrict__ dout, const float* __restrict__ lse,
+                                     float* __restrict__ nl2, float* __restrict__ ndelta, int Sq, int Sq_pad, int64_t rows) {
     const int lane = threadIdx.x & 31;
     const int64_t warps = static_cast<int64_t>(gridDim.x) * (blockDim.x >> 5);
-    for (int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); row < rows; row += warps) {
+    for (int64_t prow = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); prow < rows; prow += warps) {
+        const int64_t bh = prow / Sq_pad;
+        const int i = static_cast<int>(prow - bh * Sq_pad);
+        if (i >= Sq) {
+            if (lane == 0) {
+                nl2[prow] = 0.f;
+                ndelta[prow] = 0.f;
+            }
+            continue;
+        }
+        const int64_t row = bh * Sq + i;
         float acc = 0.f;
         if constexpr (D == 128) {
             const uint2 a = reinterpret_cast<const uint2*>(static_cast<const uint8_t*>(o) + row * D * 2)[lane];
@@ -131,7 +145,11 @@ __global__ void attn_bwd_delta_kernel(const void* __restrict__ o, const void* __
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (lane == 0) delta[row] = acc;
+        if (lane == 0) {
+            const float l = lse[row];
+            nl2[prow] = (l == -INFINITY) ? -INFINITY : -l * 1.4426950408889634f;
+            ndelta[prow] = -acc;
+        }
     }
 }
 
@@ -146,7 +164,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 const BwdParams prm) {
     using C = BwdCfg<D>;
     constexpr int BT = C::BT, BS = C::BS, NBOX = C::NBOX, NSTAGE = C::NSTAGE;
-    constexpr float LOG2E = 1.4426950408889634f;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -155,7 +172,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
     auto sT = [&](int stage, int w) { return smem_base + 2 * C::RES_BYTES + (2 * stage + w) * C::STR_BYTES; };  // streamed tile w
     constexpr int OST_OFF = 2 * C::RES_BYTES + 2 * NSTAGE * C::STR_BYTES;
     const uint32_t sOst = smem_base + OST_OFF;
-    float* vec = reinterpret_cast<float*>(smem_gen + OST_OFF + C::OST_BYTES);   // [group][buffer][-L log2 e | -delta][BS]
+    float* vec = reinterpret_cast<float*>(smem_gen + OST_OFF + C::OST_BYTES);   // [stage][-L log2 e | -delta][BS]
+    const uint32_t sVec = smem_base + OST_OFF + C::OST_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
     const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
     enum {
@@ -165,11 +183,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         B_PFULL = 5,      // [2] the 16-bit operands of a step are in operand region g (128 threads)
         B_OPFREE = 7,     // [2] the accumulating products of a step have read operand region g (MMA commit)
         B_ACCFINAL = 9,   // the last accumulating product has finished
-        B_GSYNC = 10,     // [2] barrier among the 128 threads of a group
-        B_ESYNC = 12,     // barrier among all 256 element-wise threads (epilogue)
-        B_TFULL = 13,     // [NSTAGE] streamed tiles loaded
-        B_TEMPTY = 13 + NSTAGE,
-        B_COUNT = 13 + 2 * NSTAGE
+        B_ESYNC = 10,     // barrier among all 256 element-wise threads (epilogue)
+        B_TFULL = 11,     // [NSTAGE] streamed tiles (and, MODE 1, their row vectors) loaded
+        B_TEMPTY = 11 + NSTAGE,
+        B_COUNT = 11 + 2 * NSTAGE
     };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
@@ -231,7 +248,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             mbar_init(bar(B_SREAD + b), 128);
             mbar_init(bar(B_PFULL + b), 128);
             mbar_init(bar(B_OPFREE + b), 1);
-            mbar_init(bar(B_GSYNC + b), 128);
         }
         mbar_init(bar(B_ACCFINAL), 1);
         mbar_init(bar(B_ESYNC), 256);
@@ -278,8 +294,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             const int st = u % NSTAGE;
             if (!mbar_wait(bar(B_TEMPTY + st), ((u / NSTAGE) & 1) ^ 1, abort_flag)) break;
             if (leader) {
-                mbar_arrive_expect_tx(bar(B_TFULL + st), 2 * C::STR_BYTES);
+                mbar_arrive_expect_tx(bar(B_TFULL + st), 2 * C::STR_BYTES + (MODE == 1 ? 2 * BS * 4 : 0));
                 const int head = step_head(u), row0 = step_sub(u) * BS;
+                if constexpr (MODE == 1) {
+                    // the prepared row vectors of the 64 streamed query rows (aligned and in bounds by construction)
+                    const int64_t off = static_cast<int64_t>(head) * prm.Sq_pad + row0;
+                    bulk_load_1d(sVec + st * 2 * BS * 4, prm.nl2 + off, BS * 4, bar(B_TFULL + st));
+                    bulk_load_1d(sVec + st * 2 * BS * 4 + BS * 4, prm.ndelta + off, BS * 4, bar(B_TFULL + st));
+                }
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx) {
                     tma_load_3d(sT(st, 0) + bx * BS * 128, &tmT0, bar(B_TFULL + st), bx * 64, row0, head);
@@ -374,7 +396,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         const int grp = warp >> 2;
         const int half = grp;                                // epilogue: which 32 of every 64 output columns
         const int r = (warp & 3) * 32 + lane;                // tensor-memory lane: query row (MODE 0) / key row (MODE 1)
-        const int gt = tid & 127;                            // thread index inside the group
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + C::S_COL + lane_off, tDP = tmem + C::DP_COL + lane_off;
         const uint32_t tOP = tmem + C::op_col(grp) + lane_off;
@@ -384,54 +405,28 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         float my_nl2 = 0.f, my_ndelta = 0.f;                 // MODE 0: minus this row's L * log2(e), minus its delta
         if constexpr (MODE == 0) {
             if (my_row < prm.Sq) {
-                const float l = prm.lse[static_cast<int64_t>(bh_res) * prm.Sq + my_row];
-                my_nl2 = (l == -INFINITY) ? -INFINITY : -l * LOG2E;   // a row without visible keys has P = 0
-                my_ndelta = -prm.delta[static_cast<int64_t>(bh_res) * prm.Sq + my_row];
+                my_nl2 = prm.nl2[static_cast<int64_t>(bh_res) * prm.Sq_pad + my_row];
+                my_ndelta = prm.ndelta[static_cast<int64_t>(bh_res) * prm.Sq_pad + my_row];
             }
         }
         bool ok = true;
-        // Barriers among element-wise threads are mbarriers with the same bounded wait as everything else (a plain
-        // bar.sync would wait forever for a thread that has left through the time-out path).
-        uint32_t gsync_phase = 0, esync_phase = 0;
-        auto group_sync = [&]() -> bool {
-            mbar_arrive(bar(B_GSYNC + grp));
-            const bool done = mbar_wait(bar(B_GSYNC + grp), gsync_phase & 1, abort_flag);
-            ++gsync_phase;
-            return done;
-        };
+        // The barrier among the element-wise threads is an mbarrier with the same bounded wait as everything else (a
+        // plain bar.sync would wait forever for a thread that has left through the time-out path).
+        uint32_t esync_phase = 0;
         auto all_sync = [&]() -> bool {
             mbar_arrive(bar(B_ESYNC));
             const bool done = mbar_wait(bar(B_ESYNC), esync_phase & 1, abort_flag);
             ++esync_phase;
             return done;
         };
-        // MODE 1: this group's 128 threads fetch one value of a step's 64 query rows each: threads 0..63 -L log2(e),
-        // 64..127 -delta.  The value for the group's NEXT step is fetched before the current step is computed, so the
-        // latency of the load is not on the path.
-        // (The loaded value is not touched until it is stored to shared memory one step later: any arithmetic on it
-        // here would make the thread wait for the load at once.)
-        auto fetch_vec = [&](int u) -> float {
-            float raw = 0.f;
-            if (u < n_steps) {
-                const int qr = step_sub(u) * BS + (gt & (BS - 1));
-                if (qr < prm.Sq) raw = (gt < BS ? prm.lse : prm.delta)[static_cast<int64_t>(step_head(u)) * prm.Sq + qr];
-            }
-            return raw;
-        };
-        float vec_next = 0.f;
-        if constexpr (MODE == 1) vec_next = fetch_vec(grp);
         for (int u = grp; u < n_steps && ok; u += 2) {
             const int t = step_sub(u);
-            // MODE 1: the step's values in one of the group's two buffers
-            float* vnl2 = vec + (grp * 2 + ((u >> 1) & 1)) * 2 * BS;
-            float* vndl = vnl2 + BS;
-            if constexpr (MODE == 1) {
-                // A thread that writes buffer x for step u has passed the barrier of step u - 2, which every thread
-                // of the group reaches only after its reads of buffer x for step u - 4.
-                // L = -inf: a row without visible keys, P = 0
-                (gt < BS ? vnl2 : vndl)[gt & (BS - 1)] = gt < BS ? (vec_next == -INFINITY ? -INFINITY : -vec_next * LOG2E) : -vec_next;
-                if (!(ok = group_sync())) break;
-                vec_next = fetch_vec(u + 2);
+            // MODE 1: -L log2(e) and -delta of the step's 64 query rows arrived with its streamed tiles (the S / dP
+            // products below were issued after that stage's "full" barrier, so the values are in place)
+            const float* vnl2 = vec + (u % NSTAGE) * 2 * BS;
+            const float* vndl = vnl2 + BS;
+            if constexpr (MODE == 1) {   // observe the bulk copies' barrier ourselves (it completed before S was issued)
+                if (!(ok = mbar_wait(bar(B_TFULL + u % NSTAGE), (u / NSTAGE) & 1, abort_flag))) break;
             }
             if (!(ok = mbar_wait(bar(B_SFULL + grp), (u >> 1) & 1, abort_flag))) break;
             tc_fence_after_sync();

@@ -111,6 +111,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap
         : "memory");
 }
 
+// Untiled bulk copy global -> shared memory (both addresses 16-byte aligned, `bytes` a multiple of 16);
+// completion is counted in bytes on `bar`.  No multicast.
+__device__ __forceinline__ void bulk_load_1d(uint32_t smem_dst, const void* gptr, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(gptr), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
 // Hint: bring `bytes` (a multiple of 16, from a 16-byte aligned address) of global memory into L2.
 __device__ __forceinline__ void bulk_prefetch_l2(const void* gptr, uint32_t bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");

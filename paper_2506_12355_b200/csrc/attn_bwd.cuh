@@ -31,10 +31,13 @@
 //
 //   warps 0-3  element-wise group of the even steps (one thread per tensor-memory lane), then the epilogue
 //   warps 4-7  element-wise group of the odd steps
-//   warp  8    MMA issuer
+//   warp  8    MMA issuer of the S and dP products
 //   warp  9    TMA producer
-//   warps 10-11 idle (they complete the third warpgroup so that registers can be re-balanced: an element-wise
-//              thread holds a whole S and dP row of a step, 128 registers, while it computes)
+//   warp  10   MMA issuer of the accumulating products (two issuers: a tcgen05.mma issue holds its thread while the
+//              tensor core's queue is full, and a single issuer's barrier polls between the two kinds of product
+//              left the queue running empty ~30 % of the time)
+//   warp  11   idle (it completes the third warpgroup so that registers can be re-balanced: an element-wise thread
+//              holds a whole S and dP row of a step, 128 registers, while it computes)
 //
 // Every wait is bounded (see sm100_ptx.cuh); a timed-out wait ends the CTA through the normal exit.
 #pragma once
@@ -309,8 +312,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 }
             }
         }
-      } else if (warp == 8) {
-        // =========================== MMA issuer ===========================
+      } else if (warp == 8 || warp == 10) {
+        // =========================== MMA issuers ===========================
         const bool leader = elect_one();
         constexpr uint32_t IDESC_S = make_idesc_f16(BT, BS, DTYPE, 0, 0);    // both operands K-major (contraction over D)
         constexpr uint32_t IDESC_ACC = make_idesc_f16(BT, D, DTYPE, 0, 1);   // A from tensor memory, B MN-major (N = D)
@@ -333,11 +336,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 mma_commit(bar(B_SFULL + (u & 1)));
             }
         };
-        bool ok = mbar_wait(bar(B_RFULL), 0, abort_flag) && mbar_wait(bar(B_TFULL), 0, abort_flag);
-        if (ok) {
-            tc_fence_after_sync();
-            issue_s(0);
-        }
         // accumulating products of step v (contraction step kk, 16 values = 8 columns, starts at column 8 kk of its
         // operand); afterwards its streamed tiles and its operand region are free
         auto issue_acc = [&](int v) {
@@ -368,20 +366,25 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 if (v + 1 == n_steps) mma_commit(bar(B_ACCFINAL));
             }
         };
-        // Iteration u: S and dP of step u + 1 as soon as step u's are in its group's registers, then the
-        // accumulating products of step u - 1, whose operands have had a whole step to get ready: the tensor core
-        // does not wait for the element-wise warps unless they fall a full step behind.
-        for (int u = 0; u <= n_steps && ok; ++u) {
-            if (u < n_steps) {
-                if (!(ok = mbar_wait(bar(B_SREAD + (u & 1)), (u >> 1) & 1, abort_flag))) break;
-                if (u + 1 < n_steps) {
-                    if (!(ok = mbar_wait(bar(B_TFULL + (u + 1) % NSTAGE), ((u + 1) / NSTAGE) & 1, abort_flag))) break;
-                    tc_fence_after_sync();
-                    issue_s(u + 1);
-                }
+        if (warp == 8) {
+            // S and dP of step u + 1 as soon as step u's are in its group's registers
+            bool ok = mbar_wait(bar(B_RFULL), 0, abort_flag) && mbar_wait(bar(B_TFULL), 0, abort_flag);
+            if (ok) {
+                tc_fence_after_sync();
+                issue_s(0);
             }
-            if (u >= 1) {
-                const int v = u - 1;
+            for (int u = 0; u + 1 < n_steps && ok; ++u) {
+                if (!(ok = mbar_wait(bar(B_SREAD + (u & 1)), (u >> 1) & 1, abort_flag))) break;
+                if (!(ok = mbar_wait(bar(B_TFULL + (u + 1) % NSTAGE), ((u + 1) / NSTAGE) & 1, abort_flag))) break;
+                tc_fence_after_sync();
+                issue_s(u + 1);
+            }
+        } else {
+            // the accumulating products of step v as soon as its operands are in tensor memory (its streamed tiles
+            // were loaded before its S and dP; this warp observes that barrier itself all the same)
+            bool ok = true;
+            for (int v = 0; v < n_steps && ok; ++v) {
+                if (!(ok = mbar_wait(bar(B_TFULL + v % NSTAGE), (v / NSTAGE) & 1, abort_flag))) break;
                 if (!(ok = mbar_wait(bar(B_PFULL + (v & 1)), (v >> 1) & 1, abort_flag))) break;
                 tc_fence_after_sync();
                 issue_acc(v);

@@ -44,13 +44,14 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 // consecutive output elements (16 bytes).  `src` says where shard r's partial result lies: src.lse(r, row)
 // and src.o(r, row, seg) (seg: 16-byte piece of the row).  o: [rows_total, D]; lse: [rows_total].
 template <int DTYPE, int BATCH, class Src>
-__device__ __forceinline__ void merge_rows(const Src& src, int n_parts, uint4* __restrict__ o, float* __restrict__ lse,
+__device__ __forceinline__ void merge_rows(const Src src, int n_parts, uint4* __restrict__ o, float* __restrict__ lse,
                                            int64_t row0, int64_t n_rows, int segs_per_row) {
     const int64_t total = n_rows * segs_per_row;
     for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
          idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-        const int64_t row = row0 + idx / segs_per_row;
-        const int seg = static_cast<int>(idx % segs_per_row);
+        const int64_t local_row = idx / segs_per_row;
+        const int seg = static_cast<int>(idx - local_row * segs_per_row);
+        const int64_t row = row0 + local_row;
         float mx = -INFINITY;
         for (int r = 0; r < n_parts; ++r) mx = fmaxf(mx, src.lse(r, row));
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -91,11 +92,11 @@ __device__ __forceinline__ void merge_rows(const Src& src, int n_parts, uint4* _
 // Shards stacked in one allocation of this GPU: o_parts [n_parts, rows, D] 16-bit, lse_parts [n_parts, rows] fp32
 // (read through the read-only path).
 struct StackedParts {
-    const uint4* o_parts;
-    const float* lse_parts;
+    const uint4* __restrict__ o_parts;
+    const float* __restrict__ lse_parts;
     int64_t rows;
     int segs_per_row;
-    __device__ __forceinline__ float lse(int r, int64_t row) const { return __ldg(lse_parts + r * rows + row); }
+    __device__ __forceinline__ float lse(int r, int64_t row) const { return lse_parts[r * rows + row]; }
     __device__ __forceinline__ uint4 o(int r, int64_t row, int seg) const {
         return __ldg(o_parts + (r * rows + row) * segs_per_row + seg);
     }

@@ -69,6 +69,8 @@ struct BwdCfg {
     static constexpr int S_COL = 0, DP_COL = 64;
     __host__ __device__ static constexpr int op_col(int g) { return 128 + 64 * g; }
     static constexpr int ACC0_COL = 256, ACC1_COL = 256 + D;
+    // the resident tiles as 16-bit A operands in tensor memory (where the columns allow it): tile w in D / 2 columns
+    __host__ __device__ static constexpr int rt_col(int w) { return 512 - D + w * (D / 2); }
     static constexpr int TMEM_COLS = 512;
     static_assert(D == 64 || D == 128, "head dims 64 and 128");
 };
@@ -167,6 +169,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 const BwdParams prm) {
     using C = BwdCfg<D>;
     constexpr int BT = C::BT, BS = C::BS, NBOX = C::NBOX, NSTAGE = C::NSTAGE;
+    // The S and dP products read their resident operand (A) from tensor memory wherever 512 columns allow it: with both
+    // operands in shared memory an M 128 x N 64 instruction is paced by shared-memory bandwidth (6 KB per 32 tensor
+    // cycles), with A in tensor memory it reads 2 KB.  The dK/dV pass at D = 128 has no columns left for it.
+    constexpr bool A_TMEM = !(MODE == 1 && D == 128);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -187,9 +193,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         B_OPFREE = 7,     // [2] the accumulating products of a step have read operand region g (MMA commit)
         B_ACCFINAL = 9,   // the last accumulating product has finished
         B_ESYNC = 10,     // barrier among all 256 element-wise threads (epilogue)
-        B_TFULL = 11,     // [NSTAGE] streamed tiles (and, MODE 1, their row vectors) loaded
-        B_TEMPTY = 11 + NSTAGE,
-        B_COUNT = 11 + 2 * NSTAGE
+        B_RTMEM = 11,     // the resident tiles have been copied into tensor memory (256 element-wise threads)
+        B_TFULL = 12,     // [NSTAGE] streamed tiles (and, MODE 1, their row vectors) loaded
+        B_TEMPTY = 12 + NSTAGE,
+        B_COUNT = 12 + 2 * NSTAGE
     };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
@@ -254,6 +261,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         }
         mbar_init(bar(B_ACCFINAL), 1);
         mbar_init(bar(B_ESYNC), 256);
+        mbar_init(bar(B_RTMEM), 256);
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(bar(B_TFULL + s), 1);
             mbar_init(bar(B_TEMPTY + s), 1);
@@ -330,7 +338,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                     for (int kk = 0; kk < D / 16; ++kk) {
                         const uint32_t offa = ((kk >> 2) * BT * 128 + (kk & 3) * 32) >> 4;
                         const uint32_t offb = ((kk >> 2) * BS * 128 + (kk & 3) * 32) >> 4;
-                        mma_f16_ss_lohi(tmem + (w == 0 ? C::S_COL : C::DP_COL), r_lo[w] + offa, b0 + offb, DESC_HI, IDESC_S, kk > 0);
+                        if constexpr (A_TMEM)
+                            mma_f16_ts_lohi(tmem + (w == 0 ? C::S_COL : C::DP_COL), tmem + C::rt_col(w) + kk * 8, b0 + offb, DESC_HI, IDESC_S, kk > 0);
+                        else
+                            mma_f16_ss_lohi(tmem + (w == 0 ? C::S_COL : C::DP_COL), r_lo[w] + offa, b0 + offb, DESC_HI, IDESC_S, kk > 0);
                     }
                 }
                 mma_commit(bar(B_SFULL + (u & 1)));
@@ -368,7 +379,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         };
         if (warp == 8) {
             // S and dP of step u + 1 as soon as step u's are in its group's registers
-            bool ok = mbar_wait(bar(B_RFULL), 0, abort_flag) && mbar_wait(bar(B_TFULL), 0, abort_flag);
+            bool ok = mbar_wait(bar(A_TMEM ? B_RTMEM : B_RFULL), 0, abort_flag) && mbar_wait(bar(B_TFULL), 0, abort_flag);
             if (ok) {
                 tc_fence_after_sync();
                 issue_s(0);
@@ -413,6 +424,26 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             }
         }
         bool ok = true;
+        if constexpr (A_TMEM) {
+            // Group g copies resident tile g from shared memory (rows of 128 bytes per 64-column box, 16-byte chunks
+            // swizzled by row) into tensor memory: lane = row, two 16-bit values per column in memory order.
+            if ((ok = mbar_wait(bar(B_RFULL), 0, abort_flag))) {
+                const uint32_t src = sR(grp) + r * 128;
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx) {
+                    uint32_t w[32];
+#pragma unroll
+                    for (int g8 = 0; g8 < 8; ++g8)
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(w[g8 * 4 + 0]), "=r"(w[g8 * 4 + 1]), "=r"(w[g8 * 4 + 2]), "=r"(w[g8 * 4 + 3])
+                                     : "r"(src + bx * BT * 128 + ((g8 ^ (r & 7)) << 4)) : "memory");
+                    tmem_st_32x32b_x32(tmem + C::rt_col(grp) + bx * 32 + lane_off, w);
+                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(bar(B_RTMEM));
+            }
+        }
         // The barrier among the element-wise threads is an mbarrier with the same bounded wait as everything else (a
         // plain bar.sync would wait forever for a thread that has left through the time-out path).
         uint32_t esync_phase = 0;

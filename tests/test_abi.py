@@ -107,6 +107,30 @@ def test_fp8_entry_validation(lib):
         assert f8() in (7, 8)                   # valid arguments reach the device check
 
 
+def test_bwd_entry_validation(lib):
+    ws_bytes = lib.attn_bwd_workspace_bytes
+    ws_bytes.restype = ctypes.c_size_t
+    # two fp32 row vectors, rows padded to a multiple of 64 per head, each 256-byte aligned
+    assert ws_bytes(2, 3, 100) == 2 * ((2 * 3 * 128 * 4 + 255) // 256 * 256)
+    assert ws_bytes(1, 1, 64) == 2 * 256 and ws_bytes(-1, 1, 1) == 0
+
+    def bwd(q=0x1000, k=0x2000, v=0x3000, o=0x4000, lse=0x5000, dout=0x6000, dq=0x7000, dk=0x8000, dv=0x9000, B=1, H=4,
+            Hkv=2, Sq=128, Sk=256, D=128, scale=0.1, causal=1, dtype=1, ws=0x10000, ws_n=1 << 20):
+        return lib.attn_bwd(q, k, v, o, lse, dout, dq, dk, dv, B, H, Hkv, Sq, Sk, D, scale, causal, dtype, ws, ws_n, None)
+    for name in ("q", "k", "v", "o", "lse", "dout", "dq", "dk", "dv"):
+        assert bwd(**{name: None}) == 1, name
+    assert bwd(B=-1) == 2 and bwd(H=4, Hkv=3) == 2
+    for d in (256, 96, 0):
+        assert bwd(D=d) == 3                    # backward kernels: head dims 64 and 128
+    assert bwd(dtype=2) == 4
+    assert bwd(dout=0x6008) == 5 and bwd(dk=0x8004) == 5
+    assert bwd(scale=float("nan")) == 6 and bwd(scale=-1.0) == 6
+    assert bwd(ws=None) == 10 and bwd(ws=0x10010) == 10 and bwd(ws_n=100) == 10
+    assert bwd(Sq=0, Sk=0) == 0                 # nothing to do
+    if no_device():
+        assert bwd() in (7, 8)                  # valid arguments reach the device check
+
+
 def test_splitkv_entry_validation(lib):
     lib.attn_fwd_splitkv_workspace_bytes.restype = __import__("ctypes").c_size_t
     assert lib.attn_fwd_splitkv_workspace_bytes(1, 4, 3, 128, 6) == (6 * 12 * 128 * 2 + 255) // 256 * 256 + (6 * 12 * 4 + 255) // 256 * 256

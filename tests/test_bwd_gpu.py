@@ -108,6 +108,44 @@ def test_bwd_keys_that_no_query_sees_and_sharp_scale():
     run_case(1, 2, 1, 256, 256, 128, inputs.DTYPE_FP16, False, seed=8201, scale=1.0)
 
 
+def test_bwd_in_a_cuda_graph_and_on_two_streams():
+    # the three launches of a call captured once and replayed; two calls in flight on two streams
+    dev = torch.device("cuda:0")
+    cases = []
+    for i, (D, causal) in enumerate(((128, True), (64, False))):
+        q, k, v = (t.to(dev) for t in inputs.make_qkv(2, 4, 700, 700, D, inputs.DTYPE_BF16, seed=8400 + i))
+        dout = inputs.randn16((2, 4, 700, D), 8410 + i, inputs.DTYPE_BF16).to(dev)
+        o, lse = api.attn_fwd(q, k, v, D ** -0.5, causal)
+        ref = api.attn_bwd(q, k, v, o, lse, dout, D ** -0.5, causal)
+        cases.append((q, k, v, o, lse, dout, D ** -0.5, causal, ref))
+    torch.cuda.synchronize()
+    q, k, v, o, lse, dout, scale, causal, ref = cases[0]
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    ws = torch.empty(api.attn_bwd_workspace_bytes(2, 4, 700), dtype=torch.uint8, device=dev)
+    st = torch.cuda.Stream(device=dev)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            api.attn_bwd(q, k, v, o, lse, dout, scale, causal, dq=dq, dk=dk, dv=dv, workspace=ws, stream=st)
+    for _ in range(3):
+        dq.zero_(); dk.zero_(); dv.zero_()
+        g.replay()
+    torch.cuda.synchronize()
+    for got, want in zip((dq, dk, dv), ref):
+        assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    streams = [torch.cuda.Stream(device=dev) for _ in cases]
+    outs = []
+    for _ in range(4):
+        for c, s_ in zip(cases, streams):
+            with torch.cuda.stream(s_):
+                outs.append((api.attn_bwd(*c[:8], stream=s_), c[8]))
+    torch.cuda.synchronize()
+    assert api.attn_last_device_status() == 0
+    for got, want in outs:
+        for a, b in zip(got, want):
+            assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
 def test_bwd_is_bitwise_deterministic_and_validates():
     dev = torch.device("cuda:0")
     q, k, v = (t.to(dev) for t in inputs.make_qkv(2, 4, 640, 640, 128, inputs.DTYPE_BF16, seed=8300))

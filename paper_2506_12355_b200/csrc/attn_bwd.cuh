@@ -58,9 +58,9 @@ struct BwdCfg {
     static constexpr int RES_BYTES = BT * D * 2;            // one resident tile
     static constexpr int STR_BYTES = BS * D * 2;            // one streamed tile
     static constexpr int NSTAGE = D == 128 ? 4 : 6;           // ring stages, each holds the two streamed tiles
-    static constexpr int OST_BYTES = BT * 128;              // epilogue staging: 128 rows x 64 columns
+    static constexpr int OST_BYTES = BT * 128;              // one epilogue staging tile: 128 rows x 64 columns (placed in the ring)
     static constexpr int VEC_BYTES = NSTAGE * 2 * BS * 4;   // MODE 1: -L log2(e) and -delta of a stage's 64 streamed query rows
-    static constexpr int TILE_BYTES = 2 * RES_BYTES + NSTAGE * 2 * STR_BYTES + OST_BYTES + VEC_BYTES;
+    static constexpr int TILE_BYTES = 2 * RES_BYTES + NSTAGE * 2 * STR_BYTES + VEC_BYTES;
     static constexpr int MISC_BYTES = 256;
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
     static constexpr int THREADS = 384;
@@ -179,10 +179,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     auto sR = [&](int w) { return smem_base + w * C::RES_BYTES; };                                          // resident tile w
     auto sT = [&](int stage, int w) { return smem_base + 2 * C::RES_BYTES + (2 * stage + w) * C::STR_BYTES; };  // streamed tile w
-    constexpr int OST_OFF = 2 * C::RES_BYTES + 2 * NSTAGE * C::STR_BYTES;
-    const uint32_t sOst = smem_base + OST_OFF;
-    float* vec = reinterpret_cast<float*>(smem_gen + OST_OFF + C::OST_BYTES);   // [stage][-L log2 e | -delta][BS]
-    const uint32_t sVec = smem_base + OST_OFF + C::OST_BYTES;
+    constexpr int VEC_OFF = 2 * C::RES_BYTES + 2 * NSTAGE * C::STR_BYTES;
+    float* vec = reinterpret_cast<float*>(smem_gen + VEC_OFF);   // [stage][-L log2 e | -delta][BS]
+    const uint32_t sVec = smem_base + VEC_OFF;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
     const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
     enum {
@@ -543,42 +542,49 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             mbar_arrive(bar(B_PFULL + grp));
         }
 
-        // ---- epilogue: accumulators -> 16-bit -> swizzled staging tile -> TMA store (rows beyond the tensor clipped) ----
+        // ---- epilogue: accumulators -> 16-bit -> swizzled staging tiles -> TMA stores (rows beyond the tensor clipped).
+        // The ring of streamed tiles is idle by now (every load has been consumed, every product that read it has
+        // finished), so each 64-column piece of the output gets a staging tile of its own there: one barrier, then
+        // all stores at once. ----
         if (ok && (ok = mbar_wait(bar(B_ACCFINAL), 0, abort_flag))) {
             tc_fence_after_sync();
             constexpr int NACC = MODE == 0 ? 1 : 2;
+            static_assert(NACC * (D / 64) * C::OST_BYTES <= NSTAGE * 2 * C::STR_BYTES, "staging tiles must fit the ring");
+            const uint32_t stage0 = sT(0, 0);
 #pragma unroll
-            for (int a = 0; a < NACC && ok; ++a) {
+            for (int a = 0; a < NACC; ++a) {
                 // MODE 0: dQ (x scale).  MODE 1: accumulator 0 = dV, accumulator 1 = dK (x scale).
                 const float f = (MODE == 0 || a == 1) ? prm.scale : 1.f;
                 const uint32_t tA = tmem + (a == 0 ? C::ACC0_COL : C::ACC1_COL) + lane_off;
 #pragma unroll
-                for (int h = 0; h < D / 64 && ok; ++h) {
-                    // 64 output columns per round; this thread converts the 32 of its column half
+                for (int h = 0; h < D / 64; ++h) {
+                    // 64 output columns per staging tile; this thread converts the 32 of its column half
                     uint32_t acc[32];
                     tmem_ld_32x32b_x32(tA + h * 64 + 32 * half, acc);
                     tmem_ld_wait();
-                    if (tid == 0) tma_store_wait_read<0>();        // the previous store has read the staging tile
-                    if (!(ok = all_sync())) break;
+                    const uint32_t ost = stage0 + (a * (D / 64) + h) * C::OST_BYTES;
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         const uint32_t w0 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 0]) * f, __uint_as_float(acc[g * 8 + 1]) * f);
                         const uint32_t w1 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 2]) * f, __uint_as_float(acc[g * 8 + 3]) * f);
                         const uint32_t w2 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 4]) * f, __uint_as_float(acc[g * 8 + 5]) * f);
                         const uint32_t w3 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 6]) * f, __uint_as_float(acc[g * 8 + 7]) * f);
-                        const uint32_t dst = sOst + r * 128 + (((4 * half + g) ^ (r & 7)) << 4);   // 128-byte swizzle
+                        const uint32_t dst = ost + r * 128 + (((4 * half + g) ^ (r & 7)) << 4);   // 128-byte swizzle
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
-                    }
-                    fence_proxy_async_smem();
-                    if (!(ok = all_sync())) break;
-                    if (tid == 0) {
-                        tma_store_3d(a == 0 ? &tmOut0 : &tmOut1, sOst, h * 64, tile * BT, bh_res);
-                        tma_store_commit();
                     }
                 }
             }
+            fence_proxy_async_smem();
+            if ((ok = all_sync()) && tid == 0) {
+#pragma unroll
+                for (int a = 0; a < NACC; ++a)
+#pragma unroll
+                    for (int h = 0; h < D / 64; ++h)
+                        tma_store_3d(a == 0 ? &tmOut0 : &tmOut1, stage0 + (a * (D / 64) + h) * C::OST_BYTES, h * 64, tile * BT, bh_res);
+                tma_store_commit();
+            }
         }
-        if (tid == 0) tma_store_wait_all<0>();   // the staging tile must outlive its last store
+        if (tid == 0) tma_store_wait_all<0>();   // the staging tiles must outlive their stores
     }
 
     // ---- teardown (also reached after a timed-out wait) ----

@@ -11,17 +11,19 @@
 // tile resident, the other side streamed through a TMA ring, the S x S matrices never leave the SM):
 //
 //   MODE 0 (dQ):      CTA = one 128-row Q tile; Q_i, dO_i resident; K_j, V_j streamed.
-//                     S = Q_i K_j^T and dP = dO_i V_j^T (both operands in shared memory) -> tensor memory;
-//                     one thread per query row turns them into dS (16-bit, written over S);
-//                     dQ += dS K_j with dS read from tensor memory, K_j as the MN-major operand.
+//                     S = Q_i K_j^T and dP = dO_i V_j^T -> tensor memory; one thread per query row turns them
+//                     into dS (16-bit, tensor memory); dQ += dS K_j with K_j as the MN-major operand.
 //   MODE 1 (dK, dV):  CTA = one 128-key K/V tile; K_j, V_j resident; Q_i, dO_i streamed (all query heads of
 //                     the K/V head's group).  The TRANSPOSED tiles S^T = K_j Q_i^T and dP^T = V_j dO_i^T are
 //                     computed, so that P^T and dS^T land in tensor memory with keys on the lanes, which is
 //                     the A operand that dV += P^T dO_i and dK += dS^T Q_i need; one thread per key row, the
-//                     per-query L and delta come from shared memory.
+//                     per-query -L log2(e) and -delta arrive in shared memory with the streamed tiles.
 //
 // Recomputing S and dP in both passes costs 7 tile products instead of 5 but needs no atomics and no
-// cross-CTA reduction, so the results are deterministic.  delta is computed by a small kernel first.
+// cross-CTA reduction, so the results are deterministic.  A small kernel first prepares the two row vectors
+// (-L log2(e) and -delta) in the caller's workspace.  Where the 512 tensor-memory columns allow it (everywhere but
+// MODE 1 at D = 128) the resident tiles are copied into tensor memory once and are the A operand of the S / dP
+// products from there; with both operands in shared memory those products are paced by shared-memory bandwidth.
 //
 // The streamed side advances 64 rows per step.  The fp32 S / dP tiles of a step (128 lanes x 64 columns each)
 // have ONE place in tensor memory, which an element-wise group frees as soon as it has the tile in registers;
@@ -29,8 +31,8 @@
 // the tensor core already produces S and dP of the next step for the other group, and the accumulating products
 // of a step run whenever its operands are ready.
 //
-//   warps 0-3  element-wise group of the even steps (one thread per tensor-memory lane), then the epilogue
-//   warps 4-7  element-wise group of the odd steps
+//   warps 0-3  element-wise group of the even steps (one thread per tensor-memory lane); both groups then run the
+//   warps 4-7  element-wise group of the odd steps                                          epilogue together
 //   warp  8    MMA issuer of the S and dP products
 //   warp  9    TMA producer
 //   warp  10   MMA issuer of the accumulating products (two issuers: a tcgen05.mma issue holds its thread while the

@@ -101,6 +101,18 @@ def test_bwd_many_tiles(D, dtype, causal):
         D, dtype, causal, *w["dq"], *w["dk"], *w["dv"]))
 
 
+def test_bwd_long_ragged_sequence_and_no_queries():
+    # 65 x 65 tiles per head with ragged tails on both axes (Sq != Sk), grouped heads; then the Sq = 0 corner
+    run_case(1, 16, 8, 4133, 4101, 128, inputs.DTYPE_BF16, True, seed=8150)
+    dev = torch.device("cuda:0")
+    k = torch.randn(1, 2, 300, 64, device=dev).to(torch.float16)
+    q0 = torch.empty(1, 2, 0, 64, dtype=torch.float16, device=dev)
+    dq, dk, dv = api.attn_bwd(q0, k, k, q0, torch.empty(1, 2, 0, device=dev), q0, 0.1, False,
+                              dk=torch.full_like(k, float("nan")), dv=torch.full_like(k, float("nan")))
+    torch.cuda.synchronize()
+    assert dq.numel() == 0 and float(dk.abs().max()) == 0.0 and float(dv.abs().max()) == 0.0
+
+
 def test_bwd_keys_that_no_query_sees_and_sharp_scale():
     # Sk > Sq under the causal mask: keys beyond the last query get zero gradients (tiles with and without steps);
     # a large scale makes the softmax rows sharply peaked

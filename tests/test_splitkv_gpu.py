@@ -95,3 +95,16 @@ def test_splitkv_in_a_cuda_graph():
     torch.cuda.synchronize()
     assert api.attn_last_device_status() == 0
     assert torch.equal(o.view(torch.int16), ref_o.view(torch.int16)) and torch.equal(lse, ref_l)
+
+
+def test_bench_kv_sharded_check_single_rank():
+    # the check that bench.py adds to its line at N > 1, driven here with one rank (no process group: the single
+    # shard is merged alone): its input recipe, both exchange branches and the oracle comparison run end to end
+    import os
+    import sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    res = bench.kv_sharded_check(api, torch.device("cuda:0"), 0, 1)
+    for exchange in ("nccl", "peer"):
+        assert isinstance(res[exchange], dict), res[exchange]
+        assert res[exchange]["max_abs_o"] <= 2e-2 and res[exchange]["max_abs_lse"] <= 1e-3

@@ -101,6 +101,33 @@ def test_bwd_many_tiles(D, dtype, causal):
         D, dtype, causal, *w["dq"], *w["dk"], *w["dv"]))
 
 
+@pytest.mark.parametrize("name,heads", [("C3", None), ("C5", (0, 31))])
+def test_bwd_at_the_benchmark_shapes(name, heads):
+    # the two shapes whose backward pass bench.py times, in the same launch configuration: C3 against the oracle's
+    # gradients on every head, C5 (3.3 TFLOP of oracle work for all heads) on its first and its last head
+    cfg = inputs.CONFIGS[name]
+    dev = torch.device("cuda:0")
+    q, k, v = inputs.make_config_inputs(cfg)
+    dout = inputs.randn16((cfg.B, cfg.H, cfg.Sq, cfg.D), inputs.BASE_SEED + 1000 * cfg.index + 3, cfg.dtype)
+    qd, kd, vd, dd = q.to(dev), k.to(dev), v.to(dev), dout.to(dev)
+    o, lse = api.attn_fwd(qd, kd, vd, cfg.scale, cfg.causal)
+    got = [t.cpu() for t in api.attn_bwd(qd, kd, vd, o, lse, dd, cfg.scale, cfg.causal)]
+    assert api.attn_last_device_status() == 0
+    flat = lambda t: t.reshape(cfg.B * cfg.H, cfg.Sq, cfg.D)
+    sel = list(range(cfg.B * cfg.H)) if heads is None else list(heads)
+    pick = lambda t: flat(t)[sel].unsqueeze(0).contiguous()       # the chosen (batch, head) slices as one batch
+    ref = orc.attention_bwd(*(orc.widen(inputs.bits(pick(t)), cfg.dtype) for t in (q, k, v, dout)), cfg.scale, cfg.causal)
+    for nm, g, want in zip(("dq", "dk", "dv"), got, ref):
+        gsel = pick(g).to(torch.float64).numpy()
+        assert not np.isnan(gsel).any() and bool(torch.isfinite(g.float()).all())
+        err = np.abs(gsel - want)
+        rms = math.sqrt(float((want ** 2).mean()))
+        bound = ATOL[cfg.dtype] * max(1.0, rms) + RTOL[cfg.dtype] * np.abs(want)
+        print("%s %s: max|err| %.3g, rms err / rms %.3g (rms %.3g)" % (name, nm, err.max(), math.sqrt(float((err ** 2).mean())) / rms, rms))
+        assert np.all(err <= bound), "%s %s: max |err| = %g" % (name, nm, err.max())
+        assert math.sqrt(float((err ** 2).mean())) <= 2.0 ** -6 * rms      # bf16: small against the gradient itself
+
+
 def test_bwd_long_ragged_sequence_and_no_queries():
     # 65 x 65 tiles per head with ragged tails on both axes (Sq != Sk), grouped heads; then the Sq = 0 corner
     run_case(1, 16, 8, 4133, 4101, 128, inputs.DTYPE_BF16, True, seed=8150)

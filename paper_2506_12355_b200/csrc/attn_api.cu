@@ -851,6 +851,9 @@ int attn_bwd(const void* q, const void* k, const void* v, const void* o, const f
     prm.status = device_status_ptr();
     if (!prm.status) return ATTN_ERR_CUDA;
     // resident tiles and outputs move in boxes of 128 rows, streamed tiles in boxes of 64 rows
+    DeviceInfo di;
+    if (device_info(&di) != ATTN_OK) return ATTN_ERR_CUDA;
+    const int sms = di.sm_count;   // persistent grids: one CTA per SM
     CUtensorMap mq, mk, mv, mdo, mq64, mk64, mv64, mdo64, mdq, mdk, mdv;
     if (!make_map(&mq, q, dtype, BH, Sq, D, 128) || !make_map(&mdo, dout, dtype, BH, Sq, D, 128) ||
         !make_map(&mq64, q, dtype, BH, Sq, D, 64) || !make_map(&mdo64, dout, dtype, BH, Sq, D, 64) ||
@@ -861,11 +864,12 @@ int attn_bwd(const void* q, const void* k, const void* v, const void* o, const f
         return ATTN_ERR_CUDA;
 #define ATTN_BWD_CASE(DD, TT)                                                                                              \
     if (D == DD && dtype == TT) {                                                                                          \
-        using C = attn_grad::BwdCfg<DD>;                                                                                    \
+        using CQ = attn_grad::BwdCfg<DD, 0>;                                                                                \
+        using CKV = attn_grad::BwdCfg<DD, 1>;                                                                               \
         auto kq = attn_grad::attn_bwd_kernel<DD, TT, 0>;                                                                    \
         auto kkv = attn_grad::attn_bwd_kernel<DD, TT, 1>;                                                                   \
-        if (!allow_dynamic_smem(reinterpret_cast<const void*>(kq), C::SMEM_BYTES) ||                                       \
-            !allow_dynamic_smem(reinterpret_cast<const void*>(kkv), C::SMEM_BYTES))                                        \
+        if (!allow_dynamic_smem(reinterpret_cast<const void*>(kq), CQ::SMEM_BYTES) ||                                      \
+            !allow_dynamic_smem(reinterpret_cast<const void*>(kkv), CKV::SMEM_BYTES))                                      \
             return ATTN_ERR_CUDA;                                                                                          \
         const int64_t rows = BH * sq_pad;                                                                                  \
         int64_t blocks = (rows + 7) / 8;                                                                                   \
@@ -874,10 +878,14 @@ int attn_bwd(const void* q, const void* k, const void* v, const void* o, const f
                                                                                               prm.Sq_pad, rows);          \
         prm.out0 = dq;                                                                                                     \
         prm.out1 = nullptr;                                                                                                \
-        kq<<<static_cast<unsigned>(n_qtiles * BH), C::THREADS, C::SMEM_BYTES, st>>>(mq, mdo, mk64, mv64, mdq, mdq, prm);       \
+        prm.n_tiles_total = static_cast<int>(n_qtiles * BH);                                                               \
+        kq<<<static_cast<unsigned>(prm.n_tiles_total < sms ? prm.n_tiles_total : sms), CQ::THREADS, CQ::SMEM_BYTES, st>>>(  \
+            mq, mdo, mk64, mv64, mdq, mdq, prm);                                                                           \
         prm.out0 = dv;                                                                                                     \
         prm.out1 = dk;                                                                                                     \
-        kkv<<<static_cast<unsigned>(n_ktiles * BHkv), C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mq64, mdo64, mdv, mdk, prm);    \
+        prm.n_tiles_total = static_cast<int>(n_ktiles * BHkv);                                                             \
+        kkv<<<static_cast<unsigned>(prm.n_tiles_total < sms ? prm.n_tiles_total : sms), CKV::THREADS, CKV::SMEM_BYTES, st>>>( \
+            mk, mv, mq64, mdo64, mdv, mdk, prm);                                                                           \
         return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;                                                \
     }
     ATTN_BWD_CASE(64, 0)

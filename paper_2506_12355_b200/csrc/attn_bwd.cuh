@@ -41,6 +41,12 @@
 //   warp  11   idle (it completes the third warpgroup so that registers can be re-balanced: an element-wise thread
 //              holds a whole S and dP row of a step, 128 registers, while it computes)
 //
+// Persistent grid: one CTA per SM walks its tiles (tile index = block index + k * grid size; tiles of one head are
+// neighbours, causal tiles heaviest first, so the round-robin hands every CTA a similar mix).  Barriers, tensor memory
+// and the streamed ring live across tiles: the producer loads the next tile's resident tiles while the current tile
+// still computes, the element-wise warps copy them into tensor memory right after their last step, and the S / dP
+// products of the next tile's first step run while the accumulators of the current tile drain.
+//
 // Every wait is bounded (see sm100_ptx.cuh); a timed-out wait ends the CTA through the normal exit.
 #pragma once
 #include <type_traits>
@@ -52,19 +58,23 @@ namespace attn_grad {
 using namespace sm100;
 using attn_tc::finish_cta;
 
-template <int D>
+template <int D, int MODE>
 struct BwdCfg {
     static constexpr int BT = 128;                          // rows of the resident tiles = tensor-memory lanes
     static constexpr int BS = 64;                           // rows of the streamed tiles = columns of one step
     static constexpr int NBOX = D / 64;                     // 128-byte wide TMA boxes per tile row
     static constexpr int RES_BYTES = BT * D * 2;            // one resident tile
     static constexpr int STR_BYTES = BS * D * 2;            // one streamed tile
-    static constexpr int NSTAGE = D == 128 ? 4 : 6;           // ring stages, each holds the two streamed tiles
-    static constexpr int OST_BYTES = BT * 128;              // one epilogue staging tile: 128 rows x 64 columns (placed in the ring)
-    static constexpr int VEC_BYTES = NSTAGE * 2 * BS * 4;   // MODE 1: -L log2(e) and -delta of a stage's 64 streamed query rows
-    static constexpr int TILE_BYTES = 2 * RES_BYTES + NSTAGE * 2 * STR_BYTES + VEC_BYTES;
+    static constexpr int NACC = MODE == 0 ? 1 : 2;          // accumulators: dQ, or dV and dK
+    static constexpr int OST_BYTES = BT * 128;              // one epilogue staging tile: 128 rows x 64 columns
+    static constexpr int STG_BYTES = NACC * (D / 64) * OST_BYTES;   // a staging tile for every 64-column piece of the output
+    // ring stages, each holds the two streamed tiles (three where the staging tiles leave no room for four)
+    static constexpr int NSTAGE = D == 64 ? 6 : (MODE == 0 ? 4 : 3);
+    static constexpr int VEC_BYTES = MODE == 1 ? NSTAGE * 2 * BS * 4 : 0;   // -L log2(e) and -delta of a stage's 64 query rows
+    static constexpr int TILE_BYTES = 2 * RES_BYTES + NSTAGE * 2 * STR_BYTES + STG_BYTES + VEC_BYTES;
     static constexpr int MISC_BYTES = 256;
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
+    static_assert(SMEM_BYTES <= 232448, "shared memory budget");
     static constexpr int THREADS = 384;
     // tensor memory: fp32 S in columns 0 .. 63, fp32 dP in 64 .. 127; operand region g (steps u = g mod 2) at
     // 128 + 64 g: first 16-bit operand (dS in MODE 0, P^T in MODE 1) in its columns 0 .. 31, second (dS^T) in 32 .. 63
@@ -90,6 +100,7 @@ struct BwdParams {
     int causal;
     int H, Hkv;
     int n_qtiles, n_ktiles; // 128-row tiles of the query and of the key axis
+    int n_tiles_total;      // tiles of this pass over all heads: the persistent CTAs walk them round-robin
     int* status;
 };
 
@@ -160,6 +171,14 @@ __global__ void attn_bwd_rows_kernel(const void* __restrict__ o, const void* __r
     }
 }
 
+// One tile of a pass, decoded identically by every role.
+struct BwdTile {
+    int tile, bh_res;       // index of the 128-row tile inside its head; (batch, head) of the resident tensors
+    int sub_lo, sub_hi;     // range of 64-row tiles of the streamed axis
+    int n_steps;            // 0: nothing reaches this tile (its gradients are zero)
+    int kv_bh_of_q;         // MODE 0: K/V head of this query head
+};
+
 // tmR0 / tmR1: maps of the resident tiles, boxes of 128 rows (MODE 0: Q, dO; MODE 1: K, V); tmT0 / tmT1: maps of
 // the streamed tiles, boxes of 64 rows (MODE 0: K, V; MODE 1: Q, dO); tmOut0 / tmOut1: MODE 0: dQ, unused;
 // MODE 1: dV, dK (boxes of 128 rows).
@@ -169,8 +188,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 const __grid_constant__ CUtensorMap tmT0, const __grid_constant__ CUtensorMap tmT1,
                 const __grid_constant__ CUtensorMap tmOut0, const __grid_constant__ CUtensorMap tmOut1,
                 const BwdParams prm) {
-    using C = BwdCfg<D>;
-    constexpr int BT = C::BT, BS = C::BS, NBOX = C::NBOX, NSTAGE = C::NSTAGE;
+    using C = BwdCfg<D, MODE>;
+    constexpr int BT = C::BT, BS = C::BS, NBOX = C::NBOX, NSTAGE = C::NSTAGE, NACC = C::NACC;
     // The S and dP products read their resident operand (A) from tensor memory wherever 512 columns allow it: with both
     // operands in shared memory an M 128 x N 64 instruction is paced by shared-memory bandwidth (6 KB per 32 tensor
     // cycles), with A in tensor memory it reads 2 KB.  The dK/dV pass at D = 128 has no columns left for it.
@@ -181,23 +200,29 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     auto sR = [&](int w) { return smem_base + w * C::RES_BYTES; };                                          // resident tile w
     auto sT = [&](int stage, int w) { return smem_base + 2 * C::RES_BYTES + (2 * stage + w) * C::STR_BYTES; };  // streamed tile w
-    constexpr int VEC_OFF = 2 * C::RES_BYTES + 2 * NSTAGE * C::STR_BYTES;
+    constexpr int STG_OFF = 2 * C::RES_BYTES + 2 * NSTAGE * C::STR_BYTES;
+    const uint32_t sStg = smem_base + STG_OFF;                                                              // staging tiles
+    constexpr int VEC_OFF = STG_OFF + C::STG_BYTES;
     float* vec = reinterpret_cast<float*>(smem_gen + VEC_OFF);   // [stage][-L log2 e | -delta][BS]
     const uint32_t sVec = smem_base + VEC_OFF;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + C::TILE_BYTES);
     const uint32_t bars_u32 = smem_base + C::TILE_BYTES;
+    // Per-tile barriers complete once per (non-empty) tile of this CTA, per-step barriers once per step of their
+    // group or stage; every role counts tiles (kk) and steps (gs) the same way, across tiles.
     enum {
-        B_RFULL = 0,      // resident tiles loaded (TMA bytes)
-        B_SFULL = 1,      // [2] S and dP of a step of group g are in tensor memory (MMA commit)
-        B_SREAD = 3,      // [2] group g has them in registers: S and dP may be overwritten (128 threads)
-        B_PFULL = 5,      // [2] the 16-bit operands of a step are in operand region g (128 threads)
-        B_OPFREE = 7,     // [2] the accumulating products of a step have read operand region g (MMA commit)
-        B_ACCFINAL = 9,   // the last accumulating product has finished
-        B_ESYNC = 10,     // barrier among all 256 element-wise threads (epilogue)
-        B_RTMEM = 11,     // the resident tiles have been copied into tensor memory (256 element-wise threads)
-        B_TFULL = 12,     // [NSTAGE] streamed tiles (and, MODE 1, their row vectors) loaded
-        B_TEMPTY = 12 + NSTAGE,
-        B_COUNT = 12 + 2 * NSTAGE
+        B_RFULL = 0,      // tile: resident tiles loaded (TMA bytes)
+        B_RTMEM = 1,      // tile: resident tiles copied into tensor memory (256 element-wise threads)
+        B_SLAST = 2,      // tile: its last S / dP product has finished (MMA commit): resident operand no longer read
+        B_ACCFINAL = 3,   // tile: its last accumulating product has finished (MMA commit)
+        B_ACCFREE = 4,    // tile: the accumulators are in registers, the next tile may overwrite them (256 threads)
+        B_ESYNC = 5,      // barrier among all 256 element-wise threads (epilogue)
+        B_SFULL = 6,      // [2] step: S and dP of a step of group g are in tensor memory (MMA commit)
+        B_SREAD = 8,      // [2] step: group g has them in registers: S and dP may be overwritten (128 threads)
+        B_PFULL = 10,     // [2] step: the 16-bit operands of a step are in operand region g (128 threads)
+        B_OPFREE = 12,    // [2] step: the accumulating products of a step have read operand region g (MMA commit)
+        B_TFULL = 14,     // [NSTAGE] step: streamed tiles (and, MODE 1, their row vectors) loaded
+        B_TEMPTY = 14 + NSTAGE,
+        B_COUNT = 14 + 2 * NSTAGE
     };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
@@ -205,64 +230,66 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // ---- this CTA's tile and its steps ----
-    // The grid is one-dimensional, tiles of one head next to each other (their streamed tiles are shared in L2).
+    // ---- the tiles of this CTA ----
+    // Tiles of one head are neighbours in the order (their streamed tiles are shared in L2).
     // MODE 0: 128-row Q tile (causal: longest first) of a (batch, query head); steps = 64-key K/V tiles.
     // MODE 1: 128-key K/V tile (the first has the most steps) of a (batch, K/V head);
     //         steps = (query head of the group, 64-row Q tile) pairs.
     const int group = prm.H / prm.Hkv;
     const int tiles_per_head = MODE == 0 ? prm.n_qtiles : prm.n_ktiles;
-    const int bid_tile = static_cast<int>(blockIdx.x % static_cast<unsigned>(tiles_per_head));
-    const int bh_res = static_cast<int>(blockIdx.x / static_cast<unsigned>(tiles_per_head));
-    int tile, sub_lo, sub_hi, n_steps;
-    if constexpr (MODE == 0) {
-        tile = prm.causal ? prm.n_qtiles - 1 - bid_tile : bid_tile;
-        const int last_key = attn_tc::last_visible_key(tile * BT + BT - 1, prm.Sk, prm.causal, 0);
-        sub_lo = 0;
-        sub_hi = last_key < 0 ? 0 : last_key / BS + 1;
-        n_steps = sub_hi;
-    } else {
-        tile = bid_tile;
-        sub_lo = prm.causal ? (tile * BT) / BS : 0;     // first 64-row Q tile with a row that sees key tile * BT
-        sub_hi = (prm.Sq + BS - 1) / BS;
-        if (sub_lo > sub_hi) sub_lo = sub_hi;
-        n_steps = (sub_hi - sub_lo) * group;
-    }
-    const int kv_bh_of_q = (bh_res / prm.H) * prm.Hkv + (bh_res % prm.H) / group;   // MODE 0: K/V head of this query head
-    // streamed tile of step u: (head index in its tensor, index of the 64-row tile)
-    auto step_head = [&](int u) {
-        if constexpr (MODE == 0) return kv_bh_of_q;
-        else return (bh_res / prm.Hkv) * prm.H + (bh_res % prm.Hkv) * group + u / (sub_hi - sub_lo);
-    };
-    auto step_sub = [&](int u) {
-        if constexpr (MODE == 0) return u;
-        else return sub_lo + u % (sub_hi - sub_lo);
-    };
-
-    if (n_steps == 0) {
-        // nothing reaches this tile (keys that no query sees, or no keys at all): the gradients are zero
-        const int rows_total = MODE == 0 ? prm.Sq : prm.Sk;
-        const int rows = rows_total - tile * BT < BT ? rows_total - tile * BT : BT;
-        if (rows > 0) {
-            const int64_t first = static_cast<int64_t>(bh_res) * rows_total + tile * BT;
-            zero_rows(prm.out0, first, rows, D, tid, C::THREADS);
-            if constexpr (MODE == 1) zero_rows(prm.out1, first, rows, D, tid, C::THREADS);
+    auto decode = [&](int lin) {
+        BwdTile t;
+        const int bid_tile = lin % tiles_per_head;
+        t.bh_res = lin / tiles_per_head;
+        if constexpr (MODE == 0) {
+            t.tile = prm.causal ? prm.n_qtiles - 1 - bid_tile : bid_tile;
+            const int last_key = attn_tc::last_visible_key(t.tile * BT + BT - 1, prm.Sk, prm.causal, 0);
+            t.sub_lo = 0;
+            t.sub_hi = last_key < 0 ? 0 : last_key / BS + 1;
+            t.n_steps = t.sub_hi;
+        } else {
+            t.tile = bid_tile;
+            t.sub_lo = prm.causal ? (t.tile * BT) / BS : 0;     // first 64-row Q tile with a row that sees key tile * BT
+            t.sub_hi = (prm.Sq + BS - 1) / BS;
+            if (t.sub_lo > t.sub_hi) t.sub_lo = t.sub_hi;
+            t.n_steps = (t.sub_hi - t.sub_lo) * group;
         }
-        return;
-    }
+        t.kv_bh_of_q = (t.bh_res / prm.H) * prm.Hkv + (t.bh_res % prm.H) / group;
+        return t;
+    };
+    // streamed tile of step u of tile t: (head index in its tensor, index of the 64-row tile)
+    auto step_head = [&](const BwdTile& t, int u) {
+        if constexpr (MODE == 0) return t.kv_bh_of_q;
+        else return (t.bh_res / prm.Hkv) * prm.H + (t.bh_res % prm.Hkv) * group + u / (t.sub_hi - t.sub_lo);
+    };
+    auto step_sub = [&](const BwdTile& t, int u) {
+        if constexpr (MODE == 0) return u;
+        else return t.sub_lo + u % (t.sub_hi - t.sub_lo);
+    };
+    // the next non-empty tile of this CTA at or after position k of its round-robin walk (-1: none)
+    auto next_work = [&](int k, BwdTile& t) {
+        for (;; ++k) {
+            const int64_t lin = static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(k) * gridDim.x;
+            if (lin >= prm.n_tiles_total) return -1;
+            t = decode(static_cast<int>(lin));
+            if (t.n_steps > 0) return k;
+        }
+    };
 
     if (tid == 0) {
         *abort_flag = 0;
         mbar_init(bar(B_RFULL), 1);
+        mbar_init(bar(B_RTMEM), 256);
+        mbar_init(bar(B_SLAST), 1);
+        mbar_init(bar(B_ACCFINAL), 1);
+        mbar_init(bar(B_ACCFREE), 256);
+        mbar_init(bar(B_ESYNC), 256);
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(B_SFULL + b), 1);
             mbar_init(bar(B_SREAD + b), 128);
             mbar_init(bar(B_PFULL + b), 128);
             mbar_init(bar(B_OPFREE + b), 1);
         }
-        mbar_init(bar(B_ACCFINAL), 1);
-        mbar_init(bar(B_ESYNC), 256);
-        mbar_init(bar(B_RTMEM), 256);
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(bar(B_TFULL + s), 1);
             mbar_init(bar(B_TEMPTY + s), 1);
@@ -294,30 +321,38 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
       if (warp == 9) {
         // =========================== TMA producer ===========================
         const bool leader = elect_one();
-        if (leader) {
-            mbar_arrive_expect_tx(bar(B_RFULL), 2 * C::RES_BYTES);
-#pragma unroll
-            for (int bx = 0; bx < NBOX; ++bx) {
-                tma_load_3d(sR(0) + bx * BT * 128, &tmR0, bar(B_RFULL), bx * 64, tile * BT, bh_res);
-                tma_load_3d(sR(1) + bx * BT * 128, &tmR1, bar(B_RFULL), bx * 64, tile * BT, bh_res);
-            }
-        }
-        for (int u = 0; u < n_steps; ++u) {
-            const int st = u % NSTAGE;
-            if (!mbar_wait(bar(B_TEMPTY + st), ((u / NSTAGE) & 1) ^ 1, abort_flag)) break;
+        BwdTile t;
+        int gs = 0, kk = 0;   // steps and tiles so far
+        bool ok = true;
+        for (int k = next_work(0, t); k >= 0 && ok; k = next_work(k + 1, t), ++kk) {
+            // the resident tiles' shared memory is free once the previous tile's have been copied into tensor memory
+            // or, where they are read in place, once its last S / dP product has finished
+            if (kk > 0 && !(ok = mbar_wait(bar(A_TMEM ? B_RTMEM : B_SLAST), (kk - 1) & 1, abort_flag))) break;
             if (leader) {
-                mbar_arrive_expect_tx(bar(B_TFULL + st), 2 * C::STR_BYTES + (MODE == 1 ? 2 * BS * 4 : 0));
-                const int head = step_head(u), row0 = step_sub(u) * BS;
-                if constexpr (MODE == 1) {
-                    // the prepared row vectors of the 64 streamed query rows (aligned and in bounds by construction)
-                    const int64_t off = static_cast<int64_t>(head) * prm.Sq_pad + row0;
-                    bulk_load_1d(sVec + st * 2 * BS * 4, prm.nl2 + off, BS * 4, bar(B_TFULL + st));
-                    bulk_load_1d(sVec + st * 2 * BS * 4 + BS * 4, prm.ndelta + off, BS * 4, bar(B_TFULL + st));
-                }
+                mbar_arrive_expect_tx(bar(B_RFULL), 2 * C::RES_BYTES);
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx) {
-                    tma_load_3d(sT(st, 0) + bx * BS * 128, &tmT0, bar(B_TFULL + st), bx * 64, row0, head);
-                    tma_load_3d(sT(st, 1) + bx * BS * 128, &tmT1, bar(B_TFULL + st), bx * 64, row0, head);
+                    tma_load_3d(sR(0) + bx * BT * 128, &tmR0, bar(B_RFULL), bx * 64, t.tile * BT, t.bh_res);
+                    tma_load_3d(sR(1) + bx * BT * 128, &tmR1, bar(B_RFULL), bx * 64, t.tile * BT, t.bh_res);
+                }
+            }
+            for (int u = 0; u < t.n_steps; ++u, ++gs) {
+                const int st = gs % NSTAGE;
+                if (!(ok = mbar_wait(bar(B_TEMPTY + st), ((gs / NSTAGE) & 1) ^ 1, abort_flag))) break;
+                if (leader) {
+                    mbar_arrive_expect_tx(bar(B_TFULL + st), 2 * C::STR_BYTES + (MODE == 1 ? 2 * BS * 4 : 0));
+                    const int head = step_head(t, u), row0 = step_sub(t, u) * BS;
+                    if constexpr (MODE == 1) {
+                        // the prepared row vectors of the 64 streamed query rows (aligned and in bounds by construction)
+                        const int64_t off = static_cast<int64_t>(head) * prm.Sq_pad + row0;
+                        bulk_load_1d(sVec + st * 2 * BS * 4, prm.nl2 + off, BS * 4, bar(B_TFULL + st));
+                        bulk_load_1d(sVec + st * 2 * BS * 4 + BS * 4, prm.ndelta + off, BS * 4, bar(B_TFULL + st));
+                    }
+#pragma unroll
+                    for (int bx = 0; bx < NBOX; ++bx) {
+                        tma_load_3d(sT(st, 0) + bx * BS * 128, &tmT0, bar(B_TFULL + st), bx * 64, row0, head);
+                        tma_load_3d(sT(st, 1) + bx * BS * 128, &tmT1, bar(B_TFULL + st), bx * 64, row0, head);
+                    }
                 }
             }
         }
@@ -328,10 +363,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         constexpr uint32_t IDESC_ACC = make_idesc_f16(BT, D, DTYPE, 0, 1);   // A from tensor memory, B MN-major (N = D)
         constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
         const uint32_t r_lo[2] = {smem_desc_lo(sR(0), 16), smem_desc_lo(sR(1), 16)};
-        // S (or S^T) = R0 T0^T, dP (or dP^T) = R1 T1^T of step u : D / 16 instructions each (M 128, N 64, K 16)
-        auto issue_s = [&](int u) {
+        // S (or S^T) = R0 T0^T, dP (or dP^T) = R1 T1^T of global step gs : D / 16 instructions each (M 128, N 64, K 16)
+        auto issue_s = [&](int gs) {
             if (leader) {
-                const int st = u % NSTAGE;
+                const int st = gs % NSTAGE;
 #pragma unroll
                 for (int w = 0; w < 2; ++w) {
                     const uint32_t b0 = smem_desc_lo(sT(st, w), 16);
@@ -345,69 +380,74 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                             mma_f16_ss_lohi(tmem + (w == 0 ? C::S_COL : C::DP_COL), r_lo[w] + offa, b0 + offb, DESC_HI, IDESC_S, kk > 0);
                     }
                 }
-                mma_commit(bar(B_SFULL + (u & 1)));
+                mma_commit(bar(B_SFULL + (gs & 1)));
             }
         };
-        // accumulating products of step v (contraction step kk, 16 values = 8 columns, starts at column 8 kk of its
-        // operand); afterwards its streamed tiles and its operand region are free
-        auto issue_acc = [&](int v) {
+        // accumulating products of global step gs, step u of its tile (contraction step kk, 16 values = 8 columns,
+        // starts at column 8 kk of its operand); afterwards its streamed tiles and its operand region are free
+        auto issue_acc = [&](int gs, int u) {
             if (leader) {
-                const int st = v % NSTAGE;
-                const uint32_t op = tmem + C::op_col(v & 1);
+                const int st = gs % NSTAGE;
+                const uint32_t op = tmem + C::op_col(gs & 1);
                 if constexpr (MODE == 0) {
                     // dQ += dS K_j : dS from tensor memory, K_j MN-major
                     const uint32_t b0 = smem_desc_lo(sT(st, 0), BS * 128);
 #pragma unroll
                     for (int kk = 0; kk < BS / 16; ++kk)
                         mma_f16_ts_lohi(tmem + C::ACC0_COL, op + kk * 8, b0 + ((kk * 16 * 128) >> 4), DESC_HI,
-                                        IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
+                                        IDESC_ACC, (u > 0 || kk > 0) ? 1u : 0u);
                 } else {
                     // dV += P^T dO_i, dK += dS^T Q_i; dO_i and Q_i MN-major
                     const uint32_t bdo = smem_desc_lo(sT(st, 1), BS * 128), bq = smem_desc_lo(sT(st, 0), BS * 128);
 #pragma unroll
                     for (int kk = 0; kk < BS / 16; ++kk)
                         mma_f16_ts_lohi(tmem + C::ACC0_COL, op + kk * 8, bdo + ((kk * 16 * 128) >> 4), DESC_HI,
-                                        IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
+                                        IDESC_ACC, (u > 0 || kk > 0) ? 1u : 0u);
 #pragma unroll
                     for (int kk = 0; kk < BS / 16; ++kk)
                         mma_f16_ts_lohi(tmem + C::ACC1_COL, op + 32 + kk * 8, bq + ((kk * 16 * 128) >> 4), DESC_HI,
-                                        IDESC_ACC, (v > 0 || kk > 0) ? 1u : 0u);
+                                        IDESC_ACC, (u > 0 || kk > 0) ? 1u : 0u);
                 }
                 mma_commit(bar(B_TEMPTY + st));
-                mma_commit(bar(B_OPFREE + (v & 1)));
-                if (v + 1 == n_steps) mma_commit(bar(B_ACCFINAL));
+                mma_commit(bar(B_OPFREE + (gs & 1)));
             }
         };
+        BwdTile t;
+        int gs = 0, kk = 0;
+        bool ok = true;
         if (warp == 8) {
-            // S and dP of step u + 1 as soon as step u's are in its group's registers
-            bool ok = mbar_wait(bar(A_TMEM ? B_RTMEM : B_RFULL), 0, abort_flag) && mbar_wait(bar(B_TFULL), 0, abort_flag);
-            if (ok) {
-                tc_fence_after_sync();
-                issue_s(0);
-            }
-            for (int u = 0; u + 1 < n_steps && ok; ++u) {
-                if (!(ok = mbar_wait(bar(B_SREAD + (u & 1)), (u >> 1) & 1, abort_flag))) break;
-                if (!(ok = mbar_wait(bar(B_TFULL + (u + 1) % NSTAGE), ((u + 1) / NSTAGE) & 1, abort_flag))) break;
-                tc_fence_after_sync();
-                issue_s(u + 1);
+            // S and dP of a step as soon as the previous step's are in its group's registers (also across tiles)
+            for (int k = next_work(0, t); k >= 0 && ok; k = next_work(k + 1, t), ++kk) {
+                if (!(ok = mbar_wait(bar(A_TMEM ? B_RTMEM : B_RFULL), kk & 1, abort_flag))) break;
+                for (int u = 0; u < t.n_steps; ++u, ++gs) {
+                    if (gs > 0 && !(ok = mbar_wait(bar(B_SREAD + ((gs - 1) & 1)), ((gs - 1) >> 1) & 1, abort_flag))) break;
+                    if (!(ok = mbar_wait(bar(B_TFULL + gs % NSTAGE), (gs / NSTAGE) & 1, abort_flag))) break;
+                    tc_fence_after_sync();
+                    issue_s(gs);
+                    if (u + 1 == t.n_steps && leader) mma_commit(bar(B_SLAST));
+                }
             }
         } else {
-            // the accumulating products of step v as soon as its operands are in tensor memory (its streamed tiles
-            // were loaded before its S and dP; this warp observes that barrier itself all the same)
-            bool ok = true;
-            for (int v = 0; v < n_steps && ok; ++v) {
-                if (!(ok = mbar_wait(bar(B_TFULL + v % NSTAGE), (v / NSTAGE) & 1, abort_flag))) break;
-                if (!(ok = mbar_wait(bar(B_PFULL + (v & 1)), (v >> 1) & 1, abort_flag))) break;
-                tc_fence_after_sync();
-                issue_acc(v);
+            // the accumulating products of a step as soon as its operands are in tensor memory (its streamed tiles
+            // were loaded before its S and dP; this warp observes that barrier itself all the same); the first of a
+            // tile overwrites the accumulators, which the previous tile's epilogue must have read
+            for (int k = next_work(0, t); k >= 0 && ok; k = next_work(k + 1, t), ++kk) {
+                for (int u = 0; u < t.n_steps; ++u, ++gs) {
+                    if (!(ok = mbar_wait(bar(B_TFULL + gs % NSTAGE), (gs / NSTAGE) & 1, abort_flag))) break;
+                    if (!(ok = mbar_wait(bar(B_PFULL + (gs & 1)), (gs >> 1) & 1, abort_flag))) break;
+                    if (u == 0 && kk > 0 && !(ok = mbar_wait(bar(B_ACCFREE), (kk - 1) & 1, abort_flag))) break;
+                    tc_fence_after_sync();
+                    issue_acc(gs, u);
+                    if (u + 1 == t.n_steps && leader) mma_commit(bar(B_ACCFINAL));
+                }
             }
         }
       }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         // =========================== element-wise groups + epilogue ===========================
-        // Group g (warps 4g .. 4g+3) takes the steps u = g, g + 2, ...: always step buffer g.  While one group
-        // waits for its tile or for tensor memory, the other computes.
+        // Group g (warps 4g .. 4g+3) takes the steps with an even (g = 0) or odd (g = 1) global index: always operand
+        // region g.  While one group waits for its tile or for tensor memory, the other computes.
         const int grp = warp >> 2;
         const int half = grp;                                // epilogue: which 32 of every 64 output columns
         const int r = (warp & 3) * 32 + lane;                // tensor-memory lane: query row (MODE 0) / key row (MODE 1)
@@ -416,35 +456,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         const uint32_t tOP = tmem + C::op_col(grp) + lane_off;
         const float c = prm.scale_log2;
         const uint64_t c2 = pack_f32x2(c, c);
-        const int my_row = tile * BT + r;                    // global query row (MODE 0) or key index (MODE 1)
-        float my_nl2 = 0.f, my_ndelta = 0.f;                 // MODE 0: minus this row's L * log2(e), minus its delta
-        if constexpr (MODE == 0) {
-            if (my_row < prm.Sq) {
-                my_nl2 = prm.nl2[static_cast<int64_t>(bh_res) * prm.Sq_pad + my_row];
-                my_ndelta = prm.ndelta[static_cast<int64_t>(bh_res) * prm.Sq_pad + my_row];
-            }
-        }
         bool ok = true;
-        if constexpr (A_TMEM) {
-            // Group g copies resident tile g from shared memory (rows of 128 bytes per 64-column box, 16-byte chunks
-            // swizzled by row) into tensor memory: lane = row, two 16-bit values per column in memory order.
-            if ((ok = mbar_wait(bar(B_RFULL), 0, abort_flag))) {
-                const uint32_t src = sR(grp) + r * 128;
-#pragma unroll
-                for (int bx = 0; bx < NBOX; ++bx) {
-                    uint32_t w[32];
-#pragma unroll
-                    for (int g8 = 0; g8 < 8; ++g8)
-                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                     : "=r"(w[g8 * 4 + 0]), "=r"(w[g8 * 4 + 1]), "=r"(w[g8 * 4 + 2]), "=r"(w[g8 * 4 + 3])
-                                     : "r"(src + bx * BT * 128 + ((g8 ^ (r & 7)) << 4)) : "memory");
-                    tmem_st_32x32b_x32(tmem + C::rt_col(grp) + bx * 32 + lane_off, w);
-                }
-                tmem_st_wait();
-                tc_fence_before_sync();
-                mbar_arrive(bar(B_RTMEM));
-            }
-        }
         // The barrier among the element-wise threads is an mbarrier with the same bounded wait as everything else (a
         // plain bar.sync would wait forever for a thread that has left through the time-out path).
         uint32_t esync_phase = 0;
@@ -454,105 +466,146 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             ++esync_phase;
             return done;
         };
-        for (int u = grp; u < n_steps && ok; u += 2) {
-            const int t = step_sub(u);
-            // MODE 1: -L log2(e) and -delta of the step's 64 query rows arrived with its streamed tiles (the S / dP
-            // products below were issued after that stage's "full" barrier, so the values are in place)
-            const float* vnl2 = vec + (u % NSTAGE) * 2 * BS;
-            const float* vndl = vnl2 + BS;
-            if constexpr (MODE == 1) {   // observe the bulk copies' barrier ourselves (it completed before S was issued)
-                if (!(ok = mbar_wait(bar(B_TFULL + u % NSTAGE), (u / NSTAGE) & 1, abort_flag))) break;
-            }
-            if (!(ok = mbar_wait(bar(B_SFULL + grp), (u >> 1) & 1, abort_flag))) break;
-            tc_fence_after_sync();
-            // does any element of this step need the mask?  (uniform over the CTA)
-            //   MODE 0: rows tile*128 .. +127, keys t*64 .. +63;  MODE 1: keys tile*128 .. +127, rows t*64 .. +63
-            const int key0 = MODE == 0 ? t * BS : tile * BT, nkeys = MODE == 0 ? BS : BT;
-            const int row0 = MODE == 0 ? tile * BT : t * BS;
-            const bool partial = (key0 + nkeys > prm.Sk) || (prm.causal && key0 + nkeys - 1 > row0);
-            // the whole S and dP row of this step into registers, then tensor memory is free for the next step
-            uint32_t sr[BS], dpr[BS];
+        // Group g copies resident tile g of the kk-th tile from shared memory (rows of 128 bytes per 64-column box,
+        // 16-byte chunks swizzled by row) into tensor memory: lane = row, two 16-bit values per column in memory order.
+        auto copy_resident = [&](int kk) -> bool {
+            if (!mbar_wait(bar(B_RFULL), kk & 1, abort_flag)) return false;
+            const uint32_t src = sR(grp) + r * 128;
 #pragma unroll
-            for (int ch = 0; ch < BS / 32; ++ch) {
-                tmem_ld_32x32b_x32(tS + 32 * ch, sr + 32 * ch);
-                tmem_ld_32x32b_x32(tDP + 32 * ch, dpr + 32 * ch);
-            }
-            tmem_ld_wait();
-            tc_fence_before_sync();
-            mbar_arrive(bar(B_SREAD + grp));
-            // operand region `grp` was last read by the accumulating products of step u - 2
-            bool op_free = u < 2;
-            // Two instances of the arithmetic: steps that need the mask (diagonal and ragged tiles) and all others,
-            // whose code then carries no trace of the mask (predicated-off mask code more than doubled its time).
-            auto make_operands = [&](auto masked_tag) {
-            constexpr bool MASKED = decltype(masked_tag)::value;
+            for (int bx = 0; bx < NBOX; ++bx) {
+                uint32_t w[32];
 #pragma unroll
-            for (int ch = 0; ch < BS / 32; ++ch) {
-                uint32_t pk_p[16], pk_ds[16];
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    const int col = 32 * ch + e;
-                    uint64_t nl2_2, ndl_2;
-                    if constexpr (MODE == 0) {
-                        nl2_2 = pack_f32x2(my_nl2, my_nl2);
-                        ndl_2 = pack_f32x2(my_ndelta, my_ndelta);
-                    } else {
-                        const float2 a = *reinterpret_cast<const float2*>(vnl2 + col);
-                        const float2 d = *reinterpret_cast<const float2*>(vndl + col);
-                        nl2_2 = pack_f32x2(a.x, a.y);
-                        ndl_2 = pack_f32x2(d.x, d.y);
-                    }
-                    float x0, x1;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[col]), __uint_as_float(sr[col + 1])), c2, nl2_2), x0, x1);
-                    float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                    if constexpr (MASKED) {
-                        bool v0, v1;
-                        if constexpr (MODE == 0) {
-                            v0 = key0 + col < prm.Sk && (!prm.causal || key0 + col <= my_row);
-                            v1 = key0 + col + 1 < prm.Sk && (!prm.causal || key0 + col + 1 <= my_row);
-                        } else {
-                            v0 = my_row < prm.Sk && (!prm.causal || my_row <= row0 + col);
-                            v1 = my_row < prm.Sk && (!prm.causal || my_row <= row0 + col + 1);
-                        }
-                        p0 = v0 ? p0 : 0.f;
-                        p1 = v1 ? p1 : 0.f;
-                    }
-                    float d0, d1;
-                    unpack_f32x2(mul_f32x2(pack_f32x2(p0, p1),
-                                           add_f32x2(pack_f32x2(__uint_as_float(dpr[col]), __uint_as_float(dpr[col + 1])), ndl_2)), d0, d1);
-                    if constexpr (MODE == 1) pk_p[e / 2] = pack2<DTYPE>(p0, p1);
-                    pk_ds[e / 2] = pack2<DTYPE>(d0, d1);
-                }
-                // 32 values -> 16 columns of this group's operand region
-                if (!op_free) {
-                    if (!(ok = mbar_wait(bar(B_OPFREE + grp), ((u >> 1) - 1) & 1, abort_flag))) break;
-                    tc_fence_after_sync();
-                    op_free = true;
-                }
-                if constexpr (MODE == 0) {
-                    tmem_st_32x32b_x16(tOP + 16 * ch, pk_ds);
-                } else {
-                    tmem_st_32x32b_x16(tOP + 16 * ch, pk_p);
-                    tmem_st_32x32b_x16(tOP + 32 + 16 * ch, pk_ds);
-                }
+                for (int g8 = 0; g8 < 8; ++g8)
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(w[g8 * 4 + 0]), "=r"(w[g8 * 4 + 1]), "=r"(w[g8 * 4 + 2]), "=r"(w[g8 * 4 + 3])
+                                 : "r"(src + bx * BT * 128 + ((g8 ^ (r & 7)) << 4)) : "memory");
+                tmem_st_32x32b_x32(tmem + C::rt_col(grp) + bx * 32 + lane_off, w);
             }
-            };
-            if (partial) make_operands(std::true_type{}); else make_operands(std::false_type{});
-            if (!ok) break;
             tmem_st_wait();
             tc_fence_before_sync();
-            mbar_arrive(bar(B_PFULL + grp));
-        }
+            mbar_arrive(bar(B_RTMEM));
+            return true;
+        };
 
-        // ---- epilogue: accumulators -> 16-bit -> swizzled staging tiles -> TMA stores (rows beyond the tensor clipped).
-        // The ring of streamed tiles is idle by now (every load has been consumed, every product that read it has
-        // finished), so each 64-column piece of the output gets a staging tile of its own there: one barrier, then
-        // all stores at once. ----
-        if (ok && (ok = mbar_wait(bar(B_ACCFINAL), 0, abort_flag))) {
+        BwdTile t, tn;
+        int gs0 = 0, kk = 0;   // global index of the tile's first step; tiles so far
+        int k = next_work(0, t);
+        if (A_TMEM && k >= 0) ok = copy_resident(0);
+        for (; k >= 0 && ok; ++kk) {
+            const int my_row = t.tile * BT + r;                  // global query row (MODE 0) or key index (MODE 1)
+            float my_nl2 = 0.f, my_ndelta = 0.f;                 // MODE 0: minus this row's L * log2(e), minus its delta
+            if constexpr (MODE == 0) {
+                if (my_row < prm.Sq) {
+                    my_nl2 = prm.nl2[static_cast<int64_t>(t.bh_res) * prm.Sq_pad + my_row];
+                    my_ndelta = prm.ndelta[static_cast<int64_t>(t.bh_res) * prm.Sq_pad + my_row];
+                }
+            }
+            for (int u = (gs0 + grp) & 1; u < t.n_steps && ok; u += 2) {     // own steps: global index gs0 + u = grp mod 2
+                const int gs = gs0 + u;
+                const int ts = step_sub(t, u);
+                // MODE 1: -L log2(e) and -delta of the step's 64 query rows arrived with its streamed tiles
+                const float* vnl2 = vec + (gs % NSTAGE) * 2 * BS;
+                const float* vndl = vnl2 + BS;
+                if constexpr (MODE == 1) {   // observe the bulk copies' barrier ourselves (it completed before S was issued)
+                    if (!(ok = mbar_wait(bar(B_TFULL + gs % NSTAGE), (gs / NSTAGE) & 1, abort_flag))) break;
+                }
+                if (!(ok = mbar_wait(bar(B_SFULL + grp), (gs >> 1) & 1, abort_flag))) break;
+                tc_fence_after_sync();
+                // does any element of this step need the mask?  (uniform over the CTA)
+                //   MODE 0: rows tile*128 .. +127, keys ts*64 .. +63;  MODE 1: keys tile*128 .. +127, rows ts*64 .. +63
+                const int key0 = MODE == 0 ? ts * BS : t.tile * BT, nkeys = MODE == 0 ? BS : BT;
+                const int row0 = MODE == 0 ? t.tile * BT : ts * BS;
+                const bool partial = (key0 + nkeys > prm.Sk) || (prm.causal && key0 + nkeys - 1 > row0);
+                // the whole S and dP row of this step into registers, then tensor memory is free for the next step
+                uint32_t sr[BS], dpr[BS];
+#pragma unroll
+                for (int ch = 0; ch < BS / 32; ++ch) {
+                    tmem_ld_32x32b_x32(tS + 32 * ch, sr + 32 * ch);
+                    tmem_ld_32x32b_x32(tDP + 32 * ch, dpr + 32 * ch);
+                }
+                tmem_ld_wait();
+                tc_fence_before_sync();
+                mbar_arrive(bar(B_SREAD + grp));
+                // operand region `grp` was last read by the accumulating products of global step gs - 2
+                bool op_free = gs < 2;
+                // Two instances of the arithmetic: steps that need the mask (diagonal and ragged tiles) and all others,
+                // whose code then carries no trace of the mask (predicated-off mask code more than doubled its time).
+                auto make_operands = [&](auto masked_tag) {
+                constexpr bool MASKED = decltype(masked_tag)::value;
+#pragma unroll
+                for (int ch = 0; ch < BS / 32; ++ch) {
+                    uint32_t pk_p[16], pk_ds[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const int col = 32 * ch + e;
+                        uint64_t nl2_2, ndl_2;
+                        if constexpr (MODE == 0) {
+                            nl2_2 = pack_f32x2(my_nl2, my_nl2);
+                            ndl_2 = pack_f32x2(my_ndelta, my_ndelta);
+                        } else {
+                            const float2 a = *reinterpret_cast<const float2*>(vnl2 + col);
+                            const float2 d = *reinterpret_cast<const float2*>(vndl + col);
+                            nl2_2 = pack_f32x2(a.x, a.y);
+                            ndl_2 = pack_f32x2(d.x, d.y);
+                        }
+                        float x0, x1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[col]), __uint_as_float(sr[col + 1])), c2, nl2_2), x0, x1);
+                        float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                        if constexpr (MASKED) {
+                            bool v0, v1;
+                            if constexpr (MODE == 0) {
+                                v0 = key0 + col < prm.Sk && (!prm.causal || key0 + col <= my_row);
+                                v1 = key0 + col + 1 < prm.Sk && (!prm.causal || key0 + col + 1 <= my_row);
+                            } else {
+                                v0 = my_row < prm.Sk && (!prm.causal || my_row <= row0 + col);
+                                v1 = my_row < prm.Sk && (!prm.causal || my_row <= row0 + col + 1);
+                            }
+                            p0 = v0 ? p0 : 0.f;
+                            p1 = v1 ? p1 : 0.f;
+                        }
+                        float d0, d1;
+                        unpack_f32x2(mul_f32x2(pack_f32x2(p0, p1),
+                                               add_f32x2(pack_f32x2(__uint_as_float(dpr[col]), __uint_as_float(dpr[col + 1])), ndl_2)), d0, d1);
+                        if constexpr (MODE == 1) pk_p[e / 2] = pack2<DTYPE>(p0, p1);
+                        pk_ds[e / 2] = pack2<DTYPE>(d0, d1);
+                    }
+                    // 32 values -> 16 columns of this group's operand region
+                    if (!op_free) {
+                        if (!(ok = mbar_wait(bar(B_OPFREE + grp), ((gs >> 1) - 1) & 1, abort_flag))) break;
+                        tc_fence_after_sync();
+                        op_free = true;
+                    }
+                    if constexpr (MODE == 0) {
+                        tmem_st_32x32b_x16(tOP + 16 * ch, pk_ds);
+                    } else {
+                        tmem_st_32x32b_x16(tOP + 16 * ch, pk_p);
+                        tmem_st_32x32b_x16(tOP + 32 + 16 * ch, pk_ds);
+                    }
+                }
+                };
+                if (partial) make_operands(std::true_type{}); else make_operands(std::false_type{});
+                if (!ok) break;
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(bar(B_PFULL + grp));
+            }
+            if (!ok) break;
+
+            // ---- tile boundary ----
+            // first the next tile's resident operand into tensor memory (its columns are free once this tile's last
+            // S / dP product has finished), so that the next tile's first products run while this tile's accumulators drain
+            const int kn = next_work(k + 1, tn);
+            if (A_TMEM && kn >= 0) {
+                if (!(ok = mbar_wait(bar(B_SLAST), kk & 1, abort_flag))) break;
+                tc_fence_after_sync();
+                if (!(ok = copy_resident(kk + 1))) break;
+            }
+            // ---- epilogue: accumulators -> 16-bit -> swizzled staging tiles -> TMA stores (rows beyond the tensor clipped);
+            // every 64-column piece of the output has a staging tile of its own: one barrier, then all stores at once ----
+            if (!(ok = mbar_wait(bar(B_ACCFINAL), kk & 1, abort_flag))) break;
             tc_fence_after_sync();
-            constexpr int NACC = MODE == 0 ? 1 : 2;
-            static_assert(NACC * (D / 64) * C::OST_BYTES <= NSTAGE * 2 * C::STR_BYTES, "staging tiles must fit the ring");
-            const uint32_t stage0 = sT(0, 0);
+            if (tid == 0) tma_store_wait_read<0>();              // the previous tile's stores have read the staging tiles
+            if (!(ok = all_sync())) break;
 #pragma unroll
             for (int a = 0; a < NACC; ++a) {
                 // MODE 0: dQ (x scale).  MODE 1: accumulator 0 = dV, accumulator 1 = dK (x scale).
@@ -564,7 +617,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                     uint32_t acc[32];
                     tmem_ld_32x32b_x32(tA + h * 64 + 32 * half, acc);
                     tmem_ld_wait();
-                    const uint32_t ost = stage0 + (a * (D / 64) + h) * C::OST_BYTES;
+                    if (a == NACC - 1 && h == D / 64 - 1) {      // the accumulators are in registers: the next tile may start
+                        tc_fence_before_sync();
+                        mbar_arrive(bar(B_ACCFREE));
+                    }
+                    const uint32_t ost = sStg + (a * (D / 64) + h) * C::OST_BYTES;
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         const uint32_t w0 = pack2<DTYPE>(__uint_as_float(acc[g * 8 + 0]) * f, __uint_as_float(acc[g * 8 + 1]) * f);
@@ -577,16 +634,35 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                 }
             }
             fence_proxy_async_smem();
-            if ((ok = all_sync()) && tid == 0) {
+            if (!(ok = all_sync())) break;
+            if (tid == 0) {
 #pragma unroll
                 for (int a = 0; a < NACC; ++a)
 #pragma unroll
                     for (int h = 0; h < D / 64; ++h)
-                        tma_store_3d(a == 0 ? &tmOut0 : &tmOut1, stage0 + (a * (D / 64) + h) * C::OST_BYTES, h * 64, tile * BT, bh_res);
+                        tma_store_3d(a == 0 ? &tmOut0 : &tmOut1, sStg + (a * (D / 64) + h) * C::OST_BYTES, h * 64, t.tile * BT, t.bh_res);
                 tma_store_commit();
             }
+            gs0 += t.n_steps;
+            k = kn;
+            t = tn;
         }
         if (tid == 0) tma_store_wait_all<0>();   // the staging tiles must outlive their stores
+
+        // ---- tiles that nothing reaches (keys that no query sees): their gradients are zero ----
+        for (int kz = 0;; ++kz) {
+            const int64_t lin = static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(kz) * gridDim.x;
+            if (lin >= prm.n_tiles_total) break;
+            const BwdTile z = decode(static_cast<int>(lin));
+            if (z.n_steps > 0) continue;
+            const int rows_total = MODE == 0 ? prm.Sq : prm.Sk;
+            const int rows = rows_total - z.tile * BT < BT ? rows_total - z.tile * BT : BT;
+            if (rows > 0) {
+                const int64_t first = static_cast<int64_t>(z.bh_res) * rows_total + z.tile * BT;
+                zero_rows(prm.out0, first, rows, D, tid, 256);
+                if constexpr (MODE == 1) zero_rows(prm.out1, first, rows, D, tid, 256);
+            }
+        }
     }
 
     // ---- teardown (also reached after a timed-out wait) ----

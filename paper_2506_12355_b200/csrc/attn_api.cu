@@ -852,8 +852,14 @@ int attn_bwd(const void* q, const void* k, const void* v, const void* o, const f
     if (!prm.status) return ATTN_ERR_CUDA;
     // resident tiles and outputs move in boxes of 128 rows, streamed tiles in boxes of 64 rows
     DeviceInfo di;
-    if (device_info(&di) != ATTN_OK) return ATTN_ERR_CUDA;
-    const int sms = di.sm_count;   // persistent grids: one CTA per SM
+    int dev = 0;
+    if (device_info(&di, &dev) != ATTN_OK) return ATTN_ERR_CUDA;
+    const int sms = di.sm_count;   // persistent grids: one CTA per SM, later tiles from the stream's work counter
+    unsigned int* counter = nullptr;
+    if (n_qtiles * BH > sms || n_ktiles * BHkv > sms) {
+        rc = work_counter(di, dev, st, &counter);
+        if (rc != ATTN_OK) return rc;
+    }
     CUtensorMap mq, mk, mv, mdo, mq64, mk64, mv64, mdo64, mdq, mdk, mdv;
     if (!make_map(&mq, q, dtype, BH, Sq, D, 128) || !make_map(&mdo, dout, dtype, BH, Sq, D, 128) ||
         !make_map(&mq64, q, dtype, BH, Sq, D, 64) || !make_map(&mdo64, dout, dtype, BH, Sq, D, 64) ||
@@ -879,11 +885,13 @@ int attn_bwd(const void* q, const void* k, const void* v, const void* o, const f
         prm.out0 = dq;                                                                                                     \
         prm.out1 = nullptr;                                                                                                \
         prm.n_tiles_total = static_cast<int>(n_qtiles * BH);                                                               \
+        prm.counter = prm.n_tiles_total > sms ? counter : nullptr;                                                         \
         kq<<<static_cast<unsigned>(prm.n_tiles_total < sms ? prm.n_tiles_total : sms), CQ::THREADS, CQ::SMEM_BYTES, st>>>(  \
             mq, mdo, mk64, mv64, mdq, mdq, prm);                                                                           \
         prm.out0 = dv;                                                                                                     \
         prm.out1 = dk;                                                                                                     \
         prm.n_tiles_total = static_cast<int>(n_ktiles * BHkv);                                                             \
+        prm.counter = prm.n_tiles_total > sms ? counter : nullptr;                                                         \
         kkv<<<static_cast<unsigned>(prm.n_tiles_total < sms ? prm.n_tiles_total : sms), CKV::THREADS, CKV::SMEM_BYTES, st>>>( \
             mk, mv, mq64, mdo64, mdv, mdk, prm);                                                                           \
         return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;                                                \

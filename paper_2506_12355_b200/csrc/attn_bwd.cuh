@@ -41,8 +41,10 @@
 //   warp  11   idle (it completes the third warpgroup so that registers can be re-balanced: an element-wise thread
 //              holds a whole S and dP row of a step, 128 registers, while it computes)
 //
-// Persistent grid: one CTA per SM walks its tiles (tile index = block index + k * grid size; tiles of one head are
-// neighbours, causal tiles heaviest first, so the round-robin hands every CTA a similar mix).  Barriers, tensor memory
+// Persistent grid: one CTA per SM; its first tile is its block index, later ones come from a device counter (tiles of
+// one head are neighbours in the order, so that their streamed tiles meet in L2, and under the causal mask a head's
+// heaviest tiles come first, so the launch ends on light ones).  The producer warp draws a tile a few steps before the
+// current one ends and publishes it to the other roles through scheduler slots in shared memory.  Barriers, tensor memory
 // and the streamed ring live across tiles: the producer loads the next tile's resident tiles while the current tile
 // still computes, the element-wise warps copy them into tensor memory right after their last step, and the S / dP
 // products of the next tile's first step run while the accumulators of the current tile drain.
@@ -72,9 +74,10 @@ struct BwdCfg {
     static constexpr int NSTAGE = D == 64 ? 6 : (MODE == 0 ? 4 : 3);
     static constexpr int VEC_BYTES = MODE == 1 ? NSTAGE * 2 * BS * 4 : 0;   // -L log2(e) and -delta of a stage's 64 query rows
     static constexpr int TILE_BYTES = 2 * RES_BYTES + NSTAGE * 2 * STR_BYTES + STG_BYTES + VEC_BYTES;
-    static constexpr int MISC_BYTES = 256;
+    static constexpr int MISC_BYTES = 512;                  // barriers (up to 34), scheduler slots, TMEM slot, abort flag
     static constexpr int SMEM_BYTES = 1024 + TILE_BYTES + MISC_BYTES;
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+    static_assert((22 + 2 * NSTAGE) * 8 + 32 <= MISC_BYTES, "barrier area");
     static constexpr int THREADS = 384;
     // tensor memory: fp32 S in columns 0 .. 63, fp32 dP in 64 .. 127; operand region g (steps u = g mod 2) at
     // 128 + 64 g: first 16-bit operand (dS in MODE 0, P^T in MODE 1) in its columns 0 .. 31, second (dS^T) in 32 .. 63
@@ -100,7 +103,9 @@ struct BwdParams {
     int causal;
     int H, Hkv;
     int n_qtiles, n_ktiles; // 128-row tiles of the query and of the key axis
-    int n_tiles_total;      // tiles of this pass over all heads: the persistent CTAs walk them round-robin
+    int n_tiles_total;      // tiles of this pass over all heads
+    unsigned int* counter;  // work counter {next tile, CTAs done}, zero at launch and again at exit:
+                            // tile = gridDim.x + atomicAdd(counter, 1); NULL when the grid covers every tile
     int* status;
 };
 
@@ -220,13 +225,16 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         B_SREAD = 8,      // [2] step: group g has them in registers: S and dP may be overwritten (128 threads)
         B_PFULL = 10,     // [2] step: the 16-bit operands of a step are in operand region g (128 threads)
         B_OPFREE = 12,    // [2] step: the accumulating products of a step have read operand region g (MMA commit)
-        B_TFULL = 14,     // [NSTAGE] step: streamed tiles (and, MODE 1, their row vectors) loaded
-        B_TEMPTY = 14 + NSTAGE,
-        B_COUNT = 14 + 2 * NSTAGE
+        B_SCHEDFULL = 14, // [4] scheduler slot holds the CTA's next tile index (-1: no more)
+        B_SCHEDEMPTY = 18,// [4] slot read by the two MMA warps and the 8 element-wise warps
+        B_TFULL = 22,     // [NSTAGE] step: streamed tiles (and, MODE 1, their row vectors) loaded
+        B_TEMPTY = 22 + NSTAGE,
+        B_COUNT = 22 + 2 * NSTAGE
     };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 1;
+    volatile int* sched_slot = reinterpret_cast<volatile int*>(bars + B_COUNT) + 2;   // [4]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -266,13 +274,22 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         if constexpr (MODE == 0) return u;
         else return t.sub_lo + u % (t.sub_hi - t.sub_lo);
     };
-    // the next non-empty tile of this CTA at or after position k of its round-robin walk (-1: none)
-    auto next_work = [&](int k, BwdTile& t) {
-        for (;; ++k) {
-            const int64_t lin = static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(k) * gridDim.x;
-            if (lin >= prm.n_tiles_total) return -1;
-            t = decode(static_cast<int>(lin));
-            if (t.n_steps > 0) return k;
+    // Consumers of the scheduler: the tile index at position p of this CTA's walk (-1: no more); the slot is handed
+    // back at once (the caller keeps what it needs in registers).
+    auto fetch = [&](int p, bool hand_back) -> int {
+        const int slot = p & 3;
+        if (!mbar_wait(bar(B_SCHEDFULL + slot), (p >> 2) & 1, abort_flag)) return -1;
+        const int lin = sched_slot[slot];
+        if (hand_back) mbar_arrive(bar(B_SCHEDEMPTY + slot));
+        return lin;
+    };
+    // the next tile with work at or after position p (-1: none); tiles that nothing reaches are skipped
+    auto next_work = [&](int p, bool hand_back, BwdTile& t) {
+        for (;; ++p) {
+            const int lin = fetch(p, hand_back);
+            if (lin < 0) return -1;
+            t = decode(lin);
+            if (t.n_steps > 0) return p;
         }
     };
 
@@ -293,6 +310,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(bar(B_TFULL + s), 1);
             mbar_init(bar(B_TEMPTY + s), 1);
+        }
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(bar(B_SCHEDFULL + s), 1);
+            mbar_init(bar(B_SCHEDEMPTY + s), 10);
         }
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -322,9 +343,24 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         // =========================== TMA producer ===========================
         const bool leader = elect_one();
         BwdTile t;
-        int gs = 0, kk = 0;   // steps and tiles so far
+        int gs = 0, kk = 0;   // steps and tiles (with work) so far
         bool ok = true;
-        for (int k = next_work(0, t); k >= 0 && ok; k = next_work(k + 1, t), ++kk) {
+        for (int p = 0; ok; ++p) {
+            // draw the tile at position p of this CTA's walk and publish it
+            const int slot = p & 3;
+            if (!(ok = mbar_wait(bar(B_SCHEDEMPTY + slot), ((p >> 2) & 1) ^ 1, abort_flag))) break;
+            int lin = -1;
+            if (leader) {
+                lin = (p == 0) ? static_cast<int>(blockIdx.x)
+                      : (prm.counter ? static_cast<int>(gridDim.x + atomicAdd(prm.counter, 1u)) : prm.n_tiles_total);
+                if (lin < 0 || lin >= prm.n_tiles_total) lin = -1;
+                sched_slot[slot] = lin;
+                mbar_arrive(bar(B_SCHEDFULL + slot));
+            }
+            lin = fetch(p, false);   // all lanes of the warp read it back
+            if (lin < 0) break;
+            t = decode(lin);
+            if (t.n_steps == 0) continue;
             // the resident tiles' shared memory is free once the previous tile's have been copied into tensor memory
             // or, where they are read in place, once its last S / dP product has finished
             if (kk > 0 && !(ok = mbar_wait(bar(A_TMEM ? B_RTMEM : B_SLAST), (kk - 1) & 1, abort_flag))) break;
@@ -355,6 +391,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
                     }
                 }
             }
+            ++kk;
         }
       } else if (warp == 8 || warp == 10) {
         // =========================== MMA issuers ===========================
@@ -417,7 +454,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         bool ok = true;
         if (warp == 8) {
             // S and dP of a step as soon as the previous step's are in its group's registers (also across tiles)
-            for (int k = next_work(0, t); k >= 0 && ok; k = next_work(k + 1, t), ++kk) {
+            for (int k = next_work(0, leader, t); k >= 0 && ok; k = next_work(k + 1, leader, t), ++kk) {
                 if (!(ok = mbar_wait(bar(A_TMEM ? B_RTMEM : B_RFULL), kk & 1, abort_flag))) break;
                 for (int u = 0; u < t.n_steps; ++u, ++gs) {
                     if (gs > 0 && !(ok = mbar_wait(bar(B_SREAD + ((gs - 1) & 1)), ((gs - 1) >> 1) & 1, abort_flag))) break;
@@ -431,7 +468,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             // the accumulating products of a step as soon as its operands are in tensor memory (its streamed tiles
             // were loaded before its S and dP; this warp observes that barrier itself all the same); the first of a
             // tile overwrites the accumulators, which the previous tile's epilogue must have read
-            for (int k = next_work(0, t); k >= 0 && ok; k = next_work(k + 1, t), ++kk) {
+            for (int k = next_work(0, leader, t); k >= 0 && ok; k = next_work(k + 1, leader, t), ++kk) {
                 for (int u = 0; u < t.n_steps; ++u, ++gs) {
                     if (!(ok = mbar_wait(bar(B_TFULL + gs % NSTAGE), (gs / NSTAGE) & 1, abort_flag))) break;
                     if (!(ok = mbar_wait(bar(B_PFULL + (gs & 1)), (gs >> 1) & 1, abort_flag))) break;
@@ -487,9 +524,26 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             return true;
         };
 
+        // the next tile with work at or after position p; tiles on the way that nothing reaches (keys that no query
+        // sees) get their zero gradients here
+        auto next_tile = [&](int p, BwdTile& t) {
+            for (;; ++p) {
+                const int lin = fetch(p, lane == 0);
+                if (lin < 0) return -1;
+                t = decode(lin);
+                if (t.n_steps > 0) return p;
+                const int rows_total = MODE == 0 ? prm.Sq : prm.Sk;
+                const int rows = rows_total - t.tile * BT < BT ? rows_total - t.tile * BT : BT;
+                if (rows > 0) {
+                    const int64_t first = static_cast<int64_t>(t.bh_res) * rows_total + t.tile * BT;
+                    zero_rows(prm.out0, first, rows, D, tid, 256);
+                    if constexpr (MODE == 1) zero_rows(prm.out1, first, rows, D, tid, 256);
+                }
+            }
+        };
         BwdTile t, tn;
         int gs0 = 0, kk = 0;   // global index of the tile's first step; tiles so far
-        int k = next_work(0, t);
+        int k = next_tile(0, t);
         if (A_TMEM && k >= 0) ok = copy_resident(0);
         for (; k >= 0 && ok; ++kk) {
             const int my_row = t.tile * BT + r;                  // global query row (MODE 0) or key index (MODE 1)
@@ -594,7 +648,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
             // ---- tile boundary ----
             // first the next tile's resident operand into tensor memory (its columns are free once this tile's last
             // S / dP product has finished), so that the next tile's first products run while this tile's accumulators drain
-            const int kn = next_work(k + 1, tn);
+            const int kn = next_tile(k + 1, tn);
             if (A_TMEM && kn >= 0) {
                 if (!(ok = mbar_wait(bar(B_SLAST), kk & 1, abort_flag))) break;
                 tc_fence_after_sync();
@@ -649,26 +703,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         }
         if (tid == 0) tma_store_wait_all<0>();   // the staging tiles must outlive their stores
 
-        // ---- tiles that nothing reaches (keys that no query sees): their gradients are zero ----
-        for (int kz = 0;; ++kz) {
-            const int64_t lin = static_cast<int64_t>(blockIdx.x) + static_cast<int64_t>(kz) * gridDim.x;
-            if (lin >= prm.n_tiles_total) break;
-            const BwdTile z = decode(static_cast<int>(lin));
-            if (z.n_steps > 0) continue;
-            const int rows_total = MODE == 0 ? prm.Sq : prm.Sk;
-            const int rows = rows_total - z.tile * BT < BT ? rows_total - z.tile * BT : BT;
-            if (rows > 0) {
-                const int64_t first = static_cast<int64_t>(z.bh_res) * rows_total + z.tile * BT;
-                zero_rows(prm.out0, first, rows, D, tid, 256);
-                if constexpr (MODE == 1) zero_rows(prm.out1, first, rows, D, tid, 256);
-            }
-        }
     }
 
     // ---- teardown (also reached after a timed-out wait) ----
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0) finish_cta(prm.status, *abort_flag != 0, nullptr);
+    if (tid == 0) finish_cta(prm.status, *abort_flag != 0, prm.counter);
     if (warp == 8) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 

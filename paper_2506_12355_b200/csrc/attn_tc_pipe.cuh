@@ -87,7 +87,10 @@ struct PipeItem {
     int bh, kv_bh, q0;
     int k_tile0;   // first K/V tile of this item's key range (0 unless the keys are split)
     int o_bh;      // head index of the item's rows in o and lse (bh unless the keys are split)
-    int n_kv[2];   // K/V tiles each Q tile needs (0: tile beyond Sq, or no visible key)
+    int n_kv0, n_kv1;   // K/V tiles each Q tile needs (0: tile beyond Sq, or no visible key).  Two scalars, not an
+                        // array: an array indexed by a run-time tile number puts the whole item into local memory,
+                        // and the MMA warp then reads its loop bounds from there on every step.
+    __device__ __forceinline__ int nkv(int t) const { return t ? n_kv1 : n_kv0; }
     int n_max;
 };
 
@@ -110,20 +113,20 @@ __device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int 
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
         const int qs = it.q0 + t * BM;
-        if (qs >= prm.Sq) {
-            it.n_kv[t] = 0;
-        } else {
+        int n = 0;
+        if (qs < prm.Sq) {
             const int last_key = last_visible_key(qs + BM - 1, prm.Sk, prm.causal, prm.k_offset);
-            it.n_kv[t] = last_key < 0 ? 0 : last_key / BN + 1;   // 0: no row of the tile sees a key of this shard
+            n = last_key < 0 ? 0 : last_key / BN + 1;   // 0: no row of the tile sees a key of this shard
         }
         // the part of those tiles that lies in this item's key range
-        int in_range = it.n_kv[t] - split * prm.split_tiles;
+        int in_range = n - split * prm.split_tiles;
         if (in_range > prm.split_tiles) in_range = prm.split_tiles;
-        it.n_kv[t] = in_range < 0 ? 0 : in_range;
+        n = in_range < 0 ? 0 : in_range;
+        if (t == 0) it.n_kv0 = n; else it.n_kv1 = n;
     }
     it.k_tile0 = split * prm.split_tiles;
     it.o_bh = split * prm.BH + it.bh;
-    it.n_max = it.n_kv[0] > it.n_kv[1] ? it.n_kv[0] : it.n_kv[1];
+    it.n_max = it.n_kv0 > it.n_kv1 ? it.n_kv0 : it.n_kv1;
     return it;
 }
 
@@ -174,7 +177,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         B_COUNT = 22 + 2 * NSLOT
     };
     auto bar = [&](int i) { return bars_u32 + i * 8; };
-    // scheduler slots [4][8]: item index (-1: no more work), bh, kv_bh, q0, n_kv[0], n_kv[1]
+    // scheduler slots [4][8]: item index (-1: no more work), bh, kv_bh, q0, n_kv0, n_kv1
     volatile int* sched_item = reinterpret_cast<volatile int*>(bars + B_COUNT);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT) + 32;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + B_COUNT) + 33;
@@ -228,11 +231,11 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         it.bh = e[1];
         it.kv_bh = e[2];
         it.q0 = e[3];
-        it.n_kv[0] = e[4];
-        it.n_kv[1] = e[5];
+        it.n_kv0 = e[4];
+        it.n_kv1 = e[5];
         it.k_tile0 = SPLITS ? e[6] : 0;
         it.o_bh = SPLITS ? e[7] : it.bh;
-        it.n_max = it.n_kv[0] > it.n_kv[1] ? it.n_kv[0] : it.n_kv[1];
+        it.n_max = it.n_kv0 > it.n_kv1 ? it.n_kv0 : it.n_kv1;
         if (hand_back) mbar_arrive(bar(B_SCHEDEMPTY + slot));
         return item;
     };
@@ -263,8 +266,8 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         e[1] = d.bh;
                         e[2] = d.kv_bh;
                         e[3] = d.q0;
-                        e[4] = d.n_kv[0];
-                        e[5] = d.n_kv[1];
+                        e[4] = d.n_kv0;
+                        e[5] = d.n_kv1;
                         e[6] = d.k_tile0;
                         e[7] = d.o_bh;
                     }
@@ -307,10 +310,10 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     return true;
                 };
                 bool ok = true;
-                if (it.n_kv[0] > 0) ok = load_q(0);
+                if (it.n_kv0 > 0) ok = load_q(0);
                 for (int j = 0; j < it.n_max && ok; ++j) {
                     ok = load_kv(&tmK, kv_base + 2 * j, j);
-                    if (ok && j == 0 && it.n_kv[1] > 0) ok = load_q(1);
+                    if (ok && j == 0 && it.n_kv1 > 0) ok = load_q(1);
                     if (ok) ok = load_kv(&tmV, kv_base + 2 * j + 1, j);
                 }
                 if (!ok) break;
@@ -370,13 +373,13 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (it.n_max > 0) ok = kv_full_wait(kv_base);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
-                    if (ok && it.n_kv[t] > 0) {
+                    if (ok && it.nkv(t) > 0) {
                         ok = mbar_wait(bar(B_QFULL + t), uses[t] & 1, abort_flag);
                         if (ok) {
                             tc_fence_after_sync();
                             issue_s(t, kv_base % NSLOT);
                             commit(B_SFULL + t);
-                            if (it.n_kv[t] == 1) commit(B_QEMPTY + t);
+                            if (it.nkv(t) == 1) commit(B_QEMPTY + t);
                         }
                     }
                 }
@@ -389,7 +392,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     if (j + 1 < it.n_max && !(ok = kv_full_wait(kitem))) break;
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
-                        if (j < it.n_kv[t]) {
+                        if (j < it.nkv(t)) {
                             const uint32_t par = (it_base[t] + j) & 1;
                             if (!(ok = mbar_wait(bar(B_PFULL + t), par, abort_flag))) break;
                             // the epilogue of the previous item must have read O_t before it is overwritten
@@ -399,14 +402,14 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                             if (!(ok = mbar_wait(bar(B_PFULL2 + t), par, abort_flag))) break;
                             tc_fence_after_sync();
                             issue_pv(t, vslot, true, 3 * (BN / KSTEP) / 4, BN / KSTEP);
-                            if (j + 1 == it.n_kv[t]) commit(B_OFINAL + t);
+                            if (j + 1 == it.nkv(t)) commit(B_OFINAL + t);
                         }
                         if (t == 1) commit(B_KVEMPTY + vslot);
-                        if (j + 1 < it.n_kv[t]) {
+                        if (j + 1 < it.nkv(t)) {
                             tc_fence_after_sync();
                             issue_s(t, kslot);
                             commit(B_SFULL + t);
-                            if (j + 2 == it.n_kv[t]) commit(B_QEMPTY + t);   // that was the last S of this item
+                            if (j + 2 == it.nkv(t)) commit(B_QEMPTY + t);   // that was the last S of this item
                         }
                     }
                     if (ok && j + 1 < it.n_max) commit(B_KVEMPTY + kslot);
@@ -414,8 +417,8 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 kv_base += 2 * it.n_max;
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
-                    it_base[t] += it.n_kv[t];
-                    uses[t] += it.n_kv[t] > 0 ? 1 : 0;
+                    it_base[t] += it.nkv(t);
+                    uses[t] += it.nkv(t) > 0 ? 1 : 0;
                 }
             }
         }
@@ -441,7 +444,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             PipeItem it;
             const int item = next_item(k, lane == 0, it);
             if (item < 0) break;
-            const int n = it.n_kv[t];
+            const int n = it.nkv(t);
             const int q0 = it.q0;
             const int row = q0 + t * BM + r;
             if (n == 0) {

@@ -79,15 +79,22 @@ struct BwdCfg {
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
     static_assert((22 + 2 * NSTAGE) * 8 + 32 <= MISC_BYTES, "barrier area");
     static constexpr int THREADS = 384;
-    // tensor memory: fp32 S in columns 0 .. 63, fp32 dP in 64 .. 127; operand region g (steps u = g mod 2) at
-    // 128 + 64 g: first 16-bit operand (dS in MODE 0, P^T in MODE 1) in its columns 0 .. 31, second (dS^T) in 32 .. 63
+    // tensor memory: fp32 S in columns 0 .. 63, fp32 dP in 64 .. 127; operand region g (steps u = g mod 2): first
+    // 16-bit operand (dS in MODE 0, P^T in MODE 1) in its columns 0 .. 31, second (MODE 1: dS^T) in 32 .. 63.
+    // Wherever 64 more columns are free (everywhere but the dK/dV pass at D = 128), S has a second buffer: the S of
+    // step u + 1 is then computed while the element-wise group still holds the dP columns of step u, and only the dP
+    // product is left between "S and dP of step u are in registers" and "S and dP of step u + 1 are ready".
+    static constexpr bool S2BUF = !(MODE == 1 && D == 128);
     static constexpr int S_COL = 0, DP_COL = 64;
-    __host__ __device__ static constexpr int op_col(int g) { return 128 + 64 * g; }
+    __host__ __device__ static constexpr int op_col(int g) { return MODE == 0 ? 128 + 32 * g : 128 + 64 * g; }
+    __host__ __device__ static constexpr int s_col(int b) { return (S2BUF && b) ? (MODE == 0 ? 192 : 384) : S_COL; }
     static constexpr int ACC0_COL = 256, ACC1_COL = 256 + D;
     // the resident tiles as 16-bit A operands in tensor memory (where the columns allow it): tile w in D / 2 columns
     __host__ __device__ static constexpr int rt_col(int w) { return 512 - D + w * (D / 2); }
     static constexpr int TMEM_COLS = 512;
     static_assert(D == 64 || D == 128, "head dims 64 and 128");
+    static_assert(!S2BUF || MODE == 0 || 384 + 64 <= 512 - D, "second S buffer below the resident operands");
+    static_assert(ACC0_COL + NACC * D <= (MODE == 0 ? 512 - D : (D == 64 ? 384 : 512)), "accumulators end below what follows them");
 };
 
 struct BwdParams {
@@ -401,23 +408,21 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         constexpr uint32_t DESC_HI = smem_desc_hi_sw128(1024);
         const uint32_t r_lo[2] = {smem_desc_lo(sR(0), 16), smem_desc_lo(sR(1), 16)};
         // S (or S^T) = R0 T0^T, dP (or dP^T) = R1 T1^T of global step gs : D / 16 instructions each (M 128, N 64, K 16)
-        auto issue_s = [&](int gs) {
+        // product w of global step gs: w = 0: S into the S buffer of the step's parity, w = 1: dP
+        auto issue_prod = [&](int gs, int w) {
             if (leader) {
                 const int st = gs % NSTAGE;
+                const uint32_t b0 = smem_desc_lo(sT(st, w), 16);
+                const uint32_t dcol = tmem + (w == 0 ? C::s_col(gs & 1) : C::DP_COL);
 #pragma unroll
-                for (int w = 0; w < 2; ++w) {
-                    const uint32_t b0 = smem_desc_lo(sT(st, w), 16);
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t offa = ((kk >> 2) * BT * 128 + (kk & 3) * 32) >> 4;
-                        const uint32_t offb = ((kk >> 2) * BS * 128 + (kk & 3) * 32) >> 4;
-                        if constexpr (A_TMEM)
-                            mma_f16_ts_lohi(tmem + (w == 0 ? C::S_COL : C::DP_COL), tmem + C::rt_col(w) + kk * 8, b0 + offb, DESC_HI, IDESC_S, kk > 0);
-                        else
-                            mma_f16_ss_lohi(tmem + (w == 0 ? C::S_COL : C::DP_COL), r_lo[w] + offa, b0 + offb, DESC_HI, IDESC_S, kk > 0);
-                    }
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t offa = ((kk >> 2) * BT * 128 + (kk & 3) * 32) >> 4;
+                    const uint32_t offb = ((kk >> 2) * BS * 128 + (kk & 3) * 32) >> 4;
+                    if constexpr (A_TMEM)
+                        mma_f16_ts_lohi(dcol, tmem + C::rt_col(w) + kk * 8, b0 + offb, DESC_HI, IDESC_S, kk > 0);
+                    else
+                        mma_f16_ss_lohi(dcol, r_lo[w] + offa, b0 + offb, DESC_HI, IDESC_S, kk > 0);
                 }
-                mma_commit(bar(B_SFULL + (gs & 1)));
             }
         };
         // accumulating products of global step gs, step u of its tile (contraction step kk, 16 values = 8 columns,
@@ -453,15 +458,26 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         int gs = 0, kk = 0;
         bool ok = true;
         if (warp == 8) {
-            // S and dP of a step as soon as the previous step's are in its group's registers (also across tiles)
+            // dP of a step as soon as the previous step's S and dP are in its group's registers (also across tiles).
+            // With two S buffers the S of a step was issued one step earlier, behind the previous dP (the first step of
+            // a tile excepted: its resident operand is only then in place); the buffer it goes into was read two
+            // steps ago.  With one buffer S and dP are issued together.
             for (int k = next_work(0, leader, t); k >= 0 && ok; k = next_work(k + 1, leader, t), ++kk) {
                 if (!(ok = mbar_wait(bar(A_TMEM ? B_RTMEM : B_RFULL), kk & 1, abort_flag))) break;
                 for (int u = 0; u < t.n_steps; ++u, ++gs) {
                     if (gs > 0 && !(ok = mbar_wait(bar(B_SREAD + ((gs - 1) & 1)), ((gs - 1) >> 1) & 1, abort_flag))) break;
-                    if (!(ok = mbar_wait(bar(B_TFULL + gs % NSTAGE), (gs / NSTAGE) & 1, abort_flag))) break;
+                    const bool s_pending = !C::S2BUF || u == 0;
+                    if (s_pending && !(ok = mbar_wait(bar(B_TFULL + gs % NSTAGE), (gs / NSTAGE) & 1, abort_flag))) break;
                     tc_fence_after_sync();
-                    issue_s(gs);
-                    if (u + 1 == t.n_steps && leader) mma_commit(bar(B_SLAST));
+                    if (s_pending) issue_prod(gs, 0);
+                    issue_prod(gs, 1);
+                    if (leader) mma_commit(bar(B_SFULL + (gs & 1)));
+                    if (u + 1 == t.n_steps) {
+                        if (leader) mma_commit(bar(B_SLAST));
+                    } else if (C::S2BUF) {
+                        if (!(ok = mbar_wait(bar(B_TFULL + (gs + 1) % NSTAGE), ((gs + 1) / NSTAGE) & 1, abort_flag))) break;
+                        issue_prod(gs + 1, 0);
+                    }
                 }
             }
         } else {
@@ -489,7 +505,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR0, const __grid_constant_
         const int half = grp;                                // epilogue: which 32 of every 64 output columns
         const int r = (warp & 3) * 32 + lane;                // tensor-memory lane: query row (MODE 0) / key row (MODE 1)
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + C::S_COL + lane_off, tDP = tmem + C::DP_COL + lane_off;
+        const uint32_t tS = tmem + C::s_col(grp) + lane_off, tDP = tmem + C::DP_COL + lane_off;   // own S buffer: steps of parity grp
         const uint32_t tOP = tmem + C::op_col(grp) + lane_off;
         const float c = prm.scale_log2;
         const uint64_t c2 = pack_f32x2(c, c);

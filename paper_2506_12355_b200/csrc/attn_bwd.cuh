@@ -25,11 +25,12 @@
 // MODE 1 at D = 128) the resident tiles are copied into tensor memory once and are the A operand of the S / dP
 // products from there; with both operands in shared memory those products are paced by shared-memory bandwidth.
 //
-// The streamed side advances 64 rows per step.  The fp32 S / dP tiles of a step (128 lanes x 64 columns each)
-// have ONE place in tensor memory, which an element-wise group frees as soon as it has the tile in registers;
-// the 16-bit operands it makes from them go to one of two small operand regions.  So while a group computes,
-// the tensor core already produces S and dP of the next step for the other group, and the accumulating products
-// of a step run whenever its operands are ready.
+// The streamed side advances 64 rows per step.  The fp32 dP tile of a step (128 lanes x 64 columns) has ONE place
+// in tensor memory, the S tile one or (wherever 64 columns are left: everywhere but MODE 1 at D = 128) two, which an
+// element-wise group frees as soon as it has the tiles in registers; the 16-bit operands it makes from them go to one
+// of two small operand regions.  So while a group computes, the tensor core already produces S and dP of the next
+// step for the other group (with two S buffers the next S directly behind the current dP, before the current step has
+// even been read), and the accumulating products of a step run whenever its operands are ready.
 //
 //   warps 0-3  element-wise group of the even steps (one thread per tensor-memory lane); both groups then run the
 //   warps 4-7  element-wise group of the odd steps                                          epilogue together

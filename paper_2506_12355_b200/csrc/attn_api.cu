@@ -325,6 +325,7 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
         prm.last_group = static_cast<int>(n_groups >= merge ? n_groups - merge : 0);
     }
     prm.n_items = static_cast<int>(n_pairs * BH * n_splits);
+    prm.halves_from = 2147483647;
     prm.n_splits = n_splits;
     {
         const int tiles = (Sk + C::BN - 1) / C::BN;
@@ -339,6 +340,16 @@ int launch_tc_pipe(const void* q, const void* k, const void* v, void* o, float* 
     DeviceInfo di;
     int dev = 0;
     if (device_info(&di, &dev) != ATTN_OK) return ATTN_ERR_CUDA;
+    // Without a mask all items are equally long (whole keys, n_splits == 1): when the last wave would occupy at most
+    // half of the CTAs, its items are cut into their two Q tiles (a tile alone runs a step in ~83 % of the time of
+    // two in ping-pong, so the launch ends after ~0.83 instead of 1 more item time).
+    if (!causal && n_splits == 1 && Sq >= 2 * C::BM && prm.n_items > di.sm_count && prm.n_items < 2147483647 - di.sm_count) {
+        const int rem = prm.n_items % di.sm_count;
+        if (rem > 0 && 2 * rem <= di.sm_count) {
+            prm.halves_from = prm.n_items - rem;
+            prm.n_items += rem;
+        }
+    }
     const unsigned grid = static_cast<unsigned>(prm.n_items < di.sm_count ? prm.n_items : di.sm_count);
     prm.counter = nullptr;   // small problems: every CTA takes exactly one item, no counter
     if (prm.n_items > di.sm_count) {

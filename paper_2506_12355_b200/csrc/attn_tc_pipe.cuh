@@ -67,7 +67,10 @@ struct PipeParams {
     int last_group;         // index of the final group, which takes all remaining heads
     int H, Hkv;             // query heads and key/value heads per batch element (H % Hkv == 0)
     int k_offset;           // global index of key 0 of this K/V shard (0 for whole problems); enters the causal mask
-    int n_items;            // n_pairs * BH * n_splits
+    int n_items;            // work items: n_pairs * BH * n_splits, plus one for every item at or beyond halves_from
+    int halves_from;        // items from this index on are cut into their two Q tiles (each half a work item of its own,
+                            // consecutive indices); INT_MAX: none.  Used when the last wave of a launch of equally long
+                            // items would leave more than half of the CTAs without work.
     int n_splits;           // key ranges per (head, Q tile pair): 1, or more for split-KV decoding, where range s of
     int split_tiles;        // split_tiles K/V tiles writes its partial result as head s * BH + bh of o and lse
     unsigned int* counter;  // work counter {next item, CTAs done}, zero at launch and again at exit:
@@ -87,7 +90,8 @@ struct PipeItem {
     int bh, kv_bh, q0;
     int k_tile0;   // first K/V tile of this item's key range (0 unless the keys are split)
     int o_bh;      // head index of the item's rows in o and lse (bh unless the keys are split)
-    int n_kv0, n_kv1;   // K/V tiles each Q tile needs (0: tile beyond Sq, or no visible key).  Two scalars, not an
+    int n_kv0, n_kv1;   // K/V tiles each Q tile needs (0: tile beyond Sq, or no visible key; -1: the tile belongs to
+                        // another work item and nothing of it is touched).  Two scalars, not an
                         // array: an array indexed by a run-time tile number puts the whole item into local memory,
                         // and the MMA warp then reads its loop bounds from there on every step.
     __device__ __forceinline__ int nkv(int t) const { return t ? n_kv1 : n_kv0; }
@@ -96,6 +100,13 @@ struct PipeItem {
 
 __device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int lin_all, int BM, int BN) {
     PipeItem it;
+    // the tail of the item order may consist of half items: two consecutive indices per (head, Q tile pair)
+    int only_tile = -1;
+    if (lin_all >= prm.halves_from) {
+        const int h = lin_all - prm.halves_from;
+        only_tile = h & 1;
+        lin_all = prm.halves_from + (h >> 1);
+    }
     // the key ranges of one (head, Q tile pair) are neighbours in the item order
     const int split = lin_all % prm.n_splits;
     const int lin = lin_all / prm.n_splits;
@@ -122,6 +133,7 @@ __device__ __forceinline__ PipeItem pipe_decode_item(const PipeParams& prm, int 
         int in_range = n - split * prm.split_tiles;
         if (in_range > prm.split_tiles) in_range = prm.split_tiles;
         n = in_range < 0 ? 0 : in_range;
+        if (only_tile >= 0 && only_tile != t) n = -1;
         if (t == 0) it.n_kv0 = n; else it.n_kv1 = n;
     }
     it.k_tile0 = split * prm.split_tiles;
@@ -417,7 +429,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 kv_base += 2 * it.n_max;
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
-                    it_base[t] += it.nkv(t);
+                    it_base[t] += it.nkv(t) > 0 ? it.nkv(t) : 0;
                     uses[t] += it.nkv(t) > 0 ? 1 : 0;
                 }
             }
@@ -447,9 +459,10 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             const int n = it.nkv(t);
             const int q0 = it.q0;
             const int row = q0 + t * BM + r;
-            if (n == 0) {
-                // beyond Sq, or (K/V shards under the causal mask) rows that see no key: O = 0, LSE = -inf
-                if (row < prm.Sq) {
+            if (n <= 0) {
+                // beyond Sq, or (K/V shards under the causal mask) rows that see no key: O = 0, LSE = -inf;
+                // n < 0: the tile is another work item's
+                if (n == 0 && row < prm.Sq) {
                     const int64_t grow0 = static_cast<int64_t>(it.o_bh) * prm.Sq + row;
                     uint4* orow0 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(prm.o) + grow0 * D * 2);
 #pragma unroll

@@ -394,6 +394,30 @@ def test_many_short_items_match_cross_check_kernel():
     assert float((l1 - l2).abs().max()) <= 2 * LSE_TOL
 
 
+@pytest.mark.parametrize("B,H,S,D,dtype", [(3, 25, 1000, 128, 0), (8, 20, 1024, 64, 1), (1, 50, 1000, 128, 1), (5, 31, 300, 64, 0)])
+def test_last_wave_cut_into_half_items(B, H, S, D, dtype):
+    # Without a mask, when the last wave of equally long work items would occupy at most half of the SMs, its
+    # items are cut into their two Q tiles (each half a work item of its own that must leave the other tile's
+    # rows alone).  Shapes whose item count modulo the SM count is small, with ragged last tiles; every row of
+    # every head against the oracle, outputs pre-filled with NaN.
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    items = B * H * ((S + 255) // 256)
+    assert items > sms and 0 < items % sms <= sms // 2, "the shape no longer exercises the half items on this GPU"
+    scale = f32_scale(D)
+    q, k, v = inputs.make_qkv(B, H, S, S, D, dtype, seed=4242)
+    o, lse = run_gpu(api.attn_fwd, q, k, v, scale, False)
+    assert not torch.isnan(o.float()).any() and not torch.isnan(lse).any(), "rows left unwritten"
+    qb, kb, vb = (inputs.bits(t) for t in (q, k, v))
+    worst_o = worst_l = 0.0
+    for bh in range(B * H):
+        rows = np.arange(bh * S, (bh + 1) * S, dtype=np.int64)
+        o_ref, l_ref = orc.attention_rows_16(qb, kb, vb, dtype, rows, scale, False)
+        worst_o = max(worst_o, float(np.abs(o.view(-1, D)[rows].double().numpy() - o_ref).max()))
+        worst_l = max(worst_l, float(np.abs(lse.view(-1)[rows].double().numpy() - l_ref).max()))
+    assert worst_o <= O_TOL[dtype], "max |dO| = %g" % worst_o
+    assert worst_l <= LSE_TOL, "max |dLSE| = %g" % worst_l
+
+
 def test_launches_on_two_streams_do_not_share_a_work_counter():
     dev = torch.device("cuda:0")
     cases = []

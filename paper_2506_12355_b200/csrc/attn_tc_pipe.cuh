@@ -19,7 +19,9 @@
 // L2-sized groups of heads; the first item of a CTA is its block index, later ones come from a
 // global counter (zeroed by the host before the launch).  Barriers, tensor memory and the K/V ring
 // live across items, so the producer already loads the next item's Q/K/V and the MMA warp already
-// issues its first S while the softmax groups still write the previous item's O.
+// issues its first S while the softmax groups still write the previous item's O.  Without a mask
+// (equally long items) a last wave that would fill at most half of the SMs is cut into single-tile
+// items, which the host announces through PipeParams::halves_from.
 //
 // Running maximum: the reference maximum m of a row is only advanced when the true maximum has
 // grown by more than 2^8; otherwise the stale m is kept (P values up to 256, exact after the final

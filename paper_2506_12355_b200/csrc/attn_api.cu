@@ -587,7 +587,8 @@ extern "C" {
 
 #ifdef ATTN_TEST_HOOKS
 // Test build only (never part of libattn_fwd.so): the next launch of the pipelined kernel leaves out the load
-// of this K/V ring item, so that the wait for it runs out and the kernel returns through its time-out path.
+// of this K/V ring group (group 0 of a work item is K_0, group i is V_{i-1} with K_i), so that the wait for it runs out
+// and the kernel returns through its time-out path.
 void attn_test_skip_kv_load(int ring_item) { g_test_skip_ring_item = ring_item; }
 #endif
 

@@ -17,7 +17,7 @@
 //
 // Persistence: the grid has one CTA per SM.  Items are ordered longest-first (causal) inside
 // L2-sized groups of heads; the first item of a CTA is its block index, later ones come from a
-// global counter (zeroed by the host before the launch).  Barriers, tensor memory and the K/V ring
+// device counter (zero at launch: the last CTA of the previous user resets it).  Barriers, tensor memory and the K/V ring
 // live across items, so the producer already loads the next item's Q/K/V and the MMA warp already
 // issues its first S while the softmax groups still write the previous item's O.  Without a mask
 // (equally long items) a last wave that would fill at most half of the SMs is cut into single-tile
@@ -43,7 +43,7 @@ struct PipeCfg {
     static constexpr int BOX_COLS = 128 / ES;            // elements per box row
     static constexpr int Q_BYTES = BM * D * ES;
     static constexpr int KV_BYTES = BN * D * ES;
-    static constexpr int NSLOT = (KV_BYTES == 32768) ? 4 : 8;   // ring slots (each holds one K or V tile)
+    static constexpr int NSLOT = (KV_BYTES == 32768) ? 4 : 8;   // ring tile slots (each holds one K or V tile); two of them form a group slot: V_j and K_{j+1}
     static_assert(NBOX >= 1 && (D * ES) % 128 == 0, "tile rows must be whole 128-byte boxes");
     static constexpr int OST_BYTES = BM * 128;           // epilogue staging per Q tile: 128 rows x 64 columns
     static constexpr int TILE_BYTES = 2 * Q_BYTES + NSLOT * KV_BYTES + 2 * OST_BYTES;
@@ -78,7 +78,7 @@ struct PipeParams {
     unsigned int* counter;  // work counter {next item, CTAs done}, zero at launch and again at exit:
                             // item = gridDim.x + atomicAdd(counter, 1); NULL when n_items <= grid
 #ifdef ATTN_TEST_HOOKS
-    int test_skip_ring_item;  // test build only: the K/V ring item whose load the producer leaves out (-1: none)
+    int test_skip_ring_item;  // test build only: the K/V ring group whose loads the producer leaves out (-1: none)
 #endif
 };
 
@@ -165,6 +165,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     constexpr float LAG = FP8 ? 3.f : 8.f;
     using C = PipeCfg<D, ES>;
     constexpr int BM = C::BM, BN = C::BN, NBOX = C::NBOX, NSLOT = C::NSLOT;
+    constexpr int NGRP = NSLOT / 2;   // ring groups in flight (two tile slots each)
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -262,7 +263,7 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         if (warp == 9) {
             // =========================== scheduler + TMA producer ===========================
             const bool leader = elect_one();
-            int kv_base = 0;            // ring items issued for earlier work items
+            int kv_base = 0;            // ring groups issued for earlier work items
             int q_uses[2] = {0, 0};     // work items that loaded Q tile t so far
             // Draws the k-th work item of this CTA, decodes it and publishes it in scheduler slot k & 3.
             // (Drawing one item ahead was measured and is slower: the CTAs finish less evenly.)
@@ -308,30 +309,42 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     ++q_uses[t];
                     return true;
                 };
-                auto load_kv = [&](const CUtensorMap* map, int ring_item, int j) -> bool {
-                    const int s = ring_item % NSLOT;
-                    const uint32_t use = ring_item / NSLOT;
-                    if (!mbar_wait(bar(B_KVEMPTY + s), (use & 1) ^ 1, abort_flag)) return false;
+                // Ring group i of an item (n = n_max steps): {K_0} for i = 0, {V_{i-1}, K_i} for 0 < i < n, {V_{n-1}} for
+                // i = n: what the MMA warp needs together for step i - 1 (O += P V_{i-1}, then S = Q K_i^T).  One full
+                // and one empty barrier per group; group slot g holds V in tile slot 2 g and K in tile slot 2 g + 1.
+                auto load_group = [&](int group, int i) -> bool {
+                    const int g = group % NGRP;
+                    const uint32_t use = group / NGRP;
+                    if (!mbar_wait(bar(B_KVEMPTY + g), (use & 1) ^ 1, abort_flag)) return false;
 #ifdef ATTN_TEST_HOOKS
-                    if (ring_item == prm.test_skip_ring_item) return true;   // this slot's "full" barrier never completes
+                    if (group == prm.test_skip_ring_item) return true;   // this group's "full" barrier never completes
 #endif
                     if (leader) {
-                        mbar_arrive_expect_tx(bar(B_KVFULL + s), C::KV_BYTES);
+                        const bool has_v = i > 0, has_k = i < it.n_max;
+                        mbar_arrive_expect_tx(bar(B_KVFULL + g), (has_v ? C::KV_BYTES : 0) + (has_k ? C::KV_BYTES : 0));
+                        if (has_v) {
 #pragma unroll
-                        for (int bx = 0; bx < NBOX; ++bx)
-                            tma_load_3d(sKV(s) + bx * BN * 128, map, bar(B_KVFULL + s), bx * C::BOX_COLS, (it.k_tile0 + j) * BN, it.kv_bh);
+                            for (int bx = 0; bx < NBOX; ++bx)
+                                tma_load_3d(sKV(2 * g) + bx * BN * 128, &tmV, bar(B_KVFULL + g), bx * C::BOX_COLS, (it.k_tile0 + i - 1) * BN, it.kv_bh);
+                        }
+                        if (has_k) {
+#pragma unroll
+                            for (int bx = 0; bx < NBOX; ++bx)
+                                tma_load_3d(sKV(2 * g + 1) + bx * BN * 128, &tmK, bar(B_KVFULL + g), bx * C::BOX_COLS, (it.k_tile0 + i) * BN, it.kv_bh);
+                        }
                     }
                     return true;
                 };
                 bool ok = true;
                 if (it.n_kv0 > 0) ok = load_q(0);
-                for (int j = 0; j < it.n_max && ok; ++j) {
-                    ok = load_kv(&tmK, kv_base + 2 * j, j);
-                    if (ok && j == 0 && it.n_kv1 > 0) ok = load_q(1);
-                    if (ok) ok = load_kv(&tmV, kv_base + 2 * j + 1, j);
+                if (it.n_max > 0) {
+                    for (int i = 0; i <= it.n_max && ok; ++i) {
+                        ok = load_group(kv_base + i, i);
+                        if (ok && i == 0 && it.n_kv1 > 0) ok = load_q(1);
+                    }
                 }
                 if (!ok) break;
-                kv_base += 2 * it.n_max;
+                if (it.n_max > 0) kv_base += it.n_max + 1;
             }
         } else if (warp == 8) {
             // =========================== MMA issuer ===========================
@@ -372,8 +385,8 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             auto commit = [&](int b) {
                 if (leader) mma_commit(bar(b));
             };
-            auto kv_full_wait = [&](int ring_item) {
-                return mbar_wait(bar(B_KVFULL + ring_item % NSLOT), (ring_item / NSLOT) & 1, abort_flag);
+            auto kv_full_wait = [&](int group) {   // both tiles of a ring group are loaded
+                return mbar_wait(bar(B_KVFULL + group % NGRP), (group / NGRP) & 1, abort_flag);
             };
             int kv_base = 0;
             int it_base[2] = {0, 0};   // K/V steps tile t has gone through in earlier work items
@@ -391,19 +404,18 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         ok = mbar_wait(bar(B_QFULL + t), uses[t] & 1, abort_flag);
                         if (ok) {
                             tc_fence_after_sync();
-                            issue_s(t, kv_base % NSLOT);
+                            issue_s(t, 2 * (kv_base % NGRP) + 1);
                             commit(B_SFULL + t);
                             if (it.nkv(t) == 1) commit(B_QEMPTY + t);
                         }
                     }
                 }
-                if (ok && it.n_max > 0) commit(B_KVEMPTY + kv_base % NSLOT);
+                if (ok && it.n_max > 0) commit(B_KVEMPTY + kv_base % NGRP);
                 for (int j = 0; j < it.n_max && ok; ++j) {
-                    const int vitem = kv_base + 2 * j + 1, kitem = kv_base + 2 * j + 2;
-                    const int vslot = vitem % NSLOT, kslot = kitem % NSLOT;
-                    // both tiles of this step are normally long loaded: check them off the P -> S critical path
-                    if (!(ok = kv_full_wait(vitem))) break;
-                    if (j + 1 < it.n_max && !(ok = kv_full_wait(kitem))) break;
+                    // V_j and K_{j+1} are one ring group: one wait, one release
+                    const int gslot = (kv_base + j + 1) % NGRP;
+                    const int vslot = 2 * gslot, kslot = 2 * gslot + 1;
+                    if (!(ok = kv_full_wait(kv_base + j + 1))) break;
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
                         if (j < it.nkv(t)) {
@@ -418,7 +430,6 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                             issue_pv(t, vslot, true, 3 * (BN / KSTEP) / 4, BN / KSTEP);
                             if (j + 1 == it.nkv(t)) commit(B_OFINAL + t);
                         }
-                        if (t == 1) commit(B_KVEMPTY + vslot);
                         if (j + 1 < it.nkv(t)) {
                             tc_fence_after_sync();
                             issue_s(t, kslot);
@@ -426,9 +437,9 @@ attn_fwd_tc_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                             if (j + 2 == it.nkv(t)) commit(B_QEMPTY + t);   // that was the last S of this item
                         }
                     }
-                    if (ok && j + 1 < it.n_max) commit(B_KVEMPTY + kslot);
+                    if (ok) commit(B_KVEMPTY + gslot);
                 }
-                kv_base += 2 * it.n_max;
+                if (it.n_max > 0) kv_base += it.n_max + 1;
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     it_base[t] += it.nkv(t) > 0 ? it.nkv(t) : 0;

@@ -49,7 +49,7 @@ def test_a_wait_that_runs_out_returns_a_status_and_leaves_no_trace(D, Sq, Sk, ca
     assert call(o_before, l_before) == 0
     assert lib.attn_last_device_status(stream) == 0
 
-    # the producer leaves out ring item `skip` (K and V tiles alternate, K first): its consumer gives up after 1 ms
+    # the producer leaves out ring group `skip` (group 0 is K_0, group i is V_{i-1} with K_i): its consumer gives up after 1 ms
     o_bad, l_bad = torch.empty_like(q), torch.empty_like(l_before)
     lib.attn_test_skip_kv_load(skip)
     assert call(o_bad, l_bad) == 0                                    # the launch itself succeeds
